@@ -1,0 +1,163 @@
+"""Float64 CPU oracle for the pruned-layer path -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper around ``sentry_oracle.c`` (plain C, written from the
+paper).  Only the tests, the smoke check and the benchmark's CPU-baseline /
+reference arm may import this package; the CUDA library never does, and this
+package never imports the CUDA library.
+
+Inputs may be numpy arrays or torch CPU tensors of any float dtype; they are
+widened to float64 exactly (bf16 and fp32 values are representable), so the
+oracle sees the same numbers the GPU reads.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sentry_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over samples).  Returns the path."""
+    with _lock:
+        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+            tmp = _LIB + ".tmp%d" % os.getpid()
+            cmd = ["gcc", "-O2", "-fopenmp", "-std=c99", "-shared", "-fPIC",
+                   "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        lib.oracle_threads.restype = ctypes.c_int
+        lib.oracle_num_active.restype = ctypes.c_int
+        lib.oracle_num_active.argtypes = [ctypes.c_int, ctypes.c_int]
+        lib.oracle_valid_tokens.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _f64(x) -> np.ndarray:
+    if hasattr(x, "detach"):  # torch tensor
+        import torch
+        x = x.detach().to("cpu").to(torch.float64).numpy()
+    return np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+
+
+def _i32(x) -> np.ndarray:
+    if hasattr(x, "detach"):
+        x = x.detach().to("cpu").numpy()
+    return np.ascontiguousarray(np.asarray(x, dtype=np.int32))
+
+
+def _u32(x) -> np.ndarray:
+    if hasattr(x, "detach"):
+        x = x.detach().to("cpu").numpy()
+    return np.ascontiguousarray(np.asarray(x).astype(np.uint32))
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+
+def threads() -> int:
+    return int(_load().oracle_threads())
+
+
+def num_active(T_v: int, c: int = 5) -> int:
+    """U = c * ceil(ln T_v), clamped to [1, T_v] (Section 4.4)."""
+    return int(_load().oracle_num_active(int(T_v), int(c)))
+
+
+def gate_select(scores, masks, k: int) -> np.ndarray:
+    """Top-k units of scores[mask] per mask: score descending, lower index wins
+    ties, NaN last; returned ascending by index.  scores [S, n_units] fp32."""
+    if hasattr(scores, "detach"):
+        scores = scores.detach().to("cpu").numpy()
+    sc = np.ascontiguousarray(np.asarray(scores, dtype=np.float32))
+    mk = _u32(masks)
+    S, n = sc.shape
+    assert 1 <= k <= n and (mk < S).all()
+    kept = np.empty((mk.shape[0], k), dtype=np.int32)
+    _load().oracle_gate_select(_p(sc), S, n, _p(mk), mk.shape[0], int(k), _p(kept))
+    return kept
+
+
+def kv_groups(kept_heads, heads_per_group: int) -> np.ndarray:
+    """Bitmap of referenced KV groups, floor(h / (H_q/H_k)) (Section 4.6)."""
+    kh = _i32(kept_heads)
+    out = np.zeros((kh.shape[0],), dtype=np.uint32)
+    _load().oracle_kv_groups(_p(kh), kh.shape[0], kh.shape[1], int(heads_per_group), _p(out))
+    return out
+
+
+def valid_tokens(ids, mask: int) -> np.ndarray:
+    ids = _i32(ids)
+    out = np.empty((ids.shape[0],), dtype=np.int32)
+    n = _load().oracle_valid_tokens(_p(ids), ids.shape[0], ctypes.c_uint32(int(mask)), _p(out))
+    return out[:n].copy()
+
+
+def attend(Q, K, V, kept_heads, ids, masks, *, c: int = 5, score_mode: int = 0,
+           sample_table=None, table_offsets=None, forced_active=None,
+           return_aux: bool = False):
+    """SentryAttend on the kept heads.  Q [B,Hq,T,d]; K,V [B,Hk,T,d];
+    kept_heads [B,k_h]; ids [T]; masks [B].  Returns O [B,k_h,T,d] float64
+    (and, with return_aux, the active token lists [B,k_h,U_max] padded with -1
+    and the sparsity scores [B,k_h,T], NaN on absent tokens)."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    kh, ids, mk = _i32(kept_heads), _i32(ids), _u32(masks)
+    B, Hq, T, d = Q.shape
+    Hk = K.shape[1]
+    assert K.shape == (B, Hk, T, d) and V.shape == K.shape and Hq % Hk == 0
+    k_h = kh.shape[1]
+    U_max = num_active(T, c)
+    tbl = offs = None
+    if score_mode == 0:
+        tbl = _i32(sample_table)
+        offs = np.ascontiguousarray(np.asarray(table_offsets, dtype=np.int64))
+    fa = None
+    if forced_active is not None:
+        fa = _i32(forced_active)
+        assert fa.shape == (B, k_h, U_max)
+    O = np.empty((B, k_h, T, d), dtype=np.float64)
+    act = np.empty((B, k_h, U_max), dtype=np.int32)
+    msc = np.empty((B, k_h, T), dtype=np.float64)
+    _load().oracle_attend(_p(Q), _p(K), _p(V), B, T, Hq, Hk, d, int(c), _p(kh), k_h,
+                          _p(ids), _p(mk), int(score_mode), _p(tbl), _p(offs),
+                          U_max, _p(fa), _p(O), _p(act), _p(msc))
+    if return_aux:
+        return O, act, msc
+    return O
+
+
+def ffn(X, W1, W2, kept_channels, list_of_sample=None, ids=None, masks=None) -> np.ndarray:
+    """y = gelu_erf(x W1[:, N]) W2[N, :] per row (Section 4.6).  X [B,T,D];
+    W1 [D,F]; W2 [F,D]; kept_channels [n_lists,k_c]."""
+    X, W1, W2 = _f64(X), _f64(W1), _f64(W2)
+    kc = _i32(kept_channels)
+    if kc.ndim == 1:
+        kc = kc[None, :]
+    B, T, D = X.shape
+    F = W1.shape[1]
+    assert W1.shape == (D, F) and W2.shape == (F, D)
+    los = _i32(list_of_sample) if list_of_sample is not None else None
+    ii = _i32(ids) if ids is not None else None
+    mk = _u32(masks) if masks is not None else None
+    Y = np.empty((B, T, D), dtype=np.float64)
+    _load().oracle_ffn(_p(X), _p(W1), _p(W2), B, T, D, F, _p(kc), kc.shape[1],
+                       _p(los), _p(ii), _p(mk), _p(Y))
+    return Y

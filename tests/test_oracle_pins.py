@@ -1,0 +1,366 @@
+"""Pins for the float64 oracle: each check ties a part of it to something other
+than itself -- the paper's worked example, a library routine, a closed form, an
+invariant of the method, or brute force on tiny inputs."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+from scipy.special import erf
+
+import oracle
+import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+RNG = np.random.default_rng(1234)
+
+
+# --------------------------------------------------------------------------- U
+def test_num_active_matches_paper_worked_example():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "num_active_queries.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert rows
+    for T, c, U in rows:
+        assert oracle.num_active(int(T), int(c)) == int(U)
+
+
+def test_num_active_is_natural_log_and_clamped():
+    # log2 would give 35 and log10 15 for T=128: only ln gives the paper's 25
+    assert oracle.num_active(128, 5) not in (35, 15)
+    # thresholds of ceil(ln T) sit at floor(e^k) | floor(e^k)+1
+    for k in range(1, 9):
+        lo = int(math.floor(math.e ** k))
+        assert oracle.num_active(lo, 5) == min(lo, 5 * k)
+        assert oracle.num_active(lo + 1, 5) == min(lo + 1, 5 * (k + 1))
+    assert oracle.num_active(1, 5) == 1       # ln 1 = 0 -> clamp up to 1
+    assert oracle.num_active(3, 5) == 3       # clamp down to T_v
+    assert oracle.num_active(0, 5) == 0
+    vals = [oracle.num_active(t, 5) for t in range(1, 5000)]
+    assert all(b >= a for a, b in zip(vals, vals[1:]))  # non-decreasing in T_v
+
+
+# ------------------------------------------------------------------------ gate
+def _brute_topk(row, k):
+    # definition by a full sort on the key (NaN last, score desc, index asc)
+    keyed = sorted(range(len(row)),
+                   key=lambda i: (1 if math.isnan(row[i]) else 0,
+                                  -row[i] if not math.isnan(row[i]) else 0.0, i))
+    return sorted(keyed[:k])
+
+
+@pytest.mark.parametrize("n,k", [(4, 3), (8, 4), (12, 7), (256, 128), (1536, 614), (5, 5), (7, 1)])
+def test_gate_select_equals_full_sort(n, k):
+    S = 8
+    sc = RNG.standard_normal((S, n)).astype(np.float32)
+    masks = np.array([1, 7, 3, 3, 5], dtype=np.uint32)
+    kept = oracle.gate_select(sc, masks, k)
+    assert kept.shape == (5, k)
+    for r, m in enumerate(masks):
+        assert kept[r].tolist() == _brute_topk(sc[m].tolist(), k)
+
+
+def test_gate_select_equals_library_topk_without_ties():
+    sc = RNG.standard_normal((4, 512)).astype(np.float32)
+    kept = oracle.gate_select(sc, np.array([2], dtype=np.uint32), 100)
+    ref = torch.topk(torch.from_numpy(sc[2]), 100).indices.sort().values.numpy()
+    assert kept[0].tolist() == ref.tolist()
+
+
+def test_gate_select_ties_nan_and_signed_zero():
+    row = np.array([1.0, 2.0, 2.0, np.nan, 2.0, -0.0, 0.0, np.nan, -np.inf], dtype=np.float32)
+    sc = np.stack([row, row])
+    for k, want in [(1, [1]), (2, [1, 2]), (3, [1, 2, 4]), (4, [0, 1, 2, 4]),
+                    (5, [0, 1, 2, 4, 5]),          # -0.0 ties +0.0: lower index first
+                    (6, [0, 1, 2, 4, 5, 6]),
+                    (7, [0, 1, 2, 4, 5, 6, 8]),    # -inf still beats NaN
+                    (8, [0, 1, 2, 3, 4, 5, 6, 8]),  # NaNs tie: lower index first
+                    (9, list(range(9)))]:
+        assert oracle.gate_select(sc, np.array([1], dtype=np.uint32), k)[0].tolist() == want
+
+
+def test_gate_select_permutation_equivariance():
+    n, k = 64, 20
+    row = RNG.standard_normal(n).astype(np.float32)
+    perm = RNG.permutation(n)
+    a = oracle.gate_select(row[None], np.array([0], dtype=np.uint32), k)[0]
+    b = oracle.gate_select(row[perm][None], np.array([0], dtype=np.uint32), k)[0]
+    assert sorted(perm[b].tolist()) == a.tolist()
+
+
+def test_kv_groups_formula_hand_cases():
+    # H_q = 8, H_k = 2 -> 4 heads per group (Section 4.6)
+    kept = np.array([[0, 1, 5], [4, 6, 7], [0, 1, 3]], dtype=np.int32)
+    assert oracle.kv_groups(kept, 4).tolist() == [0b11, 0b10, 0b01]
+    # H_q = 12, H_k = 4 -> 3 per group
+    assert oracle.kv_groups(np.array([[2, 3, 11]], dtype=np.int32), 3).tolist() == [0b1011]
+
+
+# ------------------------------------------------------------------- attention
+def _rand_attn(B, Hq, Hk, T, d, seed=0):
+    g = np.random.default_rng(seed)
+    return (g.standard_normal((B, Hq, T, d)), g.standard_normal((B, Hk, T, d)),
+            g.standard_normal((B, Hk, T, d)))
+
+
+def _identity_table(T, M):
+    """Table whose row i lists every key: sampled mode degenerates to exact mode."""
+    offs = np.zeros((1 << M,), dtype=np.int64)
+    return np.tile(np.arange(T, dtype=np.int32), (T, 1)).reshape(-1), offs
+
+
+def test_dense_limit_equals_library_attention():
+    # c large -> U = T_v: every row is an Eq. 6 row; group size 1; all present
+    B, H, T, d = 2, 3, 24, 8
+    Q, K, V = _rand_attn(B, H, H, T, d)
+    ids = np.zeros((T,), dtype=np.int32)
+    O = oracle.attend(Q, K, V, np.tile(np.arange(H, dtype=np.int32), (B, 1)), ids,
+                      np.ones((B,), dtype=np.uint32), c=1000, score_mode=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q), torch.from_numpy(K), torch.from_numpy(V)).numpy()
+    np.testing.assert_allclose(O, ref, rtol=0, atol=1e-12)
+    # and brute force, written independently
+    for b in range(B):
+        for h in range(H):
+            s = Q[b, h] @ K[b, h].T / math.sqrt(d)
+            p = np.exp(s - s.max(axis=1, keepdims=True))
+            p /= p.sum(axis=1, keepdims=True)
+            np.testing.assert_allclose(O[b, h], p @ V[b, h], rtol=0, atol=1e-12)
+
+
+def test_gqa_equals_duplicated_kv():
+    B, Hq, Hk, T, d = 2, 8, 2, 40, 16
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 3)
+    ids = np.repeat(np.arange(2, dtype=np.int32), T // 2)
+    masks = np.full((B,), 3, dtype=np.uint32)
+    kept = np.tile(np.array([0, 2, 5, 7], dtype=np.int32), (B, 1))
+    O1, a1, _ = oracle.attend(Q, K, V, kept, ids, masks, score_mode=1, return_aux=True)
+    Kd, Vd = np.repeat(K, Hq // Hk, axis=1), np.repeat(V, Hq // Hk, axis=1)
+    O2, a2, _ = oracle.attend(Q, Kd, Vd, kept, ids, masks, score_mode=1, return_aux=True)
+    np.testing.assert_array_equal(a1, a2)
+    np.testing.assert_allclose(O1, O2, rtol=0, atol=0)
+    # library GQA on the active rows only
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q), torch.from_numpy(K), torch.from_numpy(V), enable_gqa=True).numpy()
+    for b in range(B):
+        for j, h in enumerate(kept[b]):
+            rows = a1[b, j][a1[b, j] >= 0]
+            np.testing.assert_allclose(O1[b, j, rows], ref[b, h, rows], rtol=0, atol=1e-12)
+
+
+def test_softmax_rows_sum_to_one_and_fill_is_mean():
+    B, Hq, Hk, T, d = 1, 4, 2, 64, 8
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 5)
+    ids = np.zeros((T,), dtype=np.int32)
+    masks = np.ones((B,), dtype=np.uint32)
+    kept = np.array([[1, 2]], dtype=np.int32)
+    # V = 1 -> every present row must be exactly sum_j p_ij = 1 (active) or mean(1) = 1
+    O = oracle.attend(Q, K, np.ones_like(V), kept, ids, masks, score_mode=1)
+    np.testing.assert_allclose(O, 1.0, rtol=0, atol=1e-12)
+    # non-active rows carry mean(V_g); active rows generally differ from it
+    O, act, _ = oracle.attend(Q, K, V, kept, ids, masks, score_mode=1, return_aux=True)
+    U = oracle.num_active(T)
+    assert (act[0] >= 0).sum(axis=1).tolist() == [U, U]
+    for j, h in enumerate(kept[0]):
+        g = h // 2
+        inactive = np.setdiff1d(np.arange(T), act[0, j])
+        np.testing.assert_allclose(O[0, j, inactive], np.tile(V[0, g].mean(0), (len(inactive), 1)),
+                                   rtol=0, atol=1e-12)
+        assert np.abs(O[0, j, act[0, j]] - V[0, g].mean(0)).max() > 1e-3
+    # K = 0 -> all scores equal -> uniform softmax -> active rows equal the fill vector
+    O0 = oracle.attend(Q, np.zeros_like(K), V, kept, ids, masks, score_mode=1)
+    for j, h in enumerate(kept[0]):
+        np.testing.assert_allclose(O0[0, j], np.tile(V[0, h // 2].mean(0), (T, 1)), rtol=0, atol=1e-12)
+    # shift invariance: adding a constant vector to every key moves s_ij by q_i.const,
+    # constant along j, so each softmax row (and the fill) is unchanged
+    O_shift = oracle.attend(Q, K + 0.37, V, kept, ids, masks, score_mode=1,
+                            forced_active=act)
+    np.testing.assert_allclose(O_shift, O, rtol=0, atol=1e-10)
+
+
+def test_sparsity_score_and_selection_brute_force():
+    B, Hq, Hk, T, d = 2, 4, 2, 16, 4
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 7)
+    ids = np.zeros((T,), dtype=np.int32)
+    masks = np.ones((B,), dtype=np.uint32)
+    kept = np.tile(np.array([0, 3], dtype=np.int32), (B, 1))
+    U = oracle.num_active(T)              # 5*ceil(ln 16)=15
+    assert U == 15
+    g = np.random.default_rng(11)
+    n_s = U                                # one sampled key per retained query, as the method prescribes
+    table = np.stack([np.sort(g.choice(T, n_s, replace=False)) for _ in range(T)]).astype(np.int32)
+    offs = np.zeros((2,), dtype=np.int64)
+    O, act, msc = oracle.attend(Q, K, V, kept, ids, masks, score_mode=0,
+                                sample_table=table.reshape(-1), table_offsets=offs, return_aux=True)
+    for b in range(B):
+        for j, h in enumerate(kept[b]):
+            s = Q[b, h] @ K[b, h // 2].T / math.sqrt(d)
+            M = np.array([s[i, table[i]].max() - s[i, table[i]].mean() for i in range(T)])
+            np.testing.assert_allclose(msc[b, j], M, rtol=0, atol=1e-12)
+            order = sorted(range(T), key=lambda i: (-M[i], i))[:U]
+            assert sorted(order) == act[b, j].tolist()
+    # exact mode scores every query on all keys
+    _, _, ma = oracle.attend(Q, K, V, kept, ids, masks, score_mode=1, return_aux=True)
+    s = Q[0, 0] @ K[0, 0].T / math.sqrt(d)
+    np.testing.assert_allclose(ma[0, 0], s.max(1) - s.mean(1), rtol=0, atol=1e-12)
+    # a table that lists every key (n_s = U = T_v, reached with a large c) is the exact mode
+    tbl, offs1 = _identity_table(T, 1)
+    Oe, ae, me = oracle.attend(Q, K, V, kept, ids, masks, c=100, score_mode=1, return_aux=True)
+    Ot, at, mt = oracle.attend(Q, K, V, kept, ids, masks, c=100, score_mode=0, sample_table=tbl,
+                               table_offsets=offs1, return_aux=True)
+    np.testing.assert_array_equal(me, mt)
+    np.testing.assert_array_equal(Oe, Ot)
+
+
+def test_selection_ties_go_to_lower_index():
+    # identical queries -> identical M -> the first U tokens are selected
+    B, Hq, Hk, T, d = 1, 2, 1, 32, 4
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 9)
+    Q[:] = Q[:, :, :1, :]
+    O, act, _ = oracle.attend(Q, K, V, np.array([[0, 1]], dtype=np.int32),
+                              np.zeros((T,), dtype=np.int32), np.ones((1,), dtype=np.uint32),
+                              score_mode=1, return_aux=True)
+    U = oracle.num_active(T)
+    assert act[0, 0].tolist() == list(range(U)) and act[0, 1].tolist() == list(range(U))
+
+
+def test_pruned_heads_are_absent_and_kept_heads_unchanged():
+    B, Hq, Hk, T, d = 2, 8, 2, 48, 8
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 13)
+    ids = np.repeat(np.arange(3, dtype=np.int32), T // 3)
+    masks = np.array([7, 5], dtype=np.uint32)
+    full = np.tile(np.arange(Hq, dtype=np.int32), (B, 1))
+    kept = np.array([[1, 4, 6], [0, 2, 3]], dtype=np.int32)
+    Of = oracle.attend(Q, K, V, full, ids, masks, score_mode=1)
+    Ok = oracle.attend(Q, K, V, kept, ids, masks, score_mode=1)
+    for b in range(B):
+        np.testing.assert_array_equal(Ok[b], Of[b, kept[b]])
+    # a head that is pruned has no influence: perturbing it changes nothing
+    Q2 = Q.copy()
+    Q2[0, 0] += 5.0
+    Q2[0, 7] -= 3.0
+    np.testing.assert_array_equal(oracle.attend(Q2, K, V, kept, ids, masks, score_mode=1)[0], Ok[0])
+
+
+def test_dropping_a_modality_equals_deleting_its_tokens():
+    w = synth.config1()
+    B, Hq, Hk, T, d = 2, 4, 2, 32, 16
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 17)
+    ids = synth.token_modality_ids(w)
+    kept = np.array([[0, 1, 3], [0, 2, 3]], dtype=np.int32)
+    g = np.random.default_rng(19)
+    for mask in (1, 2):
+        keep_t = np.nonzero((mask >> ids) & 1)[0]
+        Tv = len(keep_t)
+        n_s = oracle.num_active(Tv)
+        table = np.stack([np.sort(g.choice(Tv, n_s, replace=False)) for _ in range(Tv)]).astype(np.int32)
+        offs = np.zeros((4,), dtype=np.int64)
+        masks = np.full((B,), mask, dtype=np.uint32)
+        O_drop, a_drop, _ = oracle.attend(Q, K, V, kept, ids, masks, sample_table=table.reshape(-1),
+                                          table_offsets=offs, return_aux=True)
+        # physically shortened tensors, all tokens present, same table
+        O_del, a_del, _ = oracle.attend(Q[:, :, keep_t], K[:, :, keep_t], V[:, :, keep_t], kept,
+                                        np.zeros((Tv,), dtype=np.int32),
+                                        np.ones((B,), dtype=np.uint32),
+                                        sample_table=table.reshape(-1),
+                                        table_offsets=np.zeros((2,), dtype=np.int64), return_aux=True)
+        np.testing.assert_array_equal(O_drop[:, :, keep_t], O_del)
+        gone = np.setdiff1d(np.arange(T), keep_t)
+        assert np.all(O_drop[:, :, gone] == 0.0)       # rows of absent tokens are zero
+        U = oracle.num_active(Tv)
+        np.testing.assert_array_equal(keep_t[a_del[:, :, :U]], a_drop[:, :, :U])
+        # absent tokens' K/V content is irrelevant
+        K2, V2 = K.copy(), V.copy()
+        K2[:, :, gone] = 99.0
+        V2[:, :, gone] = -99.0
+        np.testing.assert_array_equal(
+            oracle.attend(Q, K2, V2, kept, ids, masks, sample_table=table.reshape(-1),
+                          table_offsets=offs), O_drop)
+
+
+def test_output_length_preserved_and_flop_scaling():
+    # every present position gets a row (Section 4.4: output length preserved)
+    B, Hq, Hk, T, d = 1, 2, 1, 128, 4
+    Q, K, V = _rand_attn(B, Hq, Hk, T, d, 23)
+    O, act, _ = oracle.attend(Q, K, V, np.array([[0, 1]], dtype=np.int32),
+                              np.zeros((T,), dtype=np.int32), np.ones((1,), dtype=np.uint32),
+                              score_mode=1, return_aux=True)
+    assert O.shape == (1, 2, T, d) and np.isfinite(O).all()
+    assert (act[0] >= 0).sum(axis=1).tolist() == [25, 25]   # U(128) = 25, the paper's example
+    assert np.all(np.diff(act[0, 0]) > 0)                    # ascending, distinct
+
+
+# ------------------------------------------------------------------------- FFN
+def _gelu(z):
+    return 0.5 * z * (1.0 + erf(z / math.sqrt(2.0)))
+
+
+def test_ffn_equals_library_matmul_on_sliced_weights():
+    g = np.random.default_rng(29)
+    B, T, D, F, k = 3, 10, 24, 64, 20
+    X, W1, W2 = g.standard_normal((B, T, D)), g.standard_normal((D, F)) * 0.2, g.standard_normal((F, D)) * 0.2
+    kept = np.stack([np.sort(g.choice(F, k, replace=False)) for _ in range(2)]).astype(np.int32)
+    los = np.array([1, 0, 1], dtype=np.int32)
+    Y = oracle.ffn(X, W1, W2, kept, los)
+    for b in range(B):
+        N = kept[los[b]]
+        ref = _gelu(X[b] @ W1[:, N]) @ W2[N, :]
+        np.testing.assert_allclose(Y[b], ref, rtol=0, atol=1e-12)
+        # same thing as the full FFN with pruned hidden units gated to zero (gelu(0) = 0)
+        gate = np.zeros(F)
+        gate[N] = 1.0
+        ref_masked = (_gelu(X[b] @ W1) * gate) @ W2
+        np.testing.assert_allclose(Y[b], ref_masked, rtol=0, atol=1e-12)
+    # keeping every channel reproduces the unpruned FFN
+    Yall = oracle.ffn(X, W1, W2, np.arange(F, dtype=np.int32)[None])
+    np.testing.assert_allclose(Yall, _gelu(X @ W1) @ W2, rtol=0, atol=1e-12)
+    # library gelu in float64 as a second opinion on the activation
+    z = torch.from_numpy(X[0] @ W1)
+    np.testing.assert_allclose(_gelu(z.numpy()), torch.nn.functional.gelu(z).numpy(), rtol=0, atol=1e-14)
+
+
+def test_ffn_pruned_channel_contributes_zero_and_dropped_rows_are_zero():
+    g = np.random.default_rng(31)
+    B, T, D, F, k = 2, 8, 16, 32, 10
+    X, W1, W2 = g.standard_normal((B, T, D)), g.standard_normal((D, F)), g.standard_normal((F, D))
+    kept = np.sort(g.choice(F, k, replace=False)).astype(np.int32)[None]
+    Y = oracle.ffn(X, W1, W2, kept)
+    pruned = np.setdiff1d(np.arange(F), kept[0])
+    W1b, W2b = W1.copy(), W2.copy()
+    W1b[:, pruned] += 7.0
+    W2b[pruned, :] -= 7.0
+    np.testing.assert_array_equal(oracle.ffn(X, W1b, W2b, kept), Y)
+    ids = np.repeat(np.arange(2, dtype=np.int32), T // 2)
+    masks = np.array([1, 3], dtype=np.uint32)
+    Ym = oracle.ffn(X, W1, W2, kept, None, ids, masks)
+    assert np.all(Ym[0, T // 2:] == 0.0)
+    np.testing.assert_array_equal(Ym[0, :T // 2], Y[0, :T // 2])
+    np.testing.assert_array_equal(Ym[1], Y[1])
+
+
+# ------------------------------------------------------------ input generators
+def test_generators_are_seeded_and_shaped_like_the_configs():
+    w = synth.config1()
+    a = synth.generate(w, oracle.num_active)
+    b = synth.generate(w, oracle.num_active)
+    assert torch.equal(a.Q, b.Q) and np.array_equal(a.sample_table, b.sample_table)
+    assert a.Q.shape == (2, 4, 32, 16) and a.K.shape == (2, 2, 32, 16) and a.X.shape == (2, 32, 64)
+    assert a.W1.shape == (64, 256) and a.scores_heads.shape == (4, 4) and a.masks.tolist() == [3, 3]
+    assert (w.k_h, w.k_c) == (3, 128)
+    w2, w4 = synth.config2(), synth.config4()
+    assert (w2.k_h, w2.k_c, w4.k_h, w4.k_c) == (4, 256, 7, 614)
+    m2 = synth.make_masks(w2, np.random.default_rng(1))
+    assert m2.min() >= 1 and m2.max() <= 7 and len(m2) == 256
+    m4 = synth.make_masks(w4, np.random.default_rng(3))
+    assert [(m4 == s).sum() for s in (1, 2, 3)] == [43, 43, 42]
+    w5 = synth.config5(16, 64)
+    assert w5.lengths == (22, 21, 21)
+    assert synth.make_masks(w5, np.random.default_rng(4)).tolist() == [1 + b % 7 for b in range(16)]
+    i5 = synth.generate(w5, oracle.num_active, tensors=False)
+    for s in range(1, 8):
+        tv = synth.present_count(w5, s)
+        n_s = oracle.num_active(tv)
+        off = i5.table_offsets[s]
+        tbl = i5.sample_table[off:off + tv * n_s].reshape(tv, n_s)
+        assert tbl.min() >= 0 and tbl.max() < tv
+        assert np.all(np.diff(tbl, axis=1) > 0)      # distinct, ascending
