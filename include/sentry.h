@@ -1,0 +1,202 @@
+/*
+ * sentry.h -- C ABI of libsentry: inference through a deployment-pruned
+ * multimodal transformer layer on one NVIDIA B200 (sm_100a).
+ *
+ * Three operations, in the order a pruned layer uses them:
+ *   sentry_gate_select  modality-conditioned selection of the attention heads
+ *                       and FFN channels to keep         (SentryGate, Sec. 4.6)
+ *   sentry_attend_fwd   sparse grouped-query attention over the kept heads
+ *                       (SentryAttend, Sec. 4.4, Eq. 6)
+ *   sentry_ffn_fwd      feed-forward block over the kept channels only
+ *                       (Sec. 4.6: W1' = W1[:, N_keep], W2' = W2[N_keep, :])
+ *
+ * Conventions
+ *   - Every tensor argument is a caller-owned DEVICE pointer unless it says
+ *     "host".  The library never allocates or frees tensors; scratch comes
+ *     from a caller-provided workspace (sentry_set_workspace).
+ *   - All calls enqueue work on the CUDA stream passed as `stream`
+ *     (a cudaStream_t cast to void*, NULL = default stream) and return without
+ *     synchronising.  Calls that share a context and its workspace must be
+ *     ordered on one stream (or otherwise not overlap).
+ *   - Return value: 0 = SENTRY_OK, negative = error found on the host BEFORE any
+ *     launch (nothing was enqueued).  Conditions only the device can see (a
+ *     sample with an empty modality mask, a bounded wait that ran out) are
+ *     OR-ed into a device status word, read with sentry_get_last_status.
+ *   - Dense tensors are contiguous row-major in the shapes given; base
+ *     pointers must be 16-byte aligned.
+ *   - Modality masks: bit j of a mask = modality j is present.  A score table
+ *     has one row per mask value (row index = the mask's bit pattern).
+ *   - There is no CPU fallback: without a CUDA device every compute call fails.
+ */
+#ifndef SENTRY_H
+#define SENTRY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SENTRY_API __attribute__((visibility("default")))
+#else
+#define SENTRY_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sentry_ctx sentry_ctx; /* opaque: device, workspace, status word */
+
+typedef enum {
+    SENTRY_OK = 0,
+    SENTRY_ERR_INVALID_ARG = -1, /* null pointer, bad enum, misaligned pointer */
+    SENTRY_ERR_BAD_SHAPE = -2,   /* dimension out of range or inconsistent */
+    SENTRY_ERR_UNSUPPORTED = -3, /* valid but not implemented on this path */
+    SENTRY_ERR_WORKSPACE = -4,   /* workspace missing or too small */
+    SENTRY_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed */
+    SENTRY_ERR_TIMEOUT = -6,     /* device: a bounded wait expired (status word) */
+    SENTRY_ERR_EMPTY_MASK = -7   /* device: a sample had no modality present */
+} sentry_status;
+
+/* bits of the device status word returned by sentry_get_last_status */
+#define SENTRY_STATUS_BIT_TIMEOUT 1u
+#define SENTRY_STATUS_BIT_EMPTY_MASK 2u
+#define SENTRY_STATUS_BIT_BAD_INDEX 4u /* a kept index / token id out of range was skipped */
+
+typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1 } sentry_dtype;
+
+/* Create / destroy a context bound to CUDA device `device`.  Creation
+ * allocates one small device status word; nothing else. */
+SENTRY_API int sentry_create(sentry_ctx** out, int device);
+SENTRY_API int sentry_destroy(sentry_ctx* ctx);
+
+/* Synchronise `stream`, return the device status word (>= 0, SENTRY_STATUS_BIT_*)
+ * and clear it; negative on CUDA failure. */
+SENTRY_API int sentry_get_last_status(sentry_ctx* ctx, void* stream);
+
+SENTRY_API const char* sentry_status_string(int status);
+
+/* U(T_v) = max(1, min(T_v, c * ceil(ln T_v))): how many queries per head stay
+ * active among T_v present tokens (Sec. 4.4; the paper's example T=128, c=5
+ * gives 25).  It is also the number of sampled keys per query, i.e. the width
+ * of a sample-table row.  Host function, no device work.  Returns 0 for T_v<=0. */
+SENTRY_API int sentry_num_active_queries(int T_v, int c);
+
+/* Scratch memory.  sentry_workspace_bytes returns an upper bound for any
+ * sequence of the three calls with the given descriptors (either may be NULL);
+ * sentry_set_workspace hands the library a device buffer of at least that many
+ * bytes, 256-byte aligned, which it uses until replaced.  The caller keeps
+ * ownership. */
+struct sentry_attend_desc;
+struct sentry_ffn_desc;
+SENTRY_API size_t sentry_workspace_bytes(const struct sentry_attend_desc* attend,
+                              const struct sentry_ffn_desc* ffn);
+SENTRY_API int sentry_set_workspace(sentry_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* ---------------------------------------------------------------------------
+ * SentryGate selection (Sec. 4.6 "Applying SentryGate": gate outputs under a
+ * fixed modality mask are thresholded by a pruning ratio; here the ratio is an
+ * integer budget k per unit type).
+ *
+ *   scores  [S, n_units] fp32, row s = gate outputs under mask value s
+ *   masks   [n_masks] u32, each < S (a mask >= S is skipped and flagged BAD_INDEX)
+ *   k       budget, 1 <= k <= n_units
+ *   kept    out [n_masks, k] i32: the k units with the highest score in row
+ *           masks[i]; equal scores -> the lower index wins (+0 == -0; NaN ranks
+ *           below every number); written in ASCENDING index order
+ *   kv_groups  out [n_masks] u32 or NULL: bit g set iff some kept unit maps to
+ *           KV group g = floor(unit / heads_per_group) ("head pruning with GQA
+ *           consistency"); needs heads_per_group >= 1 and n_units/heads_per_group <= 32
+ * Needs a workspace of S*k*4 bytes.
+ */
+SENTRY_API int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
+                       const uint32_t* masks, int n_masks, int k, int32_t* kept,
+                       uint32_t* kv_groups, int heads_per_group, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * SentryAttend forward (Sec. 4.4, Eq. 6) on the kept heads of every sample.
+ *
+ * Per sample b, with present tokens = { t : bit ids[t] of masks[b] is set }
+ * (T_v of them, U = sentry_num_active_queries(T_v, c)), and per kept head h
+ * with KV group g = floor(h / (Hq/Hk)):
+ *   1. sparsity score of each present query i over its sampled keys S_i:
+ *        M_i = max_{j in S_i} s_ij - mean_{j in S_i} s_ij,  s_ij = q_i.k_j/sqrt(d)
+ *   2. the U present queries with the largest M_i are active (ties -> lower index)
+ *   3. active rows:   O[i] = softmax_j(s_ij) V_g[j] over ALL present keys j (Eq. 6)
+ *   4. other present rows: O[i] = mean over present keys of V_g[j]
+ *   5. rows of absent-modality tokens: 0.   Pruned heads are not computed.
+ */
+typedef struct sentry_attend_desc {
+    int B, T, Hq, Hk, d; /* batch, tokens per sample, query heads, KV heads, head dim */
+    int k_h;             /* kept heads per sample (same for every sample) */
+    int dtype;           /* sentry_dtype of Q, K, V, O */
+    int c;               /* sparsity constant of U = c*ceil(ln T_v); the paper uses 5 */
+    int score_mode;      /* 0: S_i from the sample table; 1: S_i = all present keys */
+} sentry_attend_desc;
+
+/*   Q [B,Hq,T,d]; K, V [B,Hk,T,d]; O out [B,k_h,T,d] (heads in kept-list order)
+ *   kept_heads [B,k_h] i32 ascending, in [0,Hq)
+ *   token_modality_ids [T] i32 in [0,32); masks [B] u32
+ *   sample_table i32 + sample_offsets i64 [2^M entries, indexed by mask value]
+ *     (score_mode 0 only, else NULL): sample_table + sample_offsets[m] is the
+ *     [T_v, U] table of the subset m; row i = the U key positions (indices into
+ *     the present-token list, each in [0,T_v)) on which query position i is scored.
+ *     Subsets with equal T_v may share one table.  n_subsets = entries of sample_offsets.
+ *   active_out [B,k_h,U_max] i32 or NULL, U_max = sentry_num_active_queries(T,c):
+ *     the active token indices, ascending, padded with -1
+ *   active_in  same shape or NULL: if given, step 1-2 are skipped and these
+ *     rows are the active ones (explicit-selection mode)
+ * Supported: d in {16,32,64}; Hq % Hk == 0; T <= 32768.  Workspace: see
+ * sentry_workspace_bytes.
+ */
+SENTRY_API int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const void* Q,
+                      const void* K, const void* V, const int32_t* kept_heads,
+                      const int32_t* token_modality_ids, const uint32_t* masks,
+                      const int32_t* sample_table, const int64_t* sample_offsets,
+                      int n_subsets, void* O, int32_t* active_out,
+                      const int32_t* active_in, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Channel-compacted FFN forward (Sec. 4.6): for every present row x,
+ *   y = gelu(x . W1[:, N]) . W2[N, :],  gelu(z) = z/2 (1 + erf(z/sqrt 2)),
+ * N = the kept-channel list of the row's sample.  No bias, residual or norm.
+ */
+typedef struct sentry_ffn_desc {
+    int B, T, D, F; /* batch, tokens per sample, d_model, d_ff */
+    int k_c;        /* kept channels per list */
+    int n_lists;    /* number of kept-channel lists (one per modality subset in use) */
+    int dtype;      /* sentry_dtype of X, W1, W2, Y */
+} sentry_ffn_desc;
+
+/*   X [B,T,D]; W1 [D,F]; W2 [F,D]; Y out [B,T,D]
+ *   kept_channels [n_lists,k_c] i32 ascending in [0,F)
+ *   list_of_sample [B] i32 in [0,n_lists) or NULL (list 0 for every sample)
+ *   token_modality_ids [T] + masks [B], or both NULL (every row present);
+ *   rows of absent-modality tokens get Y = 0 and cost no arithmetic.
+ * The kept columns of W1 and rows of W2 are gathered into the workspace on
+ * every call (the "materialised" pruned weights), then a fused GEMM pair runs
+ * over the present rows.  Supported: D % 8 == 0, D <= 1024.
+ */
+SENTRY_API int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X,
+                   const void* W1, const void* W2, const int32_t* kept_channels,
+                   const int32_t* list_of_sample, const int32_t* token_modality_ids,
+                   const uint32_t* masks, void* Y, void* stream);
+
+/* Number of kernels the last call on this context enqueued (for launch
+ * accounting in benchmarks). */
+SENTRY_API int sentry_last_launch_count(const sentry_ctx* ctx);
+
+/* Optional per-kernel timing for benchmarks.  While enabled, every kernel launch
+ * is bracketed by CUDA events on the caller's stream.  sentry_profile_read
+ * synchronises the device, adds up the elapsed time and the number of launches
+ * per kernel slot since the last read into host arrays ms[n] / launches[n]
+ * (n >= sentry_profile_slots()), and clears the record.  sentry_kernel_name
+ * gives the slot's kernel name.  Off by default; adds launch gaps when on. */
+SENTRY_API int sentry_profile_enable(sentry_ctx* ctx, int on);
+SENTRY_API int sentry_profile_slots(void);
+SENTRY_API int sentry_profile_read(sentry_ctx* ctx, float* ms, int* launches, int n);
+SENTRY_API const char* sentry_kernel_name(int slot);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SENTRY_H */

@@ -1,0 +1,250 @@
+"""Python binding of libsentry (C ABI in include/sentry.h).
+
+Argument marshalling only: every step of the pruned-layer path (gate selection,
+sparse grouped-query attention, channel-compacted FFN) runs in the CUDA kernels
+of the shared library.  PyTorch is used for device memory and streams.  There is
+no CPU fallback: if the library is missing or no CUDA device is present, the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsentry.so")
+
+SENTRY_F32, SENTRY_BF16 = 0, 1
+STATUS_BIT_TIMEOUT, STATUS_BIT_EMPTY_MASK, STATUS_BIT_BAD_INDEX = 1, 2, 4
+
+EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_status_string",
+           "sentry_num_active_queries", "sentry_workspace_bytes", "sentry_set_workspace",
+           "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
+           "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
+           "sentry_kernel_name"]
+
+
+class AttendDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("B", "T", "Hq", "Hk", "d", "k_h", "dtype", "c", "score_mode")]
+
+
+class FfnDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("B", "T", "D", "F", "k_c", "n_lists", "dtype")]
+
+
+class SentryError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s failed: %s (%d)" % (what, status_string(code), code))
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """dlopen libsentry.so (no compute, no CUDA call) and declare the signatures."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(
+            "%s not found: build it with `python -m paper_2604_08971_b200.build` "
+            "(there is no CPU fallback)" % p)
+    lib = ctypes.CDLL(p)
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    lib.sentry_create.argtypes = [ctypes.POINTER(vp), ci]
+    lib.sentry_destroy.argtypes = [vp]
+    lib.sentry_get_last_status.argtypes = [vp, vp]
+    lib.sentry_status_string.argtypes = [ci]
+    lib.sentry_status_string.restype = ctypes.c_char_p
+    lib.sentry_num_active_queries.argtypes = [ci, ci]
+    lib.sentry_workspace_bytes.argtypes = [ctypes.POINTER(AttendDesc), ctypes.POINTER(FfnDesc)]
+    lib.sentry_workspace_bytes.restype = ctypes.c_size_t
+    lib.sentry_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.sentry_gate_select.argtypes = [vp, vp, ci, ci, vp, ci, ci, vp, vp, ci, vp]
+    lib.sentry_attend_fwd.argtypes = [vp, ctypes.POINTER(AttendDesc), vp, vp, vp, vp, vp, vp, vp,
+                                      vp, ci, vp, vp, vp, vp]
+    lib.sentry_ffn_fwd.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sentry_last_launch_count.argtypes = [vp]
+    lib.sentry_profile_enable.argtypes = [vp, ci]
+    lib.sentry_profile_slots.argtypes = []
+    lib.sentry_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
+                                        ctypes.POINTER(ci), ci]
+    lib.sentry_kernel_name.argtypes = [ci]
+    lib.sentry_kernel_name.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("sentry_status_string", "sentry_workspace_bytes", "sentry_kernel_name"):
+            getattr(lib, name).restype = ci
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    return _build.build(force=force, verbose=verbose)
+
+
+def status_string(code: int) -> str:
+    return load_library().sentry_status_string(int(code)).decode()
+
+
+def num_active_queries(T_v: int, c: int = 5) -> int:
+    return int(load_library().sentry_num_active_queries(int(T_v), int(c)))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("libsentry takes device tensors (got a %s tensor)" % t.device)
+    if not t.is_contiguous():
+        raise ValueError("libsentry takes contiguous tensors")
+    return t.data_ptr()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SENTRY_F32
+    if t.dtype == torch.bfloat16:
+        return SENTRY_BF16
+    raise ValueError("unsupported dtype %s" % t.dtype)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Sentry:
+    """One library context on one CUDA device; owns the workspace tensor."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libsentry needs a CUDA device; there is no CPU fallback")
+        self.lib = load_library()
+        self.device = int(device)
+        h = ctypes.c_void_p()
+        rc = self.lib.sentry_create(ctypes.byref(h), self.device)
+        if rc != 0:
+            raise SentryError(rc, "sentry_create")
+        self.h = h
+        self._ws = None
+        self.ensure_workspace(1 << 20)
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.sentry_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- workspace ---------------------------------------------------------
+    def ensure_workspace(self, nbytes: int):
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = torch.empty((int(nbytes),), dtype=torch.uint8, device="cuda:%d" % self.device)
+            rc = self.lib.sentry_set_workspace(self.h, self._ws.data_ptr(), self._ws.numel())
+            if rc != 0:
+                raise SentryError(rc, "sentry_set_workspace")
+
+    def workspace_bytes(self, attend: Optional[AttendDesc] = None, ffn: Optional[FfnDesc] = None) -> int:
+        return int(self.lib.sentry_workspace_bytes(ctypes.byref(attend) if attend else None,
+                                                   ctypes.byref(ffn) if ffn else None))
+
+    def last_status(self) -> int:
+        rc = self.lib.sentry_get_last_status(self.h, _stream())
+        if rc < 0:
+            raise SentryError(rc, "sentry_get_last_status")
+        return rc
+
+    def last_launch_count(self) -> int:
+        return int(self.lib.sentry_last_launch_count(self.h))
+
+    def profile_enable(self, on: bool):
+        self.lib.sentry_profile_enable(self.h, 1 if on else 0)
+
+    def profile_read(self) -> dict:
+        """{kernel name: (total ms, launches)} since the last read (synchronises)."""
+        n = int(self.lib.sentry_profile_slots())
+        ms = (ctypes.c_float * n)()
+        cnt = (ctypes.c_int * n)()
+        rc = self.lib.sentry_profile_read(self.h, ms, cnt, n)
+        if rc != 0:
+            raise SentryError(rc, "sentry_profile_read")
+        return {self.lib.sentry_kernel_name(i).decode(): (float(ms[i]), int(cnt[i]))
+                for i in range(n) if cnt[i] > 0}
+
+    # -- the three calls -----------------------------------------------------
+    def gate_select(self, scores: torch.Tensor, masks: torch.Tensor, k: int,
+                    heads_per_group: int = 0, kept: Optional[torch.Tensor] = None):
+        """sentry_gate_select: scores [S,n] fp32, masks [n_masks] int32/uint32 bit patterns.
+        Returns kept [n_masks,k] int32 (and the KV-group bitmaps if heads_per_group > 0)."""
+        S, n = scores.shape
+        n_masks = masks.shape[0]
+        assert scores.dtype == torch.float32 and masks.dtype in (torch.int32, torch.uint32)
+        if kept is None:
+            kept = torch.empty((n_masks, k), dtype=torch.int32, device=scores.device)
+        groups = torch.empty((n_masks,), dtype=torch.int32, device=scores.device) \
+            if heads_per_group > 0 else None
+        self.ensure_workspace(max(1 << 20, S * k * 4 + S * 4 + 1024))
+        rc = self.lib.sentry_gate_select(self.h, _ptr(scores), S, n, _ptr(masks), n_masks, int(k),
+                                         _ptr(kept), _ptr(groups), int(heads_per_group), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_gate_select")
+        return (kept, groups) if heads_per_group > 0 else kept
+
+    def attend_desc(self, Q, K, k_h: int, c: int = 5, score_mode: int = 0) -> AttendDesc:
+        B, Hq, T, d = Q.shape
+        return AttendDesc(B, T, Hq, K.shape[1], d, int(k_h), _dtype_code(Q), int(c), int(score_mode))
+
+    def attend_fwd(self, Q, K, V, kept_heads, token_modality_ids, masks, sample_table=None,
+                   sample_offsets=None, *, c: int = 5, score_mode: int = 0, O=None,
+                   active_out=None, active_in=None, return_active: bool = False):
+        """sentry_attend_fwd.  Returns O [B,k_h,T,d] (and the active lists when asked)."""
+        desc = self.attend_desc(Q, K, kept_heads.shape[1], c, score_mode)
+        assert K.shape == V.shape and K.dtype == Q.dtype and V.dtype == Q.dtype
+        if O is None:
+            O = torch.empty((desc.B, desc.k_h, desc.T, desc.d), dtype=Q.dtype, device=Q.device)
+        if return_active and active_out is None:
+            U_max = num_active_queries(desc.T, c)
+            active_out = torch.empty((desc.B, desc.k_h, U_max), dtype=torch.int32, device=Q.device)
+        self.ensure_workspace(self.workspace_bytes(attend=desc))
+        n_subsets = int(sample_offsets.shape[0]) if sample_offsets is not None else 0
+        rc = self.lib.sentry_attend_fwd(self.h, ctypes.byref(desc), _ptr(Q), _ptr(K), _ptr(V),
+                                        _ptr(kept_heads), _ptr(token_modality_ids), _ptr(masks),
+                                        _ptr(sample_table), _ptr(sample_offsets), n_subsets, _ptr(O),
+                                        _ptr(active_out), _ptr(active_in), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_attend_fwd")
+        return (O, active_out) if return_active else O
+
+    def ffn_desc(self, X, W1, kept_channels) -> FfnDesc:
+        B, T, D = X.shape
+        n_lists, k_c = kept_channels.shape
+        return FfnDesc(B, T, D, W1.shape[1], k_c, n_lists, _dtype_code(X))
+
+    def ffn_fwd(self, X, W1, W2, kept_channels, list_of_sample=None, token_modality_ids=None,
+                masks=None, Y=None):
+        """sentry_ffn_fwd.  Returns Y [B,T,D]."""
+        if kept_channels.dim() == 1:
+            kept_channels = kept_channels[None, :]
+        desc = self.ffn_desc(X, W1, kept_channels)
+        assert W1.dtype == X.dtype and W2.dtype == X.dtype
+        if Y is None:
+            Y = torch.empty_like(X)
+        self.ensure_workspace(self.workspace_bytes(ffn=desc))
+        rc = self.lib.sentry_ffn_fwd(self.h, ctypes.byref(desc), _ptr(X), _ptr(W1), _ptr(W2),
+                                     _ptr(kept_channels), _ptr(list_of_sample),
+                                     _ptr(token_modality_ids), _ptr(masks), _ptr(Y), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_ffn_fwd")
+        return Y

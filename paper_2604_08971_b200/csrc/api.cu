@@ -1,0 +1,276 @@
+// C ABI of libsentry: argument validation, workspace carving and dispatch.
+// Everything numerical happens in the kernels of the other translation units.
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr size_t kMinWorkspace = 1u << 20;
+constexpr int kMaxTokens = 32768;
+constexpr int kMaxUnits = 49152;
+
+inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+size_t attend_workspace_bytes(const sentry_attend_desc& d) {
+    const int U_max = sentry_num_active(d.T, d.c);
+    WsAlloc a(nullptr, 0);
+    a.take<float>((size_t)d.B * d.k_h * d.T);
+    a.take<int32_t>((size_t)d.B * d.k_h * U_max);
+    return a.off + 256;
+}
+
+int check_attend_desc(const sentry_attend_desc* d) {
+    if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->score_mode != 0 && d->score_mode != 1) return SENTRY_ERR_INVALID_ARG;
+    if (d->B < 1 || d->T < 1 || d->Hq < 1 || d->Hk < 1 || d->k_h < 1 || d->c < 1)
+        return SENTRY_ERR_BAD_SHAPE;
+    if (d->Hq % d->Hk != 0 || d->k_h > d->Hq) return SENTRY_ERR_BAD_SHAPE;
+    if (d->T > kMaxTokens) return SENTRY_ERR_UNSUPPORTED;
+    if (d->d != 16 && d->d != 32 && d->d != 64) return SENTRY_ERR_UNSUPPORTED;
+    if ((long long)d->B * d->k_h > 0x7fffffffLL / 4) return SENTRY_ERR_UNSUPPORTED;
+    return SENTRY_OK;
+}
+
+int check_ffn_desc(const sentry_ffn_desc* d) {
+    if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->B < 1 || d->T < 1 || d->D < 1 || d->F < 1 || d->k_c < 1 || d->n_lists < 1)
+        return SENTRY_ERR_BAD_SHAPE;
+    if (d->k_c > d->F) return SENTRY_ERR_BAD_SHAPE;
+    if (d->D % 8 != 0 || d->D > 1024 || d->T > 65535 || d->n_lists > 4096)
+        return SENTRY_ERR_UNSUPPORTED;
+    if ((long long)d->B * d->T > 0x7fffffffLL - 8192) return SENTRY_ERR_UNSUPPORTED;
+    return SENTRY_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sentry_create(sentry_ctx** out, int device) {
+    if (out == nullptr) return SENTRY_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return SENTRY_ERR_CUDA;
+    SENTRY_CUDA_TRY(cudaSetDevice(device));
+    sentry_ctx* c = new (std::nothrow) sentry_ctx();
+    if (c == nullptr) return SENTRY_ERR_CUDA;
+    c->device = device;
+    c->workspace = nullptr;
+    c->workspace_bytes = 0;
+    c->last_launches = 0;
+    c->profiling = false;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return SENTRY_ERR_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc((void**)&c->d_status, sizeof(unsigned int)) != cudaSuccess) { delete c; return SENTRY_ERR_CUDA; }
+    if (cudaMemset(c->d_status, 0, sizeof(unsigned int)) != cudaSuccess) {
+        cudaFree(c->d_status);
+        delete c;
+        return SENTRY_ERR_CUDA;
+    }
+    *out = c;
+    return SENTRY_OK;
+}
+
+int sentry_destroy(sentry_ctx* ctx) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->d_status);
+    for (ProfRec& r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    for (cudaEvent_t e : ctx->pool) cudaEventDestroy(e);
+    delete ctx;
+    return SENTRY_OK;
+}
+
+int sentry_profile_enable(sentry_ctx* ctx, int on) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    ctx->profiling = on != 0;
+    return SENTRY_OK;
+}
+
+int sentry_profile_slots(void) { return KS_COUNT; }
+
+const char* sentry_kernel_name(int slot) {
+    static const char* names[KS_COUNT] = {"gate_rows", "gate_expand", "attend_score", "attend_select",
+                                          "attend_core", "ffn_plan_rows", "ffn_plan_tiles",
+                                          "ffn_prepack", "ffn_main"};
+    return (slot >= 0 && slot < KS_COUNT) ? names[slot] : "?";
+}
+
+int sentry_profile_read(sentry_ctx* ctx, float* ms, int* launches, int n) {
+    if (ctx == nullptr || ms == nullptr || launches == nullptr || n < KS_COUNT)
+        return SENTRY_ERR_INVALID_ARG;
+    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    SENTRY_CUDA_TRY(cudaDeviceSynchronize());
+    for (int i = 0; i < n; ++i) { ms[i] = 0.f; launches[i] = 0; }
+    for (ProfRec& r : ctx->prof) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, r.start, r.stop) == cudaSuccess) {
+            ms[r.slot] += t;
+            launches[r.slot] += 1;
+        }
+        ctx->pool.push_back(r.start);
+        ctx->pool.push_back(r.stop);
+    }
+    ctx->prof.clear();
+    return SENTRY_OK;
+}
+
+int sentry_get_last_status(sentry_ctx* ctx, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    SENTRY_CUDA_TRY(cudaStreamSynchronize(st));
+    unsigned int h = 0;
+    SENTRY_CUDA_TRY(cudaMemcpyAsync(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
+    SENTRY_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st));
+    SENTRY_CUDA_TRY(cudaStreamSynchronize(st));
+    return (int)(h & 0x7fffffffu);
+}
+
+const char* sentry_status_string(int status) {
+    switch (status) {
+        case SENTRY_OK: return "ok";
+        case SENTRY_ERR_INVALID_ARG: return "invalid argument";
+        case SENTRY_ERR_BAD_SHAPE: return "bad shape";
+        case SENTRY_ERR_UNSUPPORTED: return "unsupported configuration";
+        case SENTRY_ERR_WORKSPACE: return "workspace missing or too small";
+        case SENTRY_ERR_CUDA: return "CUDA call failed";
+        case SENTRY_ERR_TIMEOUT: return "device wait timed out";
+        case SENTRY_ERR_EMPTY_MASK: return "sample with empty modality mask";
+        default: return "unknown status";
+    }
+}
+
+int sentry_num_active_queries(int T_v, int c) { return sentry_num_active(T_v, c); }
+
+size_t sentry_workspace_bytes(const sentry_attend_desc* attend, const sentry_ffn_desc* ffn) {
+    size_t need = kMinWorkspace;
+    if (attend != nullptr && check_attend_desc(attend) == SENTRY_OK) {
+        const size_t a = attend_workspace_bytes(*attend);
+        if (a > need) need = a;
+    }
+    if (ffn != nullptr && check_ffn_desc(ffn) == SENTRY_OK) {
+        const size_t f = ffn_workspace_bytes(*ffn);
+        if (f > need) need = f;
+    }
+    return align_up(need, 256);
+}
+
+int sentry_set_workspace(sentry_ctx* ctx, void* dev_ptr, size_t bytes) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (dev_ptr != nullptr && !aligned(dev_ptr, 256)) return SENTRY_ERR_INVALID_ARG;
+    ctx->workspace = dev_ptr;
+    ctx->workspace_bytes = dev_ptr ? bytes : 0;
+    return SENTRY_OK;
+}
+
+int sentry_last_launch_count(const sentry_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
+                       const uint32_t* masks, int n_masks, int k, int32_t* kept,
+                       uint32_t* kv_groups, int heads_per_group, void* stream) {
+    if (ctx == nullptr || scores == nullptr || masks == nullptr || kept == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(scores, 4) || !aligned(masks, 4) || !aligned(kept, 4)) return SENTRY_ERR_INVALID_ARG;
+    if (S < 1 || n_units < 1 || n_masks < 0 || k < 1 || k > n_units) return SENTRY_ERR_BAD_SHAPE;
+    if (n_units > kMaxUnits || S > 65536) return SENTRY_ERR_UNSUPPORTED;
+    if (kv_groups != nullptr) {
+        if (heads_per_group < 1) return SENTRY_ERR_INVALID_ARG;
+        if ((n_units + heads_per_group - 1) / heads_per_group > 32) return SENTRY_ERR_BAD_SHAPE;
+    }
+    ctx->last_launches = 0;
+    if (n_masks == 0) return SENTRY_OK;
+    WsAlloc a(ctx->workspace, ctx->workspace_bytes);
+    int32_t* rows = a.take<int32_t>((size_t)S * k);
+    uint32_t* groups = a.take<uint32_t>((size_t)S);
+    if (!a.ok) return SENTRY_ERR_WORKSPACE;
+    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    return launch_gate_select(ctx, scores, S, n_units, masks, n_masks, k, kept, kv_groups,
+                              heads_per_group, rows, groups, (cudaStream_t)stream);
+}
+
+int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const void* Q,
+                      const void* K, const void* V, const int32_t* kept_heads,
+                      const int32_t* token_modality_ids, const uint32_t* masks,
+                      const int32_t* sample_table, const int64_t* sample_offsets,
+                      int n_subsets, void* O, int32_t* active_out, const int32_t* active_in,
+                      void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_attend_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (Q == nullptr || K == nullptr || V == nullptr || O == nullptr || kept_heads == nullptr ||
+        token_modality_ids == nullptr || masks == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) ||
+        !aligned(kept_heads, 4) || !aligned(token_modality_ids, 4) || !aligned(masks, 4))
+        return SENTRY_ERR_INVALID_ARG;
+    if (active_in == nullptr && desc->score_mode == 0) {
+        if (sample_table == nullptr || sample_offsets == nullptr) return SENTRY_ERR_INVALID_ARG;
+        if (n_subsets < 1) return SENTRY_ERR_BAD_SHAPE;
+        if (!aligned(sample_table, 4) || !aligned(sample_offsets, 8)) return SENTRY_ERR_INVALID_ARG;
+    }
+    ctx->last_launches = 0;
+    AttendArgs a;
+    a.d = *desc;
+    a.Q = Q; a.K = K; a.V = V;
+    a.kept_heads = kept_heads;
+    a.ids = token_modality_ids;
+    a.masks = masks;
+    a.sample_table = sample_table;
+    a.sample_offsets = sample_offsets;
+    a.n_subsets = n_subsets;
+    a.O = O;
+    a.U_max = sentry_num_active(desc->T, desc->c);
+    a.status = ctx->d_status;
+    WsAlloc ws(ctx->workspace, ctx->workspace_bytes);
+    a.mscore = ws.take<float>((size_t)desc->B * desc->k_h * desc->T);
+    int32_t* ws_active = ws.take<int32_t>((size_t)desc->B * desc->k_h * a.U_max);
+    if (!ws.ok) return SENTRY_ERR_WORKSPACE;
+    a.selection_given = active_in != nullptr;
+    a.active = a.selection_given ? const_cast<int32_t*>(active_in)
+                                 : (active_out != nullptr ? active_out : ws_active);
+    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    rc = launch_attend_generic(ctx, a, st);
+    if (rc != SENTRY_OK) return rc;
+    if (a.selection_given && active_out != nullptr && active_out != active_in) {
+        SENTRY_CUDA_TRY(cudaMemcpyAsync(active_out, active_in,
+                                        (size_t)desc->B * desc->k_h * a.U_max * sizeof(int32_t),
+                                        cudaMemcpyDeviceToDevice, st));
+    }
+    return SENTRY_OK;
+}
+
+int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, const void* W1,
+                   const void* W2, const int32_t* kept_channels, const int32_t* list_of_sample,
+                   const int32_t* token_modality_ids, const uint32_t* masks, void* Y,
+                   void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_ffn_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (X == nullptr || W1 == nullptr || W2 == nullptr || Y == nullptr || kept_channels == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if ((token_modality_ids == nullptr) != (masks == nullptr)) return SENTRY_ERR_INVALID_ARG;
+    if (desc->n_lists > 1 && list_of_sample == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(W1, 16) || !aligned(W2, 16) || !aligned(Y, 16) ||
+        !aligned(kept_channels, 4))
+        return SENTRY_ERR_INVALID_ARG;
+    ctx->last_launches = 0;
+    FfnArgs a;
+    a.d = *desc;
+    a.X = X; a.W1 = W1; a.W2 = W2;
+    a.kept = kept_channels;
+    a.list_of_sample = list_of_sample;
+    a.ids = token_modality_ids;
+    a.masks = masks;
+    a.Y = Y;
+    a.status = ctx->d_status;
+    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,315 @@
+// Channel-compacted FFN (Section 4.6): y = gelu(x W1[:, N]) W2[N, :].
+// This file holds the row plan, the weight gather ("materialising" W1', W2')
+// and the plain-ALU fp32-accumulate kernel; the tensor-core kernel for bf16
+// lives in ffn_tc.cu and shares the plan.
+#include <math.h>
+
+#include "common.cuh"
+#include "ffn_plan.cuh"
+
+int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,
+                  int kc_pad, int max_tiles, cudaStream_t st);  // ffn_tc.cu
+bool ffn_tc_supported(const sentry_ffn_desc& d);
+int ffn_tc_kc_pad(int k_c);
+
+namespace {
+
+constexpr int kGenericTileRows = 16;
+constexpr int kGenericThreads = 256;
+constexpr int kTcTileRows = 128;
+
+// grid B.  Present-token list and count of each sample; zero rows of Y for absent tokens.
+__global__ void __launch_bounds__(256)
+ffn_plan_rows_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks, int T,
+                     int row_bytes, uint16_t* __restrict__ vlist, int32_t* __restrict__ tv,
+                     uint8_t* __restrict__ Y, unsigned int* status) {
+    __shared__ int red[66];
+    const int b = blockIdx.x;
+    const uint32_t mask = (ids != nullptr) ? masks[b] : 0xffffffffu;
+    uint16_t* vl = vlist + (size_t)b * T;
+    const int Tv = block_build_valid(ids, T, mask, vl, red);
+    if (threadIdx.x == 0) {
+        tv[b] = Tv;
+        if (Tv == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
+    }
+    if (ids == nullptr || Tv == T) return;
+    // zero the absent rows: 16-byte stores, one row after the other
+    const int vec_per_row = row_bytes / 16;
+    for (int t = 0; t < T; ++t) {
+        const int m = ids[t];
+        const bool present = (m >= 0 && m < 32) && ((mask >> m) & 1u);
+        if (present) continue;
+        uint4* row = reinterpret_cast<uint4*>(Y + ((size_t)b * T + t) * row_bytes);
+        for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) row[v] = make_uint4(0, 0, 0, 0);
+    }
+}
+
+// one block.  Group samples by list, prefix rows, cut into tiles.
+__global__ void __launch_bounds__(1024)
+ffn_plan_tiles_kernel(const int32_t* __restrict__ tv, const int32_t* __restrict__ list_of_sample,
+                      int B, int n_lists, int tile_rows, FfnPlan p, unsigned int* status) {
+    __shared__ int s_warp_cnt[32], s_warp_rows[32];
+    __shared__ int s_base_cnt, s_base_rows, s_list_begin;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    if (threadIdx.x == 0) { s_list_begin = 0; p.tile_start[0] = 0; p.list_start[0] = 0; }
+    __syncthreads();
+    for (int l = 0; l < n_lists; ++l) {
+        if (threadIdx.x == 0) { s_base_cnt = 0; s_base_rows = 0; }
+        __syncthreads();
+        for (int b0 = 0; b0 < B; b0 += blockDim.x) {
+            const int b = b0 + threadIdx.x;
+            int mine = 0, rows = 0;
+            if (b < B) {
+                int lb = list_of_sample ? list_of_sample[b] : 0;
+                if (lb < 0 || lb >= n_lists) {
+                    if (l == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+                    lb = 0;
+                }
+                mine = (lb == l);
+                rows = mine ? tv[b] : 0;
+            }
+            // inclusive warp scans of (mine, rows)
+            int c = mine, r = rows;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int c2 = __shfl_up_sync(0xffffffffu, c, o);
+                const int r2 = __shfl_up_sync(0xffffffffu, r, o);
+                if (lane >= o) { c += c2; r += r2; }
+            }
+            if (lane == 31) { s_warp_cnt[wid] = c; s_warp_rows[wid] = r; }
+            __syncthreads();
+            int c_before = s_base_cnt, r_before = s_base_rows, c_tot = 0, r_tot = 0;
+            for (int w = 0; w < nw; ++w) {
+                if (w < wid) { c_before += s_warp_cnt[w]; r_before += s_warp_rows[w]; }
+                c_tot += s_warp_cnt[w]; r_tot += s_warp_rows[w];
+            }
+            if (mine) {
+                const int pos = s_list_begin + c_before + c - 1;
+                p.order[pos] = b;
+                p.row_prefix[pos] = r_before + r - rows;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) { s_base_cnt += c_tot; s_base_rows += r_tot; }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            p.list_rows[l] = s_base_rows;
+            s_list_begin += s_base_cnt;
+            p.list_start[l + 1] = s_list_begin;
+            p.tile_start[l + 1] = p.tile_start[l] + (s_base_rows + tile_rows - 1) / tile_rows;
+        }
+        __syncthreads();
+    }
+}
+
+// Weight gather.  layout 0 (plain-ALU kernel): W1g [l][D][kc_pad], W2g [l][kc_pad][D]
+//                 layout 1 (tensor-core kernel, both K-major):
+//                                 W1c [l][kc_pad][D],  W2c [l][D][kc_pad]
+// Columns / rows n >= k_c are zero.  grid (ceil(kc_pad*D/256), n_lists, 2).
+template <typename T>
+__global__ void __launch_bounds__(256)
+ffn_prepack_kernel(const T* __restrict__ W1, const T* __restrict__ W2,
+                   const int32_t* __restrict__ kept, int D, int F, int k_c, int kc_pad, int layout,
+                   T* __restrict__ out1, T* __restrict__ out2, unsigned int* status) {
+    const int l = blockIdx.y;
+    const size_t per = (size_t)kc_pad * D;
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= per) return;
+    const int32_t* N = kept + (size_t)l * k_c;
+    if (blockIdx.z == 0) {
+        // W1: destination-major index so that writes coalesce
+        int n, e;
+        if (layout == 0) { e = (int)(i / kc_pad); n = (int)(i % kc_pad); }
+        else             { n = (int)(i / D);      e = (int)(i % D); }
+        T v = from_f32<T>(0.f);
+        if (n < k_c) {
+            const int ch = N[n];
+            if (ch >= 0 && ch < F) v = W1[(size_t)e * F + ch];
+            else if (e == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+        }
+        out1[(size_t)l * per + i] = v;
+    } else {
+        int n, e;
+        if (layout == 0) { n = (int)(i / D);      e = (int)(i % D); }
+        else             { e = (int)(i / kc_pad); n = (int)(i % kc_pad); }
+        T v = from_f32<T>(0.f);
+        if (n < k_c) {
+            const int ch = N[n];
+            if (ch >= 0 && ch < F) v = W2[(size_t)ch * D + e];
+        }
+        out2[(size_t)l * per + i] = v;
+    }
+}
+
+__device__ __forceinline__ float gelu_erf(float z) {
+    return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f));
+}
+
+// Plain-ALU fused pair on a tile of 16 present rows.  grid = tile upper bound.
+template <typename T>
+__global__ void __launch_bounds__(kGenericThreads)
+ffn_generic_kernel(const T* __restrict__ X, const T* __restrict__ W1g, const T* __restrict__ W2g,
+                   FfnPlan plan, int n_lists, int Tlen, int D, int k_c, int kc_pad,
+                   T* __restrict__ Y) {
+    extern __shared__ float s_f[];
+    float* s_x = s_f;                                  // [16][D]
+    float* s_h = s_f + (size_t)kGenericTileRows * D;   // [16][256]
+    __shared__ long long s_row[kGenericTileRows];
+    int l, slot0, n_rows;
+    if (!ffn_tile_lookup(plan, n_lists, blockIdx.x, kGenericTileRows, l, slot0, n_rows)) return;
+    if (threadIdx.x < kGenericTileRows)
+        s_row[threadIdx.x] = threadIdx.x < n_rows ? ffn_row_of_slot(plan, l, slot0 + threadIdx.x, Tlen) : -1;
+    __syncthreads();
+    for (int i = threadIdx.x; i < kGenericTileRows * D; i += blockDim.x) {
+        const int r = i / D, e = i % D;
+        s_x[i] = s_row[r] >= 0 ? to_f32<T>(X[(size_t)s_row[r] * D + e]) : 0.f;
+    }
+    const T* w1 = W1g + (size_t)l * D * kc_pad;
+    const T* w2 = W2g + (size_t)l * kc_pad * D;
+    constexpr int kMaxSlots = 4;  // D <= 1024
+    float y[kMaxSlots][kGenericTileRows];
+#pragma unroll
+    for (int s = 0; s < kMaxSlots; ++s)
+#pragma unroll
+        for (int r = 0; r < kGenericTileRows; ++r) y[s][r] = 0.f;
+    __syncthreads();
+    for (int c0 = 0; c0 < k_c; c0 += kGenericThreads) {
+        const int n = c0 + threadIdx.x;
+        float hacc[kGenericTileRows];
+#pragma unroll
+        for (int r = 0; r < kGenericTileRows; ++r) hacc[r] = 0.f;
+        if (n < k_c) {
+            for (int e = 0; e < D; ++e) {
+                const float w = to_f32<T>(w1[(size_t)e * kc_pad + n]);
+#pragma unroll
+                for (int r = 0; r < kGenericTileRows; ++r) hacc[r] = fmaf(s_x[r * D + e], w, hacc[r]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kGenericTileRows; ++r)
+            s_h[r * kGenericThreads + threadIdx.x] = (n < k_c) ? gelu_erf(hacc[r]) : 0.f;
+        __syncthreads();
+        const int cn = min(kGenericThreads, k_c - c0);
+#pragma unroll
+        for (int s = 0; s < kMaxSlots; ++s) {
+            const int e = s * kGenericThreads + threadIdx.x;
+            if (e < D) {
+                for (int j = 0; j < cn; ++j) {
+                    const float w = to_f32<T>(w2[(size_t)(c0 + j) * D + e]);
+#pragma unroll
+                    for (int r = 0; r < kGenericTileRows; ++r)
+                        y[s][r] = fmaf(s_h[r * kGenericThreads + j], w, y[s][r]);
+                }
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int s = 0; s < kMaxSlots; ++s) {
+        const int e = s * kGenericThreads + threadIdx.x;
+        if (e < D) {
+#pragma unroll
+            for (int r = 0; r < kGenericTileRows; ++r)
+                if (s_row[r] >= 0) Y[(size_t)s_row[r] * D + e] = from_f32<T>(y[s][r]);
+        }
+    }
+}
+
+struct FfnWs {
+    FfnPlan plan;
+    void *w1p, *w2p;
+    bool ok;
+    size_t used;
+};
+
+FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes) {
+    WsAlloc a(ws, bytes);
+    FfnWs w;
+    const size_t esz = d.dtype == SENTRY_F32 ? 4 : 2;
+    w.plan.vlist = a.take<uint16_t>((size_t)d.B * d.T);
+    w.plan.tv = a.take<int32_t>(d.B);
+    w.plan.order = a.take<int32_t>(d.B);
+    w.plan.row_prefix = a.take<int32_t>(d.B);
+    w.plan.list_start = a.take<int32_t>(d.n_lists + 1);
+    w.plan.list_rows = a.take<int32_t>(d.n_lists);
+    w.plan.tile_start = a.take<int32_t>(d.n_lists + 1);
+    w.w1p = a.take<uint8_t>((size_t)d.n_lists * kc_pad * d.D * esz);
+    w.w2p = a.take<uint8_t>((size_t)d.n_lists * kc_pad * d.D * esz);
+    w.ok = a.ok;
+    w.used = a.off;
+    return w;
+}
+
+int kc_pad_for(const sentry_ffn_desc& d) {
+    if (d.dtype == SENTRY_BF16 && ffn_tc_supported(d)) return ffn_tc_kc_pad(d.k_c);
+    return (d.k_c + 7) / 8 * 8;
+}
+
+}  // namespace
+
+size_t ffn_workspace_bytes(const sentry_ffn_desc& d) {
+    return carve(d, kc_pad_for(d), nullptr, 0).used + 256;
+}
+
+int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cudaStream_t st) {
+    const sentry_ffn_desc& d = a.d;
+    const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
+    const int kc_pad = kc_pad_for(d);
+    FfnWs w = carve(d, kc_pad, ws, ws_bytes);
+    if (!w.ok) return SENTRY_ERR_WORKSPACE;
+    const int esz = d.dtype == SENTRY_F32 ? 4 : 2;
+    const int tile_rows = tc ? kTcTileRows : kGenericTileRows;
+
+    {
+        LaunchScope ls(ctx, KS_FFN_PLAN_ROWS, st);
+        ffn_plan_rows_kernel<<<d.B, 256, 0, st>>>(a.ids, a.masks, d.T, d.D * esz, w.plan.vlist,
+                                                   w.plan.tv, (uint8_t*)a.Y, a.status);
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    {
+        LaunchScope ls(ctx, KS_FFN_PLAN_TILES, st);
+        ffn_plan_tiles_kernel<<<1, 1024, 0, st>>>(w.plan.tv, a.list_of_sample, d.B, d.n_lists,
+                                                   tile_rows, w.plan, a.status);
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    {
+        const size_t per = (size_t)kc_pad * d.D;
+        dim3 grid((unsigned)((per + 255) / 256), d.n_lists, 2);
+        LaunchScope ls(ctx, KS_FFN_PREPACK, st);
+        if (d.dtype == SENTRY_F32)
+            ffn_prepack_kernel<float><<<grid, 256, 0, st>>>((const float*)a.W1, (const float*)a.W2,
+                                                            a.kept, d.D, d.F, d.k_c, kc_pad, 0,
+                                                            (float*)w.w1p, (float*)w.w2p, a.status);
+        else
+            ffn_prepack_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
+                (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.D, d.F, d.k_c,
+                kc_pad, tc ? 1 : 0, (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    const long long rows = (long long)d.B * d.T;
+    const int max_tiles = (int)((rows + tile_rows - 1) / tile_rows) + d.n_lists;
+    if (tc) {
+        int rc = launch_ffn_tc(ctx, a, w.plan, w.w1p, w.w2p, kc_pad, max_tiles, st);
+        if (rc != SENTRY_OK) return rc;
+    } else {
+        const size_t smem = ((size_t)kGenericTileRows * d.D + kGenericTileRows * kGenericThreads) * 4;
+        LaunchScope ls(ctx, KS_FFN_MAIN, st);
+        if (d.dtype == SENTRY_F32) {
+            auto kern = ffn_generic_kernel<float>;
+            if (smem > 48 * 1024)
+                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<max_tiles, kGenericThreads, smem, st>>>((const float*)a.X, (const float*)w.w1p,
+                                                            (const float*)w.w2p, w.plan, d.n_lists,
+                                                            d.T, d.D, d.k_c, kc_pad, (float*)a.Y);
+        } else {
+            auto kern = ffn_generic_kernel<__nv_bfloat16>;
+            if (smem > 48 * 1024)
+                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<max_tiles, kGenericThreads, smem, st>>>(
+                (const __nv_bfloat16*)a.X, (const __nv_bfloat16*)w.w1p, (const __nv_bfloat16*)w.w2p,
+                w.plan, d.n_lists, d.T, d.D, d.k_c, kc_pad, (__nv_bfloat16*)a.Y);
+        }
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}

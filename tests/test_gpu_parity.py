@@ -1,0 +1,240 @@
+"""GPU parity: libsentry (through its C ABI) against the float64 oracle on the
+same seeded inputs.  Kept-index lists bit-exact; outputs within 1e-4 (fp32) and
+2e-2 (bf16) max-abs error relative to the output RMS."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_08971_b200 as sentry
+import synth
+from tests import parity
+from tests.parity import TOL, dev, masks_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sn():
+    ctx = sentry.Sentry(0)
+    yield ctx
+    ctx.close()
+
+
+def n_s_of(tv):
+    return sentry.num_active_queries(tv, 5)
+
+
+# ------------------------------------------------------------------------ gate
+@pytest.mark.parametrize("n,k", [(4, 3), (8, 4), (8, 2), (8, 6), (12, 7), (256, 128), (512, 256),
+                                 (1024, 512), (1536, 614), (7, 7), (9, 1), (5000, 1234)])
+def test_gate_bit_exact(sn, n, k):
+    g = np.random.default_rng(n * 1000 + k)
+    S = 16
+    scores = g.standard_normal((S, n)).astype(np.float32)
+    masks = g.integers(1, S, size=300).astype(np.uint32)
+    got = sn.gate_select(dev(scores), masks_dev(masks), k).cpu().numpy()
+    np.testing.assert_array_equal(got, oracle.gate_select(scores, masks, k))
+    assert sn.last_status() == 0
+
+
+def test_gate_ties_nan_zero_and_groups(sn):
+    g = np.random.default_rng(5)
+    n = 96
+    # heavy ties: scores drawn from 5 distinct values, plus NaN, +-0, +-inf
+    pool = np.array([0.5, -0.0, 0.0, 1.5, np.nan, -np.inf, np.inf, 0.5], dtype=np.float32)
+    scores = pool[g.integers(0, len(pool), size=(8, n))]
+    masks = np.arange(8, dtype=np.uint32)
+    for k in (1, 7, 32, 95, 96):
+        got, groups = sn.gate_select(dev(scores), masks_dev(masks), k, heads_per_group=4)
+        want = oracle.gate_select(scores, masks, k)
+        np.testing.assert_array_equal(got.cpu().numpy(), want)
+        np.testing.assert_array_equal(groups.cpu().numpy().astype(np.uint32),
+                                      oracle.kv_groups(want, 4))
+
+
+def test_gate_large_fanout_and_bad_mask(sn):
+    g = np.random.default_rng(6)
+    scores = g.standard_normal((8, 1024)).astype(np.float32)
+    masks = (1 + np.arange(4096) % 7).astype(np.uint32)
+    got = sn.gate_select(dev(scores), masks_dev(masks), 512).cpu().numpy()
+    np.testing.assert_array_equal(got, oracle.gate_select(scores, masks, 512))
+    assert sn.last_status() == 0
+    bad = masks.copy()
+    bad[17] = 9  # >= S: skipped and flagged, no fault
+    sn.gate_select(dev(scores), masks_dev(bad), 512)
+    assert sn.last_status() & sentry.STATUS_BIT_BAD_INDEX
+
+
+def test_error_codes_no_launch(sn):
+    scores = torch.zeros((4, 8), device="cuda")
+    masks = torch.ones((2,), dtype=torch.int32, device="cuda")
+    with pytest.raises(sentry.SentryError) as e:
+        sn.gate_select(scores, masks, 9)
+    assert e.value.code == -2
+    with pytest.raises(sentry.SentryError) as e:
+        sn.gate_select(scores, masks, 0)
+    assert e.value.code == -2
+    Q = torch.zeros((1, 4, 8, 24), device="cuda")  # head_dim 24 unsupported
+    K = torch.zeros((1, 2, 8, 24), device="cuda")
+    kh = torch.zeros((1, 2), dtype=torch.int32, device="cuda")
+    ids = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    with pytest.raises(sentry.SentryError) as e:
+        sn.attend_fwd(Q, K, K, kh, ids, masks[:1], score_mode=1)
+    assert e.value.code == -3
+    Q = torch.zeros((1, 4, 8, 16), device="cuda")
+    K = torch.zeros((1, 2, 8, 16), device="cuda")
+    with pytest.raises(sentry.SentryError) as e:   # sampled mode without a table
+        sn.attend_fwd(Q, K, K, kh, ids, masks[:1], score_mode=0)
+    assert e.value.code == -1
+    X = torch.zeros((1, 8, 12), device="cuda")     # D % 8 != 0
+    W1 = torch.zeros((12, 16), device="cuda")
+    W2 = torch.zeros((16, 12), device="cuda")
+    kc = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+    with pytest.raises(sentry.SentryError) as e:
+        sn.ffn_fwd(X, W1, W2, kc)
+    assert e.value.code == -3
+    assert sn.last_status() == 0
+
+
+# ------------------------------------------------------------------ workloads
+def _run_workload(sn, w, attend_samples="all", ffn_samples="strat", score_mode=0):
+    inp = synth.generate(w, n_s_of)
+    kept_h, kept_c = parity.gate_lists(sn, inp)
+    strat = parity.stratified_samples(inp, 2)
+    a_s = None if attend_samples == "all" else strat
+    f_s = None if ffn_samples == "all" else strat
+    err_a, ties = parity.attend_parity(sn, inp, kept_h, a_s, score_mode)
+    err_f = parity.ffn_parity(sn, inp, kept_c, f_s)
+    assert err_a <= TOL[w.dtype], (w.name, "attend", err_a)
+    assert err_f <= TOL[w.dtype], (w.name, "ffn", err_f)
+    return err_a, err_f, ties
+
+
+def test_config1_fp32_both_score_modes_and_single_modalities(sn):
+    w = synth.config1()
+    _run_workload(sn, w, "all", "all", 0)
+    _run_workload(sn, w, "all", "all", 1)
+    inp = synth.generate(w, n_s_of)
+    kept_h, kept_c = parity.gate_lists(sn, inp)
+    for m in (1, 2):  # one modality dropped: rows of its tokens are zero, the rest as if deleted
+        inp.masks[:] = m
+        g = np.random.default_rng(m)
+        inp.sample_table, inp.table_offsets = synth.make_sample_tables(w, inp.masks, n_s_of, g)
+        inp.subsets = np.array([m], dtype=np.uint32)
+        inp.list_of_sample[:] = 0
+        err_a, _ = parity.attend_parity(sn, inp, kept_h)
+        err_f = parity.ffn_parity(sn, inp, kept_c[:1])
+        assert err_a <= TOL["f32"] and err_f <= TOL["f32"]
+
+
+def test_config2_wearable_bf16(sn):
+    _run_workload(sn, synth.config2(), "all", "strat")
+
+
+@pytest.mark.parametrize("ratio", [0.25, 0.5, 0.75])
+def test_config3_physio_head_keep_sweep(sn, ratio):
+    _run_workload(sn, synth.config3(ratio), "all", "strat")
+
+
+def test_config4_full_layer_all_subsets(sn):
+    w = synth.config4()
+    inp = synth.generate(w, n_s_of, tensors=False)
+    assert sorted(set(inp.masks.tolist())) == [1, 2, 3]
+    _run_workload(sn, w, "all", "strat")
+
+
+@pytest.mark.parametrize("B,T", [(1, 64), (16, 64), (16, 256), (1, 1024), (16, 1024), (1, 4096),
+                                 (256, 256), (14, 4096)])
+def test_config5_sweep_cells(sn, B, T):
+    _run_workload(sn, synth.config5(B, T), "strat", "strat")
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [16, 32, 64])
+def test_ragged_shapes_and_head_dims(sn, dtype, d):
+    # token counts that are not multiples of any tile; 3 modalities of unequal length
+    w = synth.Workload("ragged", dtype, 5, (37, 5, 91), 72, 6, 3, d, 200, 4, 77, "cycle7", 40 + d)
+    _run_workload(sn, w, "all", "all")
+
+
+def test_dense_degenerate_and_single_token(sn):
+    # T_v <= U: every present row is an Eq. 6 row (dense GQA attention)
+    w = synth.Workload("dense", "f32", 3, (4, 3, 2), 64, 4, 2, 16, 64, 2, 16, "cycle7", 50)
+    _run_workload(sn, w, "all", "all")
+    w1 = synth.Workload("one", "f32", 2, (1,), 64, 2, 1, 16, 64, 1, 8, "all", 51)
+    _run_workload(sn, w1, "all", "all")
+
+
+def test_whole_kv_group_pruned_and_k_extremes(sn):
+    # scores that force all kept heads into group 1: group 0 is never referenced
+    w = synth.Workload("grp", "bf16", 4, (48, 48), 64, 8, 2, 32, 128, 3, 128, "all", 52)
+    inp = synth.generate(w, n_s_of)
+    inp.scores_heads[:, :4] = -10.0
+    kept_h, kept_c = parity.gate_lists(sn, inp)
+    assert kept_h.min().item() >= 4
+    # poison the unreferenced group's K/V: the result must not change
+    inp.K[:, 0] = float("nan")
+    inp.V[:, 0] = float("nan")
+    err, _ = parity.attend_parity(sn, inp, kept_h)
+    assert err <= TOL["bf16"]
+    assert parity.ffn_parity(sn, inp, kept_c) <= TOL["bf16"]   # k_c = F: nothing pruned
+    for k_h in (1, 8):
+        w2 = w.with_(k_h=k_h, seed=53 + k_h)
+        inp2 = synth.generate(w2, n_s_of)
+        kh2, _ = parity.gate_lists(sn, inp2)
+        err, _ = parity.attend_parity(sn, inp2, kh2)
+        assert err <= TOL["bf16"]
+
+
+def test_exact_score_ties_select_lower_index(sn):
+    w = synth.Workload("ties", "f32", 2, (40,), 64, 2, 1, 16, 64, 2, 8, "all", 54)
+    inp = synth.generate(w, n_s_of)
+    inp.Q[:] = inp.Q[:, :, :1, :]          # identical queries -> identical sparsity scores
+    inp.sample_table[:] = np.tile(np.arange(n_s_of(40), dtype=np.int32), 40)  # same sampled keys
+    kept_h, _ = parity.gate_lists(sn, inp)
+    O, act = sn.attend_fwd(inp.Q.cuda(), inp.K.cuda(), inp.V.cuda(), kept_h, dev(inp.ids),
+                           masks_dev(inp.masks), dev(inp.sample_table), dev(inp.table_offsets),
+                           return_active=True)
+    U = n_s_of(40)
+    assert act.cpu().numpy()[:, :, :U].tolist() == [[list(range(U))] * 2] * 2
+
+
+def test_forced_selection_and_empty_mask_flag(sn):
+    w = synth.Workload("forced", "bf16", 3, (20, 30), 64, 4, 2, 32, 64, 2, 32, "all", 55)
+    inp = synth.generate(w, n_s_of)
+    kept_h, _ = parity.gate_lists(sn, inp)
+    g = np.random.default_rng(7)
+    U = n_s_of(50)
+    forced = np.stack([[np.sort(g.choice(50, U, replace=False)) for _ in range(2)]
+                       for _ in range(3)]).astype(np.int32)
+    O = sn.attend_fwd(inp.Q.cuda(), inp.K.cuda(), inp.V.cuda(), kept_h, dev(inp.ids),
+                      masks_dev(inp.masks), active_in=dev(forced), score_mode=1)
+    want = oracle.attend(inp.Q, inp.K, inp.V, kept_h.cpu().numpy(), inp.ids, inp.masks,
+                         score_mode=1, forced_active=forced)
+    assert parity.rel_err(O.float().cpu().numpy(), want) <= TOL["bf16"]
+    assert sn.last_status() == 0
+    # a sample whose mask is empty: zeros out, flag set, nothing faults
+    masks = inp.masks.copy()
+    masks[1] = 0
+    O = sn.attend_fwd(inp.Q.cuda(), inp.K.cuda(), inp.V.cuda(), kept_h, dev(inp.ids),
+                      masks_dev(masks), score_mode=1)
+    assert sn.last_status() & sentry.STATUS_BIT_EMPTY_MASK
+    assert torch.all(O[1] == 0)
+
+
+def test_results_are_deterministic_run_to_run(sn):
+    w = synth.config2().with_(B=16)
+    inp = synth.generate(w, n_s_of)
+    kept_h, kept_c = parity.gate_lists(sn, inp)
+    args = (inp.Q.cuda(), inp.K.cuda(), inp.V.cuda(), kept_h, dev(inp.ids), masks_dev(inp.masks),
+            dev(inp.sample_table), dev(inp.table_offsets))
+    O1 = sn.attend_fwd(*args).clone()
+    O2 = sn.attend_fwd(*args)
+    assert torch.equal(O1.view(torch.int16), O2.view(torch.int16))
+    fargs = (inp.X.cuda(), inp.W1.cuda(), inp.W2.cuda(), kept_c, dev(inp.list_of_sample),
+             dev(inp.ids), masks_dev(inp.masks))
+    Y1 = sn.ffn_fwd(*fargs).clone()
+    Y2 = sn.ffn_fwd(*fargs)
+    assert torch.equal(Y1.view(torch.int16), Y2.view(torch.int16))
