@@ -1,0 +1,482 @@
+#!/usr/bin/env python
+"""Benchmark of the pruned-layer hot path (gate selection -> sparse GQA attention ->
+channel-compacted FFN) through libsentry's C ABI on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 4] [--impl ours|reference]
+
+One "step" = one pass of the whole path over one batch of the chosen synthetic
+workload.  Prints ONE JSON line (rank 0).  `value` is whole-job present-tokens/s
+with inputs resident in HBM; `e2e` is the same through the public API with pinned
+host buffers and host<->device copies inside the timed region; `roofline` is the
+dominant kernel against the measured peak; `cpu_baseline` is the float64 oracle on
+a bounded sample of the same workload on this machine's host cores.
+
+With N > 1 (torchrun) every rank runs the full batch of the workload on its own
+GPU (weak scaling, no data-path collective); time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# --------------------------------------------------------------------------- model
+def work_model(w: synth.Workload, masks: np.ndarray, kept_heads: np.ndarray, num_active) -> dict:
+    """Algorithmic work of one step: present tokens, useful FLOPs and the bytes each
+    kernel has to move (what the method needs, not what a kernel happens to touch)."""
+    e = 4 if w.dtype == "f32" else 2
+    r = w.Hq // w.Hk
+    tokens = 0
+    att_flops = ffn_flops = 0.0
+    b_score = b_core = b_ffn_rows = 0.0
+    n_masks = len(masks)
+    for b in range(n_masks):
+        tv = synth.present_count(w, int(masks[b]))
+        U = num_active(tv)
+        G = len(set(int(h) // r for h in kept_heads[b]))
+        tokens += tv
+        att_flops += w.k_h * (2.0 * tv * U * w.d + 4.0 * U * tv * w.d) + G * tv * w.d
+        ffn_flops += 4.0 * w.D * w.k_c * tv
+        # score pass: Q of kept heads + K of referenced groups in, one fp32 score per (head, token) out
+        b_score += e * w.d * tv * (w.k_h + G) + 4.0 * w.k_h * tv
+        # core: K, V of referenced groups + active Q rows + scores in, O of kept heads out
+        b_core += e * w.d * tv * (2 * G + w.k_h) + e * w.d * U * w.k_h + 4.0 * w.k_h * tv
+        b_ffn_rows += 2.0 * w.D * e * tv
+    n_lists = len(set(int(m) for m in masks))
+    b_weights = 2.0 * w.D * w.k_c * e * n_lists
+    att_bytes = sum(e * w.d * synth.present_count(w, int(masks[b])) *
+                    (2 * w.k_h + 2 * len(set(int(h) // r for h in kept_heads[b])))
+                    for b in range(n_masks))
+    return {"tokens": tokens, "att_flops": att_flops, "ffn_flops": ffn_flops,
+            "att_bytes": float(att_bytes),
+            "kernel_bytes": {"attend_score": b_score, "attend_core": b_core,
+                             "ffn_main": b_ffn_rows + b_weights,
+                             "ffn_prepack": 2 * b_weights,
+                             "gate_expand": 4.0 * (n_masks * w.k_h + n_lists * w.k_c)},
+            "kernel_flops": {"ffn_main": ffn_flops}}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# -------------------------------------------------------------------------- clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML every 20 ms."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.samples = index, False, []
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception as ex:  # pragma: no cover
+            self.err = repr(ex)
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                sm = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                util = nv.nvmlDeviceGetUtilizationRates(self.h).gpu
+                self.samples.append((time.time(), sm, int(reasons), util))
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def summary(self, t0: float, t1: float) -> dict:
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml_unavailable"]}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1] or \
+                 [s for s in self.samples if s[3] >= 50] or self.samples
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        reasons = [n for b, n in names.items() if bits & b]
+        return {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": float(self.max_sm),
+                "reasons": reasons, "samples": len(inside)}
+
+
+# ---------------------------------------------------------------------- distributed
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), \
+        int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate(local_units: float, local_ms: float, device: str):
+    """Whole-job units (sum over ranks) and time (max over ranks).  Works on any
+    initialised backend (nccl on GPU, gloo on CPU); a no-op without one."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return local_units, local_ms
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(u.item()), float(t.item())
+
+
+def barrier_sync():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------------ reference
+def oracle_sample_run(inp: synth.Inputs, sel: np.ndarray, kept_h: np.ndarray, kept_c: np.ndarray):
+    """The oracle, as it stands, on the samples `sel` of the workload: gate + attend + ffn."""
+    import oracle
+    w = inp.w
+    masks = inp.masks[sel]
+    kh = oracle.gate_select(inp.scores_heads, masks, w.k_h)
+    kc = oracle.gate_select(inp.scores_ch, inp.subsets, w.k_c)
+    oracle.attend(inp.Q[sel], inp.K[sel], inp.V[sel], kh, inp.ids, masks, c=w.c,
+                  sample_table=inp.sample_table, table_offsets=inp.table_offsets)
+    oracle.ffn(inp.X[sel], inp.W1, inp.W2, kc, inp.list_of_sample[sel], inp.ids, masks)
+    return int(sum(synth.present_count(w, int(m)) for m in masks))
+
+
+def cpu_sample_inputs(w: synth.Workload, n_max: int):
+    """A small CPU batch with the workload's shapes and subset mix (first n_max samples of a
+    stratified order), for timing the oracle."""
+    import oracle
+    wb = w.with_(B=min(w.B, max(n_max, 1)))
+    if w.mask_rule == "thirds":  # keep all subsets represented in a short batch
+        wb = wb.with_(B=min(w.B, max(n_max, 3)))
+    inp = synth.generate(wb, lambda tv: oracle.num_active(tv, w.c))
+    return inp
+
+
+def time_oracle(w: synth.Workload, budget_s: float):
+    """Time the oracle on a bounded sample (~budget_s of CPU work).  Returns
+    (tokens/s, cores, description)."""
+    import oracle
+    cores = oracle.threads()
+    inp = cpu_sample_inputs(w, 3 * cores)
+    n_avail = inp.w.B
+    t0 = time.perf_counter()
+    tok = oracle_sample_run(inp, np.arange(min(cores, n_avail)), None, None)
+    t_probe = time.perf_counter() - t0
+    n = min(cores, n_avail)
+    reps = 1
+    if t_probe < budget_s / 2 and n_avail > n:
+        n = int(min(n_avail, max(n, n * (budget_s / max(t_probe, 1e-3)) // 1)))
+    sel = np.arange(n)
+    t0 = time.perf_counter()
+    tok = oracle_sample_run(inp, sel, None, None)
+    dt = time.perf_counter() - t0
+    while dt * (reps + 1) < budget_s and reps < 50 and dt < 1.0:
+        tok += oracle_sample_run(inp, sel, None, None)
+        reps += 1
+        dt = time.perf_counter() - t0
+    return tok / dt, cores, "%d samples x %d passes of %s (gate+attend+ffn, float64, OpenMP over samples)" % (
+        n, reps, w.name)
+
+
+def run_reference(args, w: synth.Workload):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    cores = oracle.threads()
+    total_budget = 150.0
+    inp = cpu_sample_inputs(w, 3 * cores)
+    t0 = time.perf_counter()
+    oracle_sample_run(inp, np.arange(1), None, None)
+    t_one = time.perf_counter() - t0
+    per_step = total_budget / max(1, args.steps + args.warmup)
+    n = int(max(1, min(inp.w.B, (per_step / max(t_one / 1.0, 1e-4)) * min(cores, inp.w.B) // 1)))
+    n = max(1, min(n, inp.w.B))
+    sel = np.arange(n)
+    for _ in range(args.warmup):
+        oracle_sample_run(inp, sel, None, None)
+    t0 = time.perf_counter()
+    tok = 0
+    for _ in range(args.steps):
+        tok += oracle_sample_run(inp, sel, None, None)
+    dt = time.perf_counter() - t0
+    val = tok / dt
+    line = {"impl": "reference", "metric": "pruned_layer_tokens_per_s", "value": val, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * dt / max(1, args.steps), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sample": "%d samples per step" % n},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": "%d samples of %s per step, %d steps" % (n, w.name, args.steps)},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- ours
+class DeviceSet:
+    """One resident copy of a step's inputs and outputs."""
+
+    def __init__(self, inp: synth.Inputs, dev: str, src: "DeviceSet" = None):
+        w = inp.w
+        dt = synth.torch_dtype(w)
+        if src is None:
+            self.Q, self.K, self.V, self.X = (t.to(dev) for t in (inp.Q, inp.K, inp.V, inp.X))
+        else:
+            self.Q, self.K, self.V, self.X = (t.clone() for t in (src.Q, src.K, src.V, src.X))
+        self.O = torch.empty((w.B, w.k_h, w.T, w.d), dtype=dt, device=dev)
+        self.Y = torch.empty((w.B, w.T, w.D), dtype=dt, device=dev)
+        self.kept_h = torch.empty((w.B, w.k_h), dtype=torch.int32, device=dev)
+        self.kept_c = torch.empty((len(inp.subsets), w.k_c), dtype=torch.int32, device=dev)
+
+    def nbytes(self):
+        return sum(t.numel() * t.element_size() for t in (self.Q, self.K, self.V, self.X, self.O, self.Y))
+
+
+def run_ours(args, w: synth.Workload):
+    import paper_2604_08971_b200 as sentry
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libsentry has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    sentry.build()
+    sn = sentry.Sentry(local_rank)
+    n_s_of = lambda tv: sentry.num_active_queries(tv, w.c)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    # inputs: generated on the device (seed offset by rank), resident before timing
+    inp = synth.generate(w.with_(seed=w.seed + 1000 * rank), n_s_of, device=dev)
+    ids = torch.as_tensor(inp.ids, device=dev)
+    masks = torch.as_tensor(inp.masks.astype(np.int64).astype(np.int32), device=dev)
+    subsets = torch.as_tensor(inp.subsets.astype(np.int64).astype(np.int32), device=dev)
+    los = torch.as_tensor(inp.list_of_sample, device=dev)
+    sh, sc = torch.as_tensor(inp.scores_heads, device=dev), torch.as_tensor(inp.scores_ch, device=dev)
+    tbl, offs = torch.as_tensor(inp.sample_table, device=dev), torch.as_tensor(inp.table_offsets, device=dev)
+    W1, W2 = inp.W1, inp.W2
+    base = DeviceSet(inp, dev)
+    set_bytes = base.nbytes()
+    n_sets = 1 if set_bytes >= 2 * L2_BYTES else int(min(16, -(-2 * L2_BYTES // set_bytes)))
+    sets = [base] + [DeviceSet(inp, dev, base) for _ in range(n_sets - 1)]
+    hpg = w.Hq // w.Hk
+    launches = [0]
+
+    def step(s: DeviceSet, count=False):
+        n = 0
+        sn.gate_select(sh, masks, w.k_h, kept=s.kept_h)
+        n += sn.last_launch_count()
+        sn.gate_select(sc, subsets, w.k_c, kept=s.kept_c)
+        n += sn.last_launch_count()
+        sn.attend_fwd(s.Q, s.K, s.V, s.kept_h, ids, masks, tbl, offs, c=w.c, O=s.O)
+        n += sn.last_launch_count()
+        sn.ffn_fwd(s.X, W1, W2, s.kept_c, los, ids, masks, Y=s.Y)
+        n += sn.last_launch_count()
+        if count:
+            launches[0] = n
+
+    # workspace sized once, before any capture
+    step(sets[0], count=True)
+    torch.cuda.synchronize()
+    assert sn.last_status() == 0, "device status word set during warm-up"
+
+    graphs = None
+    if not args.no_graph:
+        graphs = []
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for s in sets:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step(s)
+                graphs.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    def run_steps(n):
+        for i in range(n):
+            if graphs is not None:
+                graphs[i % n_sets].replay()
+            else:
+                step(sets[i % n_sets])
+
+    # ---- device-resident timing
+    run_steps(max(3, args.warmup))
+    barrier_sync()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    ev0.record()
+    run_steps(args.steps)
+    ev1.record()
+    barrier_sync()
+    t_wall1 = time.time()
+    local_ms = ev0.elapsed_time(ev1)
+    kept_h_host = sets[0].kept_h.cpu().numpy()
+    wm = work_model(w, inp.masks, kept_h_host, n_s_of)
+    total_tokens, ms = aggregate(float(wm["tokens"]) * args.steps, local_ms, dev)
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    # ---- per-kernel pass (same steps, events around every kernel, no graph)
+    sn.profile_enable(True)
+    for i in range(3):
+        step(sets[i % n_sets])
+    sn.profile_read()
+    n_prof = min(args.steps, 50)
+    for i in range(n_prof):
+        step(sets[i % n_sets])
+    prof = sn.profile_read()
+    sn.profile_enable(False)
+
+    # ---- end to end: pinned host buffers in, results out, every step
+    host_in = [t.cpu().pin_memory() for t in (base.Q, base.K, base.V, base.X)]
+    small_in = [t.cpu().pin_memory() for t in (ids, masks, subsets, los, sh, sc, tbl, offs, W1, W2)]
+    host_out = [torch.empty_like(base.O, device="cpu").pin_memory(),
+                torch.empty_like(base.Y, device="cpu").pin_memory()]
+    dsmall = [ids, masks, subsets, los, sh, sc, tbl, offs, W1, W2]
+    h2d = sum(t.numel() * t.element_size() for t in host_in + small_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+
+    def e2e_step():
+        for dst, src in zip((base.Q, base.K, base.V, base.X), host_in):
+            dst.copy_(src, non_blocking=True)
+        for dst, src in zip(dsmall, small_in):
+            dst.copy_(src, non_blocking=True)
+        step(base)
+        host_out[0].copy_(base.O, non_blocking=True)
+        host_out[1].copy_(base.Y, non_blocking=True)
+        torch.cuda.synchronize()
+
+    n_e2e = max(3, min(args.steps, 20))
+    for _ in range(3):
+        e2e_step()
+    barrier_sync()
+    ev0.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    ev1.record()
+    barrier_sync()
+    e2e_tokens, e2e_ms = aggregate(float(wm["tokens"]) * n_e2e, ev0.elapsed_time(ev1), dev)
+    status = sn.last_status()
+    sampler.stop_flag = True
+
+    if rank != 0:
+        return
+    peaks, peak_kind = load_peaks()
+    # dominant kernel = largest share of the per-kernel pass
+    per_kernel = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / n_prof,
+                      "share": v[0] / max(1e-9, sum(x[0] for x in prof.values()))}
+                  for k, v in prof.items()}
+    top = max(prof, key=lambda k: prof[k][0])
+    t_launch = prof[top][0] / prof[top][1] * 1e-3
+    if top == "ffn_main":
+        fl = wm["kernel_flops"]["ffn_main"]
+        by = wm["kernel_bytes"]["ffn_main"]
+        t_tensor, t_hbm = fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)
+        if t_tensor >= t_hbm and w.dtype == "bf16":
+            roof = {"bound": "tensor", "achieved": fl / t_launch / 1e12, "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s"}
+        else:
+            roof = {"bound": "hbm", "achieved": by / t_launch / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        by = wm["kernel_bytes"].get(top, 0.0)
+        roof = {"bound": "hbm", "achieved": by / t_launch / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof.update({"kernel": top, "frac": roof["achieved"] / roof["peak"], "traffic": None,
+                 "peak_source": "%s (burst figure; timed region is short)" % peak_kind,
+                 "ms_per_launch": t_launch * 1e3})
+    # whole-stage fractions from the same pass
+    t_att = sum(prof[k][0] for k in prof if k.startswith("attend")) / n_prof * 1e-3
+    t_ffn = sum(prof[k][0] for k in prof if k.startswith("ffn")) / n_prof * 1e-3
+    stages = {
+        "attend": {"ms": t_att * 1e3, "hbm_frac": wm["att_bytes"] / max(t_att, 1e-12) / 1e9 / peaks["hbm_gbs"],
+                   "useful_tflops": wm["att_flops"] / max(t_att, 1e-12) / 1e12},
+        "ffn": {"ms": t_ffn * 1e3,
+                "tensor_frac": wm["ffn_flops"] / max(t_ffn, 1e-12) / 1e12 / peaks["bf16_tflops"],
+                "useful_tflops": wm["ffn_flops"] / max(t_ffn, 1e-12) / 1e12}}
+
+    cpu = {"value": None, "unit": "tokens/s", "cores": None, "kind": "oracle", "sample": "skipped"}
+    if world == 1 and not args.no_cpu:
+        v, cores, what = time_oracle(w, args.cpu_budget)
+        cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": what}
+
+    value = total_tokens / (ms * 1e-3)
+    line = {
+        "metric": "pruned_layer_tokens_per_s", "value": value, "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "batch_per_gpu": w.B, "seq_len": w.T, "modalities": w.M,
+                   "d_model": w.D, "q_heads": w.Hq, "kv_heads": w.Hk, "head_dim": w.d, "d_ff": w.F,
+                   "kept_heads": w.k_h, "kept_channels": w.k_c, "mask_rule": w.mask_rule,
+                   "present_tokens_per_step_per_gpu": wm["tokens"], "parallelism": "replicas x%d" % world,
+                   "l2_policy": "rotating %d resident buffer sets, %.0f MB in total (> 126 MB L2)"
+                                % (n_sets, n_sets * set_bytes / 1e6),
+                   "cuda_graph": graphs is not None},
+        "useful_tflops": (wm["att_flops"] + wm["ffn_flops"]) * world * args.steps / (ms * 1e-3) / 1e12,
+        "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": n_e2e},
+        "gpu_launches": launches[0] * args.steps,
+        "clocks": clocks, "roofline": roof, "stages": stages, "kernels": per_kernel,
+        "cpu_baseline": cpu, "device_status": status,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default="4",
+                    help="1, 2, 3a|3b|3c, 4 (default: the full pruned encoder layer), 5:BxT")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    w = synth.by_name(args.config)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+        import torch.distributed as dist
+        if dist.is_available() and dist.is_initialized():
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

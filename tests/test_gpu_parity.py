@@ -73,7 +73,7 @@ def test_error_codes_no_launch(sn):
         sn.gate_select(scores, masks, 9)
     assert e.value.code == -2
     with pytest.raises(sentry.SentryError) as e:
-        sn.gate_select(scores, masks, 0)
+        sn.gate_select(scores, masks, 0, kept=torch.empty((2, 1), dtype=torch.int32, device="cuda"))
     assert e.value.code == -2
     Q = torch.zeros((1, 4, 8, 24), device="cuda")  # head_dim 24 unsupported
     K = torch.zeros((1, 2, 8, 24), device="cuda")
@@ -213,7 +213,7 @@ def test_forced_selection_and_empty_mask_flag(sn):
                       masks_dev(inp.masks), active_in=dev(forced), score_mode=1)
     want = oracle.attend(inp.Q, inp.K, inp.V, kept_h.cpu().numpy(), inp.ids, inp.masks,
                          score_mode=1, forced_active=forced)
-    assert parity.rel_err(O.float().cpu().numpy(), want) <= TOL["bf16"]
+    assert parity.rel_err(O.float().cpu().numpy(), want, "bf16") <= TOL["bf16"]
     assert sn.last_status() == 0
     # a sample whose mask is empty: zeros out, flag set, nothing faults
     masks = inp.masks.copy()
