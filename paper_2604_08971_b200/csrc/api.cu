@@ -235,7 +235,8 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
                                  : (active_out != nullptr ? active_out : ws_active);
     SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
     cudaStream_t st = (cudaStream_t)stream;
-    rc = launch_attend_generic(ctx, a, st);
+    a.active_out_user = active_out;
+    rc = attend_bf16_supported(*desc) ? launch_attend_bf16(ctx, a, st) : launch_attend_generic(ctx, a, st);
     if (rc != SENTRY_OK) return rc;
     if (a.selection_given && active_out != nullptr && active_out != active_in) {
         SENTRY_CUDA_TRY(cudaMemcpyAsync(active_out, active_in,

@@ -1,0 +1,630 @@
+// SentryAttend (Section 4.4, Eq. 6) for bf16 tensors: the fast path.
+//
+// Two kernels per call:
+//   score  one CTA per (sample, KV group, 256 query positions).  The group's present K rows are
+//          staged once in shared memory (16-byte async copies, XOR-swizzled rows); each thread
+//          owns one query position and scores it against its sampled keys for ALL kept heads of
+//          the group at once, so a sampled key row is fetched from shared memory once per group,
+//          not once per head.       M_i = max_j s_ij - mean_j s_ij   (fp32)
+//   core   one CTA per (sample, KV group).  Prologue: top-U selection per kept head (warp-level
+//          threshold search on order-preserving keys; ties -> lower index).  Main loop: K/V tiles
+//          of 64 present keys stream through shared memory once per GROUP and are shared by the
+//          kept heads; the U active rows of each head run  softmax(q K^T / sqrt d) V  on the
+//          warp-level tensor-core MMA with an online softmax (fp32 state in registers).  The
+//          column sums of V ride along and give the context vector.  Epilogue: active rows,
+//          context rows (mean of V_g) and zero rows (absent modalities) are written with
+//          16-byte stores.  Pruned heads and unreferenced KV groups are never touched.
+//
+// The contraction here is tiny (U <= 45 rows per head against T_v keys): the path is bound by
+// shared-memory gathers and HBM traffic, not by tensor throughput, which is why it uses the
+// register-resident warp MMA rather than TMEM accumulators.
+#include <math.h>
+
+#include "common.cuh"
+#include "ptx/sm100.cuh"
+
+namespace {
+
+constexpr int kMaxRK = 4;          // kept heads of one KV group handled per CTA
+constexpr int kScoreThreads = 128;
+constexpr int kCoreThreads = 256;
+constexpr int kCoreWarps = kCoreThreads / 32;
+constexpr int kKeyTile = 64;
+constexpr int kMaxActive = 48;     // U <= 45 for T <= 8103 with c = 5 (checked on the host)
+
+// Row layout in shared memory: rows of D bf16, 16-byte chunks XOR-swizzled so that both
+// 8-consecutive-row matrix loads and random row gathers spread over the banks.
+template <int D>
+struct Sw {
+    static constexpr int RB = D * 2;          // row bytes
+    static constexpr int CPR = RB / 16;       // 16-byte chunks per row
+    static constexpr int RPL = 128 / RB;      // rows per 128-byte line (>= 1 for D <= 64)
+    __device__ static __forceinline__ uint32_t off(int row, int c) {
+        return (uint32_t)row * RB + (uint32_t)((c ^ ((row / RPL) & (CPR - 1))) << 4);
+    }
+};
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = __uint_as_float(w[j] << 16);
+        f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// Kept heads of KV group g among kept_heads[b, :]: their head ids and kept-list slots.
+__device__ __forceinline__ int group_heads(const int32_t* kept, int k_h, int r, int g, int Hq,
+                                           int (&hs)[kMaxRK], int (&khs)[kMaxRK], bool& bad) {
+    int rk = 0;
+    bad = false;
+    for (int j = 0; j < k_h; ++j) {
+        const int h = kept[j];
+        if (h < 0 || h >= Hq) { bad = true; continue; }
+        if (h / r == g && rk < kMaxRK) { hs[rk] = h; khs[rk] = j; ++rk; }
+    }
+    return rk;
+}
+
+// ------------------------------------------------------------------------------------ score
+template <int D, int RK>
+__device__ __forceinline__ void score_pass(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
+                                           const uint16_t* s_valid, uint32_t ks_addr, int seg_rows,
+                                           int Tv, int Tlen, int b, int g, int Hq, int Hk,
+                                           const int* hs, const int* khs,
+                                           const int32_t* tbl_row, int cnt, int score_mode, int p,
+                                           int k_h, float* __restrict__ mscore, unsigned int* status) {
+    using S = Sw<D>;
+    const bool act = p < Tv;
+    float q[RK][D];
+    float mx[RK], sum[RK];
+#pragma unroll
+    for (int h = 0; h < RK; ++h) { mx[h] = -INFINITY; sum[h] = 0.f; }
+    if (act) {
+        const int tok = s_valid[p];
+#pragma unroll
+        for (int h = 0; h < RK; ++h) {
+            const uint4* src = reinterpret_cast<const uint4*>(Q + (((size_t)b * Hq + hs[h]) * Tlen + tok) * D);
+#pragma unroll
+            for (int c = 0; c < S::CPR; ++c) {
+                float f[8];
+                unpack8(__ldg(src + c), f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) q[h][8 * c + e] = f[e];
+            }
+        }
+    }
+    const float scale = rsqrtf((float)D);
+    const __nv_bfloat16* Kg = K + ((size_t)b * Hk + g) * Tlen * D;
+    for (int seg0 = 0; seg0 < Tv; seg0 += seg_rows) {
+        const int seg_n = min(seg_rows, Tv - seg0);
+        __syncthreads();  // the previous segment is no longer being read
+        for (int i = threadIdx.x; i < seg_n * S::CPR; i += blockDim.x) {
+            const int row = i / S::CPR, c = i % S::CPR;
+            ptx::cp_async_16(ks_addr + S::off(row, c), Kg + (size_t)s_valid[seg0 + row] * D + c * 8);
+        }
+        ptx::cp_async_wait_all();
+        __syncthreads();
+        if (act) {
+            for (int a = 0; a < cnt; ++a) {
+                int pj = score_mode == 0 ? tbl_row[a] : a;
+                if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
+                const int row = pj - seg0;
+                if (row < 0 || row >= seg_n) continue;
+                float dot[RK];
+#pragma unroll
+                for (int h = 0; h < RK; ++h) dot[h] = 0.f;
+#pragma unroll
+                for (int c = 0; c < S::CPR; ++c) {
+                    float f[8];
+                    unpack8(lds128(ks_addr + S::off(row, c)), f);
+#pragma unroll
+                    for (int h = 0; h < RK; ++h)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) dot[h] = fmaf(q[h][8 * c + e], f[e], dot[h]);
+                }
+#pragma unroll
+                for (int h = 0; h < RK; ++h) {
+                    const float s = dot[h] * scale;
+                    mx[h] = fmaxf(mx[h], s);
+                    sum[h] += s;
+                }
+            }
+        }
+    }
+    if (act) {
+#pragma unroll
+        for (int h = 0; h < RK; ++h)
+            mscore[((size_t)b * k_h + khs[h]) * Tlen + p] = mx[h] - sum[h] / (float)cnt;
+    }
+}
+
+// grid (ceil(T/threads), B*Hk).  Dynamic smem: valid list (2T bytes, 16-aligned) + K segment.
+template <int D>
+__global__ void __launch_bounds__(kScoreThreads, 2)
+attend_score_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
+                         const int32_t* __restrict__ kept_heads, const int32_t* __restrict__ ids,
+                         const uint32_t* __restrict__ masks, const int32_t* __restrict__ table,
+                         const int64_t* __restrict__ offsets, int n_subsets, int Tlen, int Hq, int Hk,
+                         int k_h, int c, int score_mode, int seg_rows, float* __restrict__ mscore,
+                         unsigned int* status) {
+    extern __shared__ __align__(128) uint8_t s_raw[];
+    __shared__ int red[66];
+    uint16_t* s_valid = reinterpret_cast<uint16_t*>(s_raw);
+    const uint32_t ks_addr = ptx::smem_u32(s_raw) + (uint32_t)((((size_t)Tlen * 2 + 127) / 128) * 128);
+    const int b = blockIdx.y / Hk, g = blockIdx.y % Hk;
+    const uint32_t mask = masks[b];
+    const int Tv = block_build_valid(ids, Tlen, mask, s_valid, red);
+    if (Tv == 0 || (int)(blockIdx.x * blockDim.x) >= Tv) return;
+    int hs[kMaxRK], khs[kMaxRK];
+    bool bad;
+    const int rk = group_heads(kept_heads + (size_t)b * k_h, k_h, Hq / Hk, g, Hq, hs, khs, bad);
+    if (bad && threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+    if (rk == 0) return;
+    const int n_s = sentry_num_active(Tv, c);
+    const int cnt = score_mode == 0 ? n_s : Tv;
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    const int32_t* tbl_row = nullptr;
+    if (score_mode == 0) {
+        if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) {
+            if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+            return;
+        }
+        tbl_row = table + offsets[mask] + (size_t)min(p, Tv - 1) * n_s;
+    }
+    // The q rows of a pass live in registers: up to 4 heads x 32 dims, or 2 heads x 64 dims.
+#define SCORE_PASS(N, H0, H1, H2, H3)                                                              \
+    {                                                                                              \
+        const int hs_[kMaxRK] = {hs[H0], hs[H1], hs[H2], hs[H3]};                                  \
+        const int khs_[kMaxRK] = {khs[H0], khs[H1], khs[H2], khs[H3]};                             \
+        score_pass<D, N>(Q, K, s_valid, ks_addr, seg_rows, Tv, Tlen, b, g, Hq, Hk, hs_, khs_,      \
+                         tbl_row, cnt, score_mode, p, k_h, mscore, status);                        \
+    }
+    if constexpr (D == 64) {
+        if (rk == 1) SCORE_PASS(1, 0, 0, 0, 0)
+        else SCORE_PASS(2, 0, 1, 0, 0)
+        if (rk == 3) SCORE_PASS(1, 2, 2, 2, 2)
+        else if (rk == 4) SCORE_PASS(2, 2, 3, 2, 2)
+    } else {
+        switch (rk) {
+            case 1: SCORE_PASS(1, 0, 0, 0, 0) break;
+            case 2: SCORE_PASS(2, 0, 1, 0, 0) break;
+            case 3: SCORE_PASS(3, 0, 1, 2, 0) break;
+            default: SCORE_PASS(4, 0, 1, 2, 3) break;
+        }
+    }
+#undef SCORE_PASS
+}
+
+// ------------------------------------------------------------------------------------- core
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t (&r)[2]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];"
+                 : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Warp-level top-k over n order keys in shared memory (larger key first, ties -> lower index).
+// Writes remap[index] of the selected entries to out[0..k) in ascending index order.
+__device__ inline void warp_select_topk(const uint32_t* keys, int n, int k, int32_t* out,
+                                        const uint16_t* remap) {
+    const int lane = threadIdx.x & 31;
+    uint32_t t = 0;
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t cand = t | (1u << bit);
+        int cnt = 0;
+        for (int i = lane; i < n; i += 32) cnt += (keys[i] >= cand);
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (cnt >= k) t = cand;
+    }
+    int gt = 0;
+    for (int i = lane; i < n; i += 32) gt += (keys[i] > t);
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    const int need_eq = k - gt;
+    int base = 0, eq_seen = 0;
+    for (int i0 = 0; i0 < n; i0 += 32) {
+        const int i = i0 + lane;
+        const uint32_t key = i < n ? keys[i] : 0u;
+        const bool is_eq = i < n && key == t, is_gt = i < n && key > t;
+        const unsigned em = __ballot_sync(0xffffffffu, is_eq);
+        const bool keep = is_gt || (is_eq && eq_seen + __popc(em & ((1u << lane) - 1u)) < need_eq);
+        const unsigned km = __ballot_sync(0xffffffffu, keep);
+        if (keep) out[base + __popc(km & ((1u << lane) - 1u))] = (int32_t)remap[i];
+        base += __popc(km);
+        eq_seen += __popc(em);
+    }
+    __syncwarp();
+}
+
+template <int D>
+struct CoreSmem {
+    static constexpr int TILE_BYTES = kKeyTile * D * 2;      // one K or V tile
+    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;       // K + V
+    static constexpr int PIPE_BYTES = 2 * STAGE_BYTES;       // double buffered
+};
+
+// grid B*Hk.  Dynamic smem: valid[T] u16 | kind[T] u8 | actbits[4][T/32] u32 | union{keys, KV pipe}
+template <int D>
+__global__ void __launch_bounds__(kCoreThreads)
+attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
+                        const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ kept_heads,
+                        const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks,
+                        const float* __restrict__ mscore, const int32_t* __restrict__ active_in,
+                        int32_t* __restrict__ active_out, int Tlen, int Hq, int Hk, int k_h, int c,
+                        int U_max, __nv_bfloat16* __restrict__ O, unsigned int* status) {
+    using S = Sw<D>;
+    using CS = CoreSmem<D>;
+    constexpr int NT = D / 8;        // n-tiles of the output (8 dims each)
+    constexpr int KS = D / 16;       // k-steps of q.k
+    extern __shared__ __align__(128) uint8_t s_raw[];
+    __shared__ int red[66];
+    __shared__ int32_t s_act[kMaxRK][kMaxActive];
+    __shared__ float s_vpart[kCoreThreads / (D / 2)][D];   // partial column sums of V
+    __shared__ __align__(16) __nv_bfloat16 s_mean[D];
+
+    const int words = (Tlen + 31) / 32;
+    size_t o = 0;
+    uint16_t* s_valid = reinterpret_cast<uint16_t*>(s_raw + o); o += (((size_t)Tlen * 2 + 127) / 128) * 128;
+    uint8_t* s_kind = s_raw + o;                                o += (((size_t)Tlen + 127) / 128) * 128;
+    uint32_t* s_abits = reinterpret_cast<uint32_t*>(s_raw + o); o += (((size_t)kMaxRK * words * 4 + 127) / 128) * 128;
+    uint8_t* s_union = s_raw + o;
+    uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_union);
+    const uint32_t pipe_addr = ptx::smem_u32(s_union);
+
+    const int b = blockIdx.x / Hk, g = blockIdx.x % Hk;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int Tv = block_build_valid(ids, Tlen, masks[b], s_valid, red);
+    int hs[kMaxRK], khs[kMaxRK];
+    bool bad;
+    const int rk = group_heads(kept_heads + (size_t)b * k_h, k_h, Hq / Hk, g, Hq, hs, khs, bad);
+    if (rk == 0) return;
+    if (Tv == 0) {  // no modality present: zero rows, flag
+        for (int hh = 0; hh < rk; ++hh) {
+            uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D);
+            for (int i = threadIdx.x; i < Tlen * S::CPR; i += blockDim.x) dst[i] = make_uint4(0, 0, 0, 0);
+            if (active_out != nullptr && active_in == nullptr)
+                for (int i = threadIdx.x; i < U_max; i += blockDim.x)
+                    active_out[((size_t)b * k_h + khs[hh]) * U_max + i] = -1;
+        }
+        if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
+        return;
+    }
+    const int U = sentry_num_active(Tv, c);
+
+    for (int t = threadIdx.x; t < Tlen; t += blockDim.x) s_kind[t] = 0;
+    for (int i = threadIdx.x; i < kMaxRK * words; i += blockDim.x) s_abits[i] = 0u;
+    for (int i = threadIdx.x; i < kMaxRK * kMaxActive; i += blockDim.x) (&s_act[0][0])[i] = -1;
+    __syncthreads();
+    for (int p = threadIdx.x; p < Tv; p += blockDim.x) s_kind[s_valid[p]] = 1;
+
+    // ---- selection of the active rows (Section 4.4: the U queries with the largest score)
+    if (active_in == nullptr) {
+        for (int hh = 0; hh < rk; ++hh) {
+            const float* m = mscore + ((size_t)b * k_h + khs[hh]) * Tlen;
+            for (int p = threadIdx.x; p < Tv; p += blockDim.x) s_keys[(size_t)hh * Tv + p] = sentry_order_key(m[p]);
+        }
+        __syncthreads();
+        if (warp < rk) warp_select_topk(s_keys + (size_t)warp * Tv, Tv, U, s_act[warp], s_valid);
+        __syncthreads();
+        if (active_out != nullptr)
+            for (int i = threadIdx.x; i < rk * U_max; i += blockDim.x) {
+                const int hh = i / U_max, a = i % U_max;
+                active_out[((size_t)b * k_h + khs[hh]) * U_max + a] = a < U ? s_act[hh][a] : -1;
+            }
+    } else {
+        __syncthreads();
+        for (int i = threadIdx.x; i < rk * kMaxActive; i += blockDim.x) {
+            const int hh = i / kMaxActive, a = i % kMaxActive;
+            int t = a < U_max ? active_in[((size_t)b * k_h + khs[hh]) * U_max + a] : -1;
+            if (t >= 0 && (t >= Tlen || s_kind[t] == 0)) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); t = -1; }
+            s_act[hh][a] = t;
+        }
+        __syncthreads();
+    }
+    for (int i = threadIdx.x; i < rk * kMaxActive; i += blockDim.x) {
+        const int hh = i / kMaxActive, t = s_act[hh][i % kMaxActive];
+        if (t >= 0) atomicOr(&s_abits[hh * words + (t >> 5)], 1u << (t & 31));
+    }
+    __syncthreads();   // s_keys is dead from here on: the union becomes the K/V pipe
+
+    // ---- row tiles of this warp: tile tt -> (head slot, 16 active rows)
+    const int WT = (min(U, kMaxActive) + 15) / 16;     // row tiles per head (<= 3)
+    const int n_tiles = rk * WT;
+    const int gq = lane >> 2, tq = lane & 3;
+    uint32_t qf[2][KS][4];
+    float acc[2][NT][4];
+    float m_run[2][2], l_run[2][2];
+    int tile_head[2], tile_row0[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int tt = warp + j * kCoreWarps;
+        tile_head[j] = tt < n_tiles ? tt / WT : -1;
+        tile_row0[j] = tt < n_tiles ? (tt % WT) * 16 : 0;
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[j][n][e] = 0.f;
+        m_run[j][0] = m_run[j][1] = -INFINITY;
+        l_run[j][0] = l_run[j][1] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) qf[j][ks][e] = 0u;
+        if (tile_head[j] >= 0) {
+            const int hh = tile_head[j];
+            const __nv_bfloat16* Qh = Q + ((size_t)b * Hq + hs[hh]) * Tlen * D;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int a = tile_row0[j] + gq + half * 8;
+                const int t = a < kMaxActive ? s_act[hh][a] : -1;
+                if (t >= 0) {
+                    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(Qh + (size_t)t * D);
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        qf[j][ks][half] = __ldg(qrow + ks * 8 + tq);          // cols 16ks + 2t, +1
+                        qf[j][ks][half + 2] = __ldg(qrow + ks * 8 + 4 + tq);  // cols 16ks + 8 + 2t, +1
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- stream K/V tiles of 64 present keys
+    const __nv_bfloat16* Kg = K + ((size_t)b * Hk + g) * Tlen * D;
+    const __nv_bfloat16* Vg = V + ((size_t)b * Hk + g) * Tlen * D;
+    const int n_kt = (Tv + kKeyTile - 1) / kKeyTile;
+    auto load_tile = [&](int kt, int stage) {
+        const uint32_t kbase = pipe_addr + stage * CS::STAGE_BYTES;
+        const uint32_t vbase = kbase + CS::TILE_BYTES;
+        const int rows = min(kKeyTile, Tv - kt * kKeyTile);
+        for (int i = threadIdx.x; i < kKeyTile * S::CPR; i += blockDim.x) {
+            const int row = i / S::CPR, cc = i % S::CPR;
+            if (row < rows) {
+                const size_t goff = (size_t)s_valid[kt * kKeyTile + row] * D + cc * 8;
+                ptx::cp_async_16(kbase + S::off(row, cc), Kg + goff);
+                ptx::cp_async_16(vbase + S::off(row, cc), Vg + goff);
+            } else {  // keys past the end: zeros (masked out of the softmax, add nothing to sums)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(kbase + S::off(row, cc)), "r"(0) : "memory");
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + S::off(row, cc)), "r"(0) : "memory");
+            }
+        }
+        ptx::cp_async_commit();
+    };
+    // V column sums: thread -> (dim pair, key residue)
+    constexpr int DP = D / 2;
+    const int vs_dp = threadIdx.x % DP, vs_k0 = threadIdx.x / DP;
+    constexpr int VS_STRIDE = kCoreThreads / DP;
+    float vsum0 = 0.f, vsum1 = 0.f;
+
+    const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;  // scale * log2(e)
+    load_tile(0, 0);
+    for (int kt = 0; kt < n_kt; ++kt) {
+        const int stage = kt & 1;
+        if (kt + 1 < n_kt) { load_tile(kt + 1, stage ^ 1); ptx::cp_async_wait_group<1>(); }
+        else ptx::cp_async_wait_group<0>();
+        __syncthreads();
+        const uint32_t kbase = pipe_addr + stage * CS::STAGE_BYTES;
+        const uint32_t vbase = kbase + CS::TILE_BYTES;
+        const int key0 = kt * kKeyTile;
+        // column sums of V (padding rows are zero)
+        for (int row = vs_k0; row < kKeyTile; row += VS_STRIDE) {
+            uint32_t w;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(vbase + S::off(row, vs_dp >> 2) + (vs_dp & 3) * 4));
+            vsum0 += __uint_as_float(w << 16);
+            vsum1 += __uint_as_float(w & 0xffff0000u);
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (tile_head[j] < 0) continue;   // warp-uniform
+            // S = q K^T for 16 rows x 64 keys
+            float s[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+                const int krow = nt * 8 + (lane & 7);
+                if constexpr (D == 32) {
+                    uint32_t bfr[4];
+                    ldmatrix_x4(kbase + S::off(krow, lane >> 3), bfr);
+                    mma_bf16_16816(s[nt], qf[j][0], bfr[0], bfr[1]);
+                    mma_bf16_16816(s[nt], qf[j][1], bfr[2], bfr[3]);
+                } else if constexpr (D == 16) {
+                    uint32_t bfr[2];
+                    ldmatrix_x2(kbase + S::off(krow, (lane >> 3) & 1), bfr);
+                    mma_bf16_16816(s[nt], qf[j][0], bfr[0], bfr[1]);
+                } else {  // D == 64
+                    uint32_t bfr[4];
+                    ldmatrix_x4(kbase + S::off(krow, lane >> 3), bfr);
+                    mma_bf16_16816(s[nt], qf[j][0], bfr[0], bfr[1]);
+                    mma_bf16_16816(s[nt], qf[j][1], bfr[2], bfr[3]);
+                    ldmatrix_x4(kbase + S::off(krow, 4 + (lane >> 3)), bfr);
+                    mma_bf16_16816(s[nt], qf[j][2], bfr[0], bfr[1]);
+                    mma_bf16_16816(s[nt], qf[j][3], bfr[2], bfr[3]);
+                }
+            }
+            // online softmax over this tile (rows gq and gq+8), base-2 exponent
+            float mt[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int key = key0 + nt * 8 + tq * 2 + (e & 1);
+                    s[nt][e] = key < Tv ? s[nt][e] * sl2 : -INFINITY;
+                    mt[e >> 1] = fmaxf(mt[e >> 1], s[nt][e]);
+                }
+            float corr[2];
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+                mt[h2] = fmaxf(mt[h2], __shfl_xor_sync(0xffffffffu, mt[h2], 1));
+                mt[h2] = fmaxf(mt[h2], __shfl_xor_sync(0xffffffffu, mt[h2], 2));
+                const float m_new = fmaxf(m_run[j][h2], mt[h2]);
+                corr[h2] = fast_exp2(m_run[j][h2] - m_new);   // 0 on the first tile
+                m_run[j][h2] = m_new;
+                l_run[j][h2] *= corr[h2];
+            }
+            float lsum[2] = {0.f, 0.f};
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    s[nt][e] = fast_exp2(s[nt][e] - m_run[j][e >> 1]);
+                    lsum[e >> 1] += s[nt][e];
+                }
+            l_run[j][0] += lsum[0];
+            l_run[j][1] += lsum[1];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                acc[j][n][0] *= corr[0]; acc[j][n][1] *= corr[0];
+                acc[j][n][2] *= corr[1]; acc[j][n][3] *= corr[1];
+            }
+            // O += P V
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t pa[4];
+                pa[0] = pack2(s[2 * ks][0], s[2 * ks][1]);
+                pa[1] = pack2(s[2 * ks][2], s[2 * ks][3]);
+                pa[2] = pack2(s[2 * ks + 1][0], s[2 * ks + 1][1]);
+                pa[3] = pack2(s[2 * ks + 1][2], s[2 * ks + 1][3]);
+                const int vrow = ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                for (int n2 = 0; n2 < NT / 2; ++n2) {
+                    uint32_t bfr[4];
+                    ldmatrix_x4_trans(vbase + S::off(vrow, 2 * n2 + (lane >> 4)), bfr);
+                    mma_bf16_16816(acc[j][2 * n2], pa, bfr[0], bfr[1]);
+                    mma_bf16_16816(acc[j][2 * n2 + 1], pa, bfr[2], bfr[3]);
+                }
+            }
+        }
+        __syncthreads();   // everyone is done with this stage before it is refilled
+    }
+
+    // ---- context vector = mean of V_g over the present keys
+    s_vpart[vs_k0][2 * vs_dp] = vsum0;
+    s_vpart[vs_k0][2 * vs_dp + 1] = vsum1;
+    __syncthreads();
+    if (threadIdx.x < D) {
+        float t = 0.f;
+        for (int i = 0; i < VS_STRIDE; ++i) t += s_vpart[i][threadIdx.x];
+        s_mean[threadIdx.x] = __float2bfloat16_rn(t / (float)Tv);
+    }
+    // ---- active rows: normalise and store
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        if (tile_head[j] < 0) continue;
+        const int hh = tile_head[j];
+        __nv_bfloat16* Oh = O + ((size_t)b * k_h + khs[hh]) * Tlen * D;
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+            float l = l_run[j][h2];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int a = tile_row0[j] + gq + h2 * 8;
+            const int t = a < kMaxActive ? s_act[hh][a] : -1;
+            if (t < 0) continue;
+            const float inv = 1.0f / l;
+            uint32_t* orow = reinterpret_cast<uint32_t*>(Oh + (size_t)t * D);
+#pragma unroll
+            for (int n = 0; n < NT; ++n)
+                orow[n * 4 + tq] = pack2(acc[j][n][2 * h2] * inv, acc[j][n][2 * h2 + 1] * inv);
+        }
+    }
+    __syncthreads();
+    // ---- context rows and zero rows, 16 bytes per store
+    const uint4* mean4 = reinterpret_cast<const uint4*>(s_mean);
+    for (int hh = 0; hh < rk; ++hh) {
+        uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D);
+        const uint32_t* bits = s_abits + hh * words;
+        for (int i = threadIdx.x; i < Tlen * S::CPR; i += blockDim.x) {
+            const int t = i / S::CPR, cc = i % S::CPR;
+            if ((bits[t >> 5] >> (t & 31)) & 1u) continue;
+            dst[i] = s_kind[t] ? mean4[cc] : make_uint4(0, 0, 0, 0);
+        }
+    }
+}
+
+template <int D>
+int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
+    const sentry_attend_desc& d = a.d;
+    const size_t valid_bytes = (((size_t)d.T * 2 + 127) / 128) * 128;
+    if (!a.selection_given) {
+        // K segment: as many rows as fit in ~64 KB (one pass for T <= 1024 at d = 32)
+        int seg_rows = (64 * 1024) / (D * 2);
+        if (seg_rows > d.T) seg_rows = (d.T + 7) / 8 * 8;
+        const size_t smem = valid_bytes + (size_t)seg_rows * D * 2;
+        auto kern = attend_score_bf16_kernel<D>;
+        SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        dim3 grid((d.T + kScoreThreads - 1) / kScoreThreads, d.B * d.Hk);
+        LaunchScope ls(ctx, KS_ATT_SCORE, st);
+        kern<<<grid, kScoreThreads, smem, st>>>((const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K,
+                                                 a.kept_heads, a.ids, a.masks, a.sample_table,
+                                                 a.sample_offsets, a.n_subsets, d.T, d.Hq, d.Hk, d.k_h,
+                                                 d.c, d.score_mode, seg_rows, a.mscore, a.status);
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    {
+        const int words = (d.T + 31) / 32;
+        size_t smem = valid_bytes + (((size_t)d.T + 127) / 128) * 128 +
+                      (((size_t)kMaxRK * words * 4 + 127) / 128) * 128;
+        size_t uni = CoreSmem<D>::PIPE_BYTES;
+        if (!a.selection_given && (size_t)kMaxRK * d.T * 4 > uni) uni = (size_t)kMaxRK * d.T * 4;
+        smem += uni;
+        auto kern = attend_core_bf16_kernel<D>;
+        SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        LaunchScope ls(ctx, KS_ATT_CORE, st);
+        kern<<<d.B * d.Hk, kCoreThreads, smem, st>>>(
+            (const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, a.kept_heads,
+            a.ids, a.masks, a.mscore, a.selection_given ? a.active : nullptr,
+            a.selection_given ? nullptr : a.active_out_user, d.T, d.Hq, d.Hk, d.k_h, d.c, a.U_max,
+            (__nv_bfloat16*)a.O, a.status);
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}
+
+}  // namespace
+
+// bf16, at most 4 query heads per KV group, U <= 48 and shared memory within reach.
+bool attend_bf16_supported(const sentry_attend_desc& d) {
+    if (d.dtype != SENTRY_BF16) return false;
+    if (d.Hq / d.Hk > kMaxRK) return false;
+    if (sentry_num_active(d.T, d.c) > kMaxActive) return false;
+    if (d.T > 8192) return false;
+    return d.d == 16 || d.d == 32 || d.d == 64;
+}
+
+int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
+    switch (a.d.d) {
+        case 16: return launch_d<16>(ctx, a, st);
+        case 32: return launch_d<32>(ctx, a, st);
+        case 64: return launch_d<64>(ctx, a, st);
+        default: return SENTRY_ERR_UNSUPPORTED;
+    }
+}

@@ -228,12 +228,15 @@ struct AttendArgs {
     int n_subsets;
     void* O;
     int32_t* active;        // [B,k_h,U_max] written by selection or given by the caller
+    int32_t* active_out_user;  // the caller's active_out (may be null)
     bool selection_given;   // true: `active` is the caller's forced selection
     float* mscore;          // workspace [B,k_h,T]
     int U_max;
     unsigned int* status;
 };
 int launch_attend_generic(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
+bool attend_bf16_supported(const sentry_attend_desc& d);
+int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 
 struct FfnArgs {
     sentry_ffn_desc d;
