@@ -183,29 +183,23 @@ def cpu_sample_inputs(w: synth.Workload, n_max: int):
 
 
 def time_oracle(w: synth.Workload, budget_s: float):
-    """Time the oracle on a bounded sample (~budget_s of CPU work).  Returns
+    """Time the oracle, as it stands, on a bounded sample: whole passes over up to 3 x cores
+    samples of the workload until about budget_s seconds of wall time have gone.  Returns
     (tokens/s, cores, description)."""
     import oracle
     cores = oracle.threads()
     inp = cpu_sample_inputs(w, 3 * cores)
-    n_avail = inp.w.B
+    sel = np.arange(inp.w.B)
+    oracle_sample_run(inp, sel[:1], None, None)  # builds/loads the library outside the timing
+    reps, tok = 0, 0
     t0 = time.perf_counter()
-    tok = oracle_sample_run(inp, np.arange(min(cores, n_avail)), None, None)
-    t_probe = time.perf_counter() - t0
-    n = min(cores, n_avail)
-    reps = 1
-    if t_probe < budget_s / 2 and n_avail > n:
-        n = int(min(n_avail, max(n, n * (budget_s / max(t_probe, 1e-3)) // 1)))
-    sel = np.arange(n)
-    t0 = time.perf_counter()
-    tok = oracle_sample_run(inp, sel, None, None)
-    dt = time.perf_counter() - t0
-    while dt * (reps + 1) < budget_s and reps < 50 and dt < 1.0:
+    dt = 0.0
+    while reps == 0 or (dt < budget_s and reps < 1000):
         tok += oracle_sample_run(inp, sel, None, None)
         reps += 1
         dt = time.perf_counter() - t0
-    return tok / dt, cores, "%d samples x %d passes of %s (gate+attend+ffn, float64, OpenMP over samples)" % (
-        n, reps, w.name)
+    return tok / dt, cores, "%d samples x %d passes of %s in %.1f s (gate+attend+ffn, float64, OpenMP over samples)" % (
+        len(sel), reps, w.name, dt)
 
 
 def run_reference(args, w: synth.Workload):
