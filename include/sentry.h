@@ -113,6 +113,40 @@ SENTRY_API int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, i
                        uint32_t* kv_groups, int heads_per_group, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Gate selection for callers that cannot allocate device memory.
+ *
+ * (No counterpart in the paper: this is a deployment convenience, not part of
+ * the method.)  Some hosts of this library may not call cudaMalloc at all --
+ * a plug-in that lives inside another runtime's memory pool, or a service
+ * that pins its device-memory budget at start-up and forbids growth.  They
+ * cannot create a context (sentry_create allocates a status word) nor hand
+ * over a workspace.  This entry point needs neither: the per-score-row
+ * scratch of the selection sits in a fixed array inside the library image,
+ * SENTRY_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the
+ * process exits.  It calls no cudaMalloc/cudaFree and no allocating routine.
+ *
+ * Arguments and results are those of sentry_gate_select, with `device` in
+ * place of the context, plus
+ *   status  device pointer to one u32 or NULL: SENTRY_STATUS_BIT_* flags are
+ *           OR-ed into it (the caller clears it).  With NULL the flags go to an
+ *           internal word that nothing reads.
+ * Limits: n_units <= 12288, and 256 + roundup256(S*k*4) + S*4 <=
+ * SENTRY_STATIC_SCRATCH_BYTES, else SENTRY_ERR_UNSUPPORTED / SENTRY_ERR_WORKSPACE
+ * before anything is enqueued.
+ * The first call on a device looks up the array's device address (one runtime
+ * query, cached); make that first call before any stream capture begins.
+ * All calls on a device share the one array and it keeps the previous call's
+ * contents (the library clears the word that must start at zero): calls whose
+ * kernels could overlap on the GPU -- different streams without an ordering
+ * between them -- race.  Order them on one stream or with events.
+ */
+#define SENTRY_STATIC_SCRATCH_BYTES (256 * 1024)
+SENTRY_API int sentry_gate_select_static(int device, const float* scores, int S, int n_units,
+                              const uint32_t* masks, int n_masks, int k, int32_t* kept,
+                              uint32_t* kv_groups, int heads_per_group, uint32_t* status,
+                              void* stream);
+
+/* ---------------------------------------------------------------------------
  * SentryAttend forward (Sec. 4.4, Eq. 6) on the kept heads of every sample.
  *
  * Per sample b, with present tokens = { t : bit ids[t] of masks[b] is set }

@@ -26,7 +26,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_num_active_queries", "sentry_workspace_bytes", "sentry_set_workspace",
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
-           "sentry_kernel_name"]
+           "sentry_kernel_name", "sentry_gate_select_static"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -69,6 +69,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_workspace_bytes.restype = ctypes.c_size_t
     lib.sentry_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
     lib.sentry_gate_select.argtypes = [vp, vp, ci, ci, vp, ci, ci, vp, vp, ci, vp]
+    lib.sentry_gate_select_static.argtypes = [ci, vp, ci, ci, vp, ci, ci, vp, vp, ci, vp, vp]
     lib.sentry_attend_fwd.argtypes = [vp, ctypes.POINTER(AttendDesc), vp, vp, vp, vp, vp, vp, vp,
                                       vp, ci, vp, vp, vp, vp]
     lib.sentry_ffn_fwd.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -119,6 +120,21 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def gate_select_static(scores: torch.Tensor, masks: torch.Tensor, k: int, kept: torch.Tensor,
+                       kv_groups: Optional[torch.Tensor] = None, heads_per_group: int = 0,
+                       status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """sentry_gate_select_static: the gate selection for callers that may not allocate device
+    memory.  No context, no workspace; every tensor (outputs included) comes from the caller,
+    and this wrapper allocates nothing either.  Returns `kept`."""
+    S, n = scores.shape
+    rc = load_library().sentry_gate_select_static(
+        scores.device.index or 0, _ptr(scores), S, n, _ptr(masks), masks.shape[0], int(k),
+        _ptr(kept), _ptr(kv_groups), int(heads_per_group), _ptr(status), _stream())
+    if rc != 0:
+        raise SentryError(rc, "sentry_gate_select_static")
+    return kept
 
 
 class Sentry:

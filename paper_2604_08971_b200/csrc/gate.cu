@@ -86,3 +86,102 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
     SENTRY_CUDA_TRY(cudaGetLastError());
     return SENTRY_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free variant of the gate selection.
+//
+// Its scratch (the per-score-row result that the fan-out kernel reads, the per-row KV-group
+// bitmaps and a status word) lives in one file-scope device array instead of a workspace, so
+// a caller that is not allowed to call cudaMalloc -- code running inside another runtime's
+// memory pool, or an embedding that fixes its device-memory budget at start-up -- can still
+// run the selection.  The array is part of the library image: every GPU that loads the
+// library holds these 256 KB until the process exits.
+//
+// In host code `g_gate_scratch` is only a handle for the symbol, not a device address;
+// the address a kernel can use comes from cudaGetSymbolAddress, asked once per device with
+// that device current (static_scratch_of below).
+#include <mutex>
+
+namespace {
+
+static __device__ __align__(256) unsigned char g_gate_scratch[SENTRY_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kStaticHeader = 256;  // status word, padded so the tables stay 256-byte aligned
+
+struct StaticDevice {
+    unsigned char* scratch = nullptr;  // device address of g_gate_scratch on this device
+    int sm_count = 0;
+};
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mu;
+
+// Device address of the scratch array on `device` (which must be current).  The first call per
+// device asks the runtime for it; later calls only read the cached value.
+int static_scratch_of(int device, StaticDevice* out) {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    StaticDevice& sd = g_static_dev[device];
+    if (sd.scratch == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_gate_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return SENTRY_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1)
+            return SENTRY_ERR_CUDA;
+        sd.sm_count = sms;
+        sd.scratch = static_cast<unsigned char*>(p);
+    }
+    *out = sd;
+    return SENTRY_OK;
+}
+
+}  // namespace
+
+extern "C" int sentry_gate_select_static(int device, const float* scores, int S, int n_units,
+                                         const uint32_t* masks, int n_masks, int k, int32_t* kept,
+                                         uint32_t* kv_groups, int heads_per_group,
+                                         uint32_t* status, void* stream) {
+    if (scores == nullptr || masks == nullptr || kept == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (((uintptr_t)scores | (uintptr_t)masks | (uintptr_t)kept | (uintptr_t)kv_groups |
+         (uintptr_t)status) % 4 != 0)
+        return SENTRY_ERR_INVALID_ARG;
+    if (device < 0 || device >= kMaxDevices) return SENTRY_ERR_INVALID_ARG;
+    if (S < 1 || n_units < 1 || n_masks < 0 || k < 1 || k > n_units) return SENTRY_ERR_BAD_SHAPE;
+    if (kv_groups != nullptr) {
+        if (heads_per_group < 1) return SENTRY_ERR_INVALID_ARG;
+        if ((n_units + heads_per_group - 1) / heads_per_group > 32) return SENTRY_ERR_BAD_SHAPE;
+    }
+    // the sort keys of one score row must fit the default shared-memory window
+    if ((size_t)n_units * sizeof(uint32_t) > 48 * 1024) return SENTRY_ERR_UNSUPPORTED;
+    // rows [S,k] i32 and groups [S] u32 must fit the static array
+    const size_t rows_bytes = align_up((size_t)S * k * sizeof(int32_t), 256);
+    const size_t groups_bytes = (size_t)S * sizeof(uint32_t);
+    if (kStaticHeader + rows_bytes + groups_bytes > (size_t)SENTRY_STATIC_SCRATCH_BYTES)
+        return SENTRY_ERR_WORKSPACE;
+    if (n_masks == 0) return SENTRY_OK;
+
+    SENTRY_CUDA_TRY(cudaSetDevice(device));
+    StaticDevice sd;
+    int rc = static_scratch_of(device, &sd);
+    if (rc != SENTRY_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned int* own_status = reinterpret_cast<unsigned int*>(sd.scratch);
+    int32_t* rows = reinterpret_cast<int32_t*>(sd.scratch + kStaticHeader);
+    uint32_t* groups = reinterpret_cast<uint32_t*>(sd.scratch + kStaticHeader + rows_bytes);
+    // The array keeps whatever the previous call left.  rows/groups are rewritten in full for
+    // all S score rows before the fan-out reads them; only the status word must start at zero.
+    SENTRY_CUDA_TRY(cudaMemsetAsync(own_status, 0, sizeof(unsigned int), st));
+    gate_rows_kernel<<<S, kGateThreads, (size_t)n_units * sizeof(uint32_t), st>>>(
+        scores, n_units, k, rows, kv_groups ? groups : nullptr, heads_per_group > 0 ? heads_per_group : 1);
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    const size_t total = (size_t)n_masks * k;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > sd.sm_count * 8) blocks = sd.sm_count * 8;
+    if (blocks < 1) blocks = 1;
+    gate_expand_kernel<<<blocks, 256, 0, st>>>(rows, groups, masks, S, n_masks, k, kept, kv_groups,
+                                               status != nullptr ? status : own_status);
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}
