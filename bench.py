@@ -67,7 +67,7 @@ def work_model(w: synth.Workload, masks: np.ndarray, kept_heads: np.ndarray, num
             "att_bytes": float(att_bytes),
             "kernel_bytes": {"attend_score": b_score, "attend_core": b_core,
                              "ffn_main": b_ffn_rows + b_weights,
-                             "ffn_prepack": 2 * b_weights,
+                             "ffn_prepare": 2 * b_weights,
                              "gate_expand": 4.0 * (n_masks * w.k_h + n_lists * w.k_c)},
             "kernel_flops": {"ffn_main": ffn_flops}}
 

@@ -13,7 +13,7 @@
 // Kernel slots for launch accounting and optional per-kernel timing.
 enum KernelSlot {
     KS_GATE_ROWS = 0, KS_GATE_EXPAND, KS_ATT_SCORE, KS_ATT_SELECT, KS_ATT_CORE,
-    KS_FFN_PLAN_ROWS, KS_FFN_PLAN_TILES, KS_FFN_PREPACK, KS_FFN_MAIN, KS_COUNT
+    KS_FFN_PLAN, KS_FFN_PREPARE, KS_FFN_MAIN, KS_COUNT
 };
 
 struct ProfRec { cudaEvent_t start, stop; int slot; };

@@ -10,7 +10,7 @@
 int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,
                   int kc_pad, int max_tiles, cudaStream_t st);  // ffn_tc.cu
 bool ffn_tc_supported(const sentry_ffn_desc& d);
-int ffn_tc_kc_pad(int k_c);
+int ffn_tc_kc_pad(int D, int k_c);
 
 namespace {
 
@@ -18,47 +18,42 @@ constexpr int kGenericTileRows = 16;
 constexpr int kGenericThreads = 256;
 constexpr int kTcTileRows = 128;
 
-// grid B.  Present-token list and count of each sample; zero rows of Y for absent tokens.
-__global__ void __launch_bounds__(256)
-ffn_plan_rows_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks, int T,
-                     int row_bytes, uint16_t* __restrict__ vlist, int32_t* __restrict__ tv,
-                     uint8_t* __restrict__ Y, unsigned int* status) {
-    __shared__ int red[66];
-    const int b = blockIdx.x;
-    const uint32_t mask = (ids != nullptr) ? masks[b] : 0xffffffffu;
-    uint16_t* vl = vlist + (size_t)b * T;
-    const int Tv = block_build_valid(ids, T, mask, vl, red);
-    if (threadIdx.x == 0) {
-        tv[b] = Tv;
-        if (Tv == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
-    }
-    if (ids == nullptr || Tv == T) return;
-    // zero the absent rows: 16-byte stores, one row after the other
-    const int vec_per_row = row_bytes / 16;
-    for (int t = 0; t < T; ++t) {
-        const int m = ids[t];
-        const bool present = (m >= 0 && m < 32) && ((mask >> m) & 1u);
-        if (present) continue;
-        uint4* row = reinterpret_cast<uint4*>(Y + ((size_t)b * T + t) * row_bytes);
-        for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) row[v] = make_uint4(0, 0, 0, 0);
-    }
-}
-
-// one block.  Group samples by list, prefix rows, cut into tiles.
+// One CTA.  Present rows per sample (from the per-modality token counts), then per list a
+// stable scan over its samples: where each sample's rows start in the row table, where
+// each list starts, and how many tiles each list needs.
 __global__ void __launch_bounds__(1024)
-ffn_plan_tiles_kernel(const int32_t* __restrict__ tv, const int32_t* __restrict__ list_of_sample,
-                      int B, int n_lists, int tile_rows, FfnPlan p, unsigned int* status) {
-    __shared__ int s_warp_cnt[32], s_warp_rows[32];
-    __shared__ int s_base_cnt, s_base_rows, s_list_begin;
+ffn_plan_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks,
+                const int32_t* __restrict__ list_of_sample, int B, int T, int n_lists,
+                int tile_rows, FfnPlan p, unsigned int* status) {
+    __shared__ int s_cnt[32];
+    __shared__ int s_warp_rows[32];
+    __shared__ int s_base_rows, s_list_row0;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    if (threadIdx.x == 0) { s_list_begin = 0; p.tile_start[0] = 0; p.list_start[0] = 0; }
+    if (threadIdx.x < 32) s_cnt[threadIdx.x] = 0;
+    if (threadIdx.x == 0) { s_list_row0 = 0; p.tile_start[0] = 0; p.list_row0[0] = 0; }
     __syncthreads();
+    if (ids != nullptr) {
+        for (int t = threadIdx.x; t < T; t += blockDim.x) {
+            const int m = ids[t];
+            if (m >= 0 && m < 32) atomicAdd(&s_cnt[m], 1);
+            else atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+        }
+        __syncthreads();
+    }
+    auto present_rows = [&](int b) {
+        if (ids == nullptr) return T;
+        uint32_t mask = masks[b];
+        int n = 0;
+        while (mask) { const int m = __ffs(mask) - 1; n += s_cnt[m]; mask &= mask - 1; }
+        return n;
+    };
     for (int l = 0; l < n_lists; ++l) {
-        if (threadIdx.x == 0) { s_base_cnt = 0; s_base_rows = 0; }
+        if (threadIdx.x == 0) s_base_rows = 0;
         __syncthreads();
         for (int b0 = 0; b0 < B; b0 += blockDim.x) {
             const int b = b0 + threadIdx.x;
-            int mine = 0, rows = 0;
+            int rows = 0;
+            bool mine = false;
             if (b < B) {
                 int lb = list_of_sample ? list_of_sample[b] : 0;
                 if (lb < 0 || lb >= n_lists) {
@@ -66,57 +61,95 @@ ffn_plan_tiles_kernel(const int32_t* __restrict__ tv, const int32_t* __restrict_
                     lb = 0;
                 }
                 mine = (lb == l);
-                rows = mine ? tv[b] : 0;
+                if (mine) {
+                    rows = present_rows(b);
+                    if (rows == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
+                }
             }
-            // inclusive warp scans of (mine, rows)
-            int c = mine, r = rows;
+            int r = rows;  // inclusive warp scan
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const int c2 = __shfl_up_sync(0xffffffffu, c, o);
                 const int r2 = __shfl_up_sync(0xffffffffu, r, o);
-                if (lane >= o) { c += c2; r += r2; }
+                if (lane >= o) r += r2;
             }
-            if (lane == 31) { s_warp_cnt[wid] = c; s_warp_rows[wid] = r; }
+            if (lane == 31) s_warp_rows[wid] = r;
             __syncthreads();
-            int c_before = s_base_cnt, r_before = s_base_rows, c_tot = 0, r_tot = 0;
+            int before = s_base_rows, tot = 0;
             for (int w = 0; w < nw; ++w) {
-                if (w < wid) { c_before += s_warp_cnt[w]; r_before += s_warp_rows[w]; }
-                c_tot += s_warp_cnt[w]; r_tot += s_warp_rows[w];
+                if (w < wid) before += s_warp_rows[w];
+                tot += s_warp_rows[w];
             }
-            if (mine) {
-                const int pos = s_list_begin + c_before + c - 1;
-                p.order[pos] = b;
-                p.row_prefix[pos] = r_before + r - rows;
-            }
+            if (mine) p.sample_row0[b] = s_list_row0 + before + r - rows;
             __syncthreads();
-            if (threadIdx.x == 0) { s_base_cnt += c_tot; s_base_rows += r_tot; }
+            if (threadIdx.x == 0) s_base_rows += tot;
             __syncthreads();
         }
         if (threadIdx.x == 0) {
-            p.list_rows[l] = s_base_rows;
-            s_list_begin += s_base_cnt;
-            p.list_start[l + 1] = s_list_begin;
+            s_list_row0 += s_base_rows;
+            p.list_row0[l + 1] = s_list_row0;
             p.tile_start[l + 1] = p.tile_start[l] + (s_base_rows + tile_rows - 1) / tile_rows;
         }
         __syncthreads();
     }
 }
 
-// Weight gather.  layout 0 (plain-ALU kernel): W1g [l][D][kc_pad], W2g [l][kc_pad][D]
-//                 layout 1 (tensor-core kernel, both K-major):
-//                                 W1c [l][kc_pad][D],  W2c [l][D][kc_pad]
-// Columns / rows n >= k_c are zero.  grid (ceil(kc_pad*D/256), n_lists, 2).
+// Blocks [0, B): row table entries of sample b (its present tokens, ascending) and zero rows
+// of Y for its absent tokens.  Blocks [B, B + prepack blocks): the weight gather, which
+// "materialises" the pruned W1', W2' of every kept list.
+//   layout 0 (plain-ALU kernel): W1g [l][D][kc_pad], W2g [l][kc_pad][D]
+//   layout 1 (tensor-core kernel, both K-major): W1c [l][kc_pad][D], W2c [l][D][kc_pad]
+// Columns / rows n >= k_c are zero.
 template <typename T>
 __global__ void __launch_bounds__(256)
-ffn_prepack_kernel(const T* __restrict__ W1, const T* __restrict__ W2,
-                   const int32_t* __restrict__ kept, int D, int F, int k_c, int kc_pad, int layout,
-                   T* __restrict__ out1, T* __restrict__ out2, unsigned int* status) {
-    const int l = blockIdx.y;
+ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks, int B,
+                   int Tlen, FfnPlan p, uint8_t* __restrict__ Y,
+                   const T* __restrict__ W1, const T* __restrict__ W2,
+                   const int32_t* __restrict__ kept, int n_lists, int D, int F, int k_c, int kc_pad,
+                   int layout, T* __restrict__ out1, T* __restrict__ out2, unsigned int* status) {
+    if ((int)blockIdx.x < B) {
+        __shared__ int red[33];
+        const int b = blockIdx.x;
+        const uint32_t mask = (ids != nullptr) ? masks[b] : 0xffffffffu;
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+        int32_t* rows = p.rowidx + p.sample_row0[b];
+        int base = 0;
+        for (int t0 = 0; t0 < Tlen; t0 += blockDim.x) {
+            const int t = t0 + threadIdx.x;
+            bool ok = false;
+            if (t < Tlen) {
+                if (ids == nullptr) ok = true;
+                else { const int m = ids[t]; ok = (m >= 0 && m < 32) && ((mask >> m) & 1u); }
+            }
+            const unsigned bm = __ballot_sync(0xffffffffu, ok);
+            __syncthreads();
+            if (lane == 0) red[wid] = __popc(bm);
+            __syncthreads();
+            int pos = base, tot = 0;
+            for (int w = 0; w < nw; ++w) { if (w < wid) pos += red[w]; tot += red[w]; }
+            if (ok) rows[pos + __popc(bm & ((1u << lane) - 1u))] = b * Tlen + t;
+            base += tot;
+        }
+        if (ids == nullptr || base == Tlen) return;
+        // zero the rows of absent tokens, 16 bytes per store, all threads busy
+        const int vpr = D * (int)sizeof(T) / 16;
+        uint4* Yb = reinterpret_cast<uint4*>(Y + (size_t)b * Tlen * D * sizeof(T));
+        for (int i = threadIdx.x; i < Tlen * vpr; i += blockDim.x) {
+            const int m = ids[i / vpr];
+            const bool present = (m >= 0 && m < 32) && ((mask >> m) & 1u);
+            if (!present) Yb[i] = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
     const size_t per = (size_t)kc_pad * D;
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t blocks_per = (per + 255) / 256;
+    size_t pb = (size_t)blockIdx.x - B;
+    const int which = (int)(pb / (blocks_per * n_lists));
+    pb -= (size_t)which * blocks_per * n_lists;
+    const int l = (int)(pb / blocks_per);
+    const size_t i = (pb % blocks_per) * 256 + threadIdx.x;
     if (i >= per) return;
     const int32_t* N = kept + (size_t)l * k_c;
-    if (blockIdx.z == 0) {
+    if (which == 0) {
         // W1: destination-major index so that writes coalesce
         int n, e;
         if (layout == 0) { e = (int)(i / kc_pad); n = (int)(i % kc_pad); }
@@ -155,10 +188,10 @@ ffn_generic_kernel(const T* __restrict__ X, const T* __restrict__ W1g, const T* 
     float* s_x = s_f;                                  // [16][D]
     float* s_h = s_f + (size_t)kGenericTileRows * D;   // [16][256]
     __shared__ long long s_row[kGenericTileRows];
-    int l, slot0, n_rows;
-    if (!ffn_tile_lookup(plan, n_lists, blockIdx.x, kGenericTileRows, l, slot0, n_rows)) return;
+    int l, row0, n_rows;
+    if (!ffn_tile_lookup(plan, n_lists, blockIdx.x, kGenericTileRows, l, row0, n_rows)) return;
     if (threadIdx.x < kGenericTileRows)
-        s_row[threadIdx.x] = threadIdx.x < n_rows ? ffn_row_of_slot(plan, l, slot0 + threadIdx.x, Tlen) : -1;
+        s_row[threadIdx.x] = threadIdx.x < n_rows ? (long long)plan.rowidx[row0 + threadIdx.x] : -1;
     __syncthreads();
     for (int i = threadIdx.x; i < kGenericTileRows * D; i += blockDim.x) {
         const int r = i / D, e = i % D;
@@ -226,13 +259,10 @@ FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes) {
     WsAlloc a(ws, bytes);
     FfnWs w;
     const size_t esz = d.dtype == SENTRY_F32 ? 4 : 2;
-    w.plan.vlist = a.take<uint16_t>((size_t)d.B * d.T);
-    w.plan.tv = a.take<int32_t>(d.B);
-    w.plan.order = a.take<int32_t>(d.B);
-    w.plan.row_prefix = a.take<int32_t>(d.B);
-    w.plan.list_start = a.take<int32_t>(d.n_lists + 1);
-    w.plan.list_rows = a.take<int32_t>(d.n_lists);
+    w.plan.sample_row0 = a.take<int32_t>(d.B);
+    w.plan.list_row0 = a.take<int32_t>(d.n_lists + 1);
     w.plan.tile_start = a.take<int32_t>(d.n_lists + 1);
+    w.plan.rowidx = a.take<int32_t>((size_t)d.B * d.T);
     w.w1p = a.take<uint8_t>((size_t)d.n_lists * kc_pad * d.D * esz);
     w.w2p = a.take<uint8_t>((size_t)d.n_lists * kc_pad * d.D * esz);
     w.ok = a.ok;
@@ -241,7 +271,7 @@ FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes) {
 }
 
 int kc_pad_for(const sentry_ffn_desc& d) {
-    if (d.dtype == SENTRY_BF16 && ffn_tc_supported(d)) return ffn_tc_kc_pad(d.k_c);
+    if (d.dtype == SENTRY_BF16 && ffn_tc_supported(d)) return ffn_tc_kc_pad(d.D, d.k_c);
     return (d.k_c + 7) / 8 * 8;
 }
 
@@ -257,33 +287,28 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cud
     const int kc_pad = kc_pad_for(d);
     FfnWs w = carve(d, kc_pad, ws, ws_bytes);
     if (!w.ok) return SENTRY_ERR_WORKSPACE;
-    const int esz = d.dtype == SENTRY_F32 ? 4 : 2;
     const int tile_rows = tc ? kTcTileRows : kGenericTileRows;
 
     {
-        LaunchScope ls(ctx, KS_FFN_PLAN_ROWS, st);
-        ffn_plan_rows_kernel<<<d.B, 256, 0, st>>>(a.ids, a.masks, d.T, d.D * esz, w.plan.vlist,
-                                                   w.plan.tv, (uint8_t*)a.Y, a.status);
-    }
-    SENTRY_CUDA_TRY(cudaGetLastError());
-    {
-        LaunchScope ls(ctx, KS_FFN_PLAN_TILES, st);
-        ffn_plan_tiles_kernel<<<1, 1024, 0, st>>>(w.plan.tv, a.list_of_sample, d.B, d.n_lists,
-                                                   tile_rows, w.plan, a.status);
+        LaunchScope ls(ctx, KS_FFN_PLAN, st);
+        ffn_plan_kernel<<<1, 1024, 0, st>>>(a.ids, a.masks, a.list_of_sample, d.B, d.T, d.n_lists,
+                                             tile_rows, w.plan, a.status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
     {
         const size_t per = (size_t)kc_pad * d.D;
-        dim3 grid((unsigned)((per + 255) / 256), d.n_lists, 2);
-        LaunchScope ls(ctx, KS_FFN_PREPACK, st);
+        const size_t grid = (size_t)d.B + 2 * (size_t)d.n_lists * ((per + 255) / 256);
+        LaunchScope ls(ctx, KS_FFN_PREPARE, st);
         if (d.dtype == SENTRY_F32)
-            ffn_prepack_kernel<float><<<grid, 256, 0, st>>>((const float*)a.W1, (const float*)a.W2,
-                                                            a.kept, d.D, d.F, d.k_c, kc_pad, 0,
-                                                            (float*)w.w1p, (float*)w.w2p, a.status);
+            ffn_prepare_kernel<float><<<(unsigned)grid, 256, 0, st>>>(
+                a.ids, a.masks, d.B, d.T, w.plan, (uint8_t*)a.Y, (const float*)a.W1,
+                (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, (float*)w.w1p,
+                (float*)w.w2p, a.status);
         else
-            ffn_prepack_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
-                (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.D, d.F, d.k_c,
-                kc_pad, tc ? 1 : 0, (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
+            ffn_prepare_kernel<__nv_bfloat16><<<(unsigned)grid, 256, 0, st>>>(
+                a.ids, a.masks, d.B, d.T, w.plan, (uint8_t*)a.Y, (const __nv_bfloat16*)a.W1,
+                (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, tc ? 1 : 0,
+                (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
     const long long rows = (long long)d.B * d.T;

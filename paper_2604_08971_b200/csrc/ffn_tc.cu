@@ -1,18 +1,28 @@
 // Channel-compacted FFN on the 5th-generation tensor cores (Section 4.6):
 //   Y = gelu(X . W1[:, N]) . W2[N, :]   for the present rows of every sample.
 //
-// One persistent CTA per SM walks tiles of 128 present rows (row plan in ffn_plan.cuh).
-// Per tile and per chunk of 128 kept channels:
-//   GEMM1  H[128 x 128] = X_tile[128 x D] . W1c_chunk^T          (tcgen05, fp32 in TMEM)
+// One persistent CTA per SM walks tiles of 128 present rows (row table in ffn_plan.cuh).
+// Per tile and per chunk of CH kept channels (CH = 256, or 128 when d_model = 384):
+//   GEMM1  H[128 x CH] = X_tile[128 x D] . W1c_chunk^T            (tcgen05, fp32 in TMEM)
 //   epilogue  H -> gelu -> bf16 -> shared memory (K-major, 128-byte swizzle)
-//   GEMM2  Y[128 x D] += H[128 x 128] . W2c_chunk                 (tcgen05, fp32 in TMEM)
+//   GEMM2  Y[128 x D] += H[128 x CH] . W2c_chunk                  (tcgen05, fp32 in TMEM)
 // The hidden activations never leave the SM.  Weights are the gathered, K-major copies made
-// by the prepack kernel; 128 x 64 tiles of them stream through a TMA ring.  X rows are
-// gathered with 16-byte async copies into the same swizzled layout TMA would produce.
+// by the prepare kernel and stream through a ring of 32 KB TMA stages; every stage feeds
+// 512 tensor-pipe cycles (four N=256 or eight N=128 instructions), which is what it takes to
+// hide the fixed cost of a stage hand-over (an mbarrier wait, the copy issue, a commit) behind
+// the arithmetic.  Two producer threads share the ring for the same reason.  X rows are
+// gathered with 16-byte async copies, one 64-column block at a time, into the swizzled layout
+// TMA would produce; a block's slot is refilled for the next tile as soon as the last chunk's
+// GEMM1 has read it.
 //
-// Warp roles (384 threads): warp 0 = weight TMA producer and TMEM owner, warp 1 = UMMA
-// issuer, warps 2-3 = X row gather, warps 4-11 = epilogue (two warps per TMEM lane quarter).
-// Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT and unwinds.
+// The tensor pipe is kept busy across chunk and tile boundaries: the issuer runs GEMM1 of the
+// next chunk (or of the next tile's first chunk) before GEMM2 of the current one, so GEMM2
+// never waits for the GELU epilogue with nothing else queued.
+//
+// Warp roles (480 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
+// warp 1 = UMMA issuer, warps 3-6 = X row gather, warps 7-14 = epilogue (two warps per TMEM
+// lane quarter).  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
+// and unwinds.
 #include <cuda.h>
 #include <math.h>
 
@@ -23,41 +33,54 @@
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kChunk = 128;            // kept channels per chunk
-constexpr int kStageBytes = 128 * 128; // one 128-row x 64-element bf16 weight tile
-constexpr int kHBytes = 128 * 128 * 2; // hidden chunk, bf16
-constexpr int kThreads = 384;
-constexpr int kEpiThreads = 256;
-constexpr int kLoaderThreads = 64;
+constexpr int kBlockBytes = 128 * 128;   // 128 rows x 64 bf16: one X block, one hidden block
+constexpr int kStageBytes = 2 * kBlockBytes;
+constexpr int kStages = 3;
+constexpr int kThreads = 480;
+constexpr int kLoaderWarp0 = 3, kLoaderWarps = 4, kLoaderThreads = kLoaderWarps * 32;
+constexpr int kEpiWarp0 = 7, kEpiWarps = 8;
 constexpr int kTmemCols = 512;
 
 template <int D>
 struct Cfg {
-    static constexpr int KB1 = D / 64;               // K blocks of GEMM1
-    static constexpr int NB2 = D / 128;              // N blocks of GEMM2
-    static constexpr int NHBUF = (D <= 256) ? 2 : 1; // hidden-chunk buffers (TMEM and smem)
-    static constexpr int NSTAGES = (D == 128) ? 6 : 5;
-    static constexpr int X_BYTES = kTileRows * D * 2;
-    static constexpr int H_COL0 = (D <= 256) ? 256 : 384;  // TMEM column of hidden buffer 0
-    static constexpr int OFF_H = X_BYTES;
-    static constexpr int OFF_W = OFF_H + NHBUF * kHBytes;
-    static constexpr int OFF_MISC = OFF_W + NSTAGES * kStageBytes;
+    static constexpr int CH = (D == 384) ? 128 : 256;  // kept channels per chunk
+    static constexpr int KB1 = D / 64;                 // X blocks per tile = K blocks of GEMM1
+    static constexpr int H_COL0 = (D == 384) ? 384 : 256;  // TMEM column of the hidden accumulator
+    static constexpr int NXS = (D == 128) ? 4 : KB1;   // X block slots (D = 128: two tiles' worth)
+    static constexpr int NHS = CH / 64;                // hidden blocks per chunk (64 channels each)
+    static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
+    static constexpr int OFF_H = NXS * kBlockBytes;
+    static constexpr int OFF_W = OFF_H + NHS * kBlockBytes;
+    static constexpr int OFF_MISC = OFF_W + kStages * kStageBytes;
     static constexpr int SMEM_BYTES = OFF_MISC + 2048 + 1024;  // + misc + alignment slack
+    static_assert(SMEM_BYTES <= 232448, "shared memory over the per-CTA limit");
 };
 
 struct Misc {
-    uint64_t w_full[8], w_empty[8];
-    uint64_t x_full, x_empty;
-    uint64_t h_full[2], h_tmem_empty[2], hs_full[2], hs_empty[2];
+    uint64_t w_full[kStages], w_empty[kStages];
+    uint64_t x_full[8], x_empty[8];
+    uint64_t h_full, h_tmem_empty;
+    uint64_t hs_full[4], hs_empty[4];
     uint64_t y_full, y_empty;
     uint32_t tmem_base;
     int abort_flag;
-    int32_t row[2][kTileRows];
 };
 static_assert(sizeof(Misc) <= 2048, "misc block too large");
 
-__device__ __forceinline__ float gelu_erf(float z) {
-    return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f));
+// gelu(z) = z/2 (1 + erf(z / sqrt 2)) = relu(z) - |z|/2 * erfc(|z| / sqrt 2).
+// erfc(x) = 2^(-q(x)), q = -log2(erfc): q(|z|/sqrt 2) is fitted by |z| times a quartic in |z|
+// (weighted least squares pushed towards minimax on |z| <= 4 sqrt 2, where erfc is below 2e-8;
+// beyond, |z| is clamped).  Largest error of gelu over all z: 7e-7, far below the resolution
+// of the bf16 value that is stored.  One special-function operation per element.
+__device__ __forceinline__ float gelu_erf_fast(float z) {
+    const float a = fminf(fabsf(z), 5.65685424949f);
+    float p = fmaf(4.880980979e-04f, a, -7.198737003e-03f);   // c4/4sqrt2, c3/4
+    p = fmaf(p, a, 5.214667618e-02f);                         // c2 / 2 sqrt 2
+    p = fmaf(p, a, 4.595957994e-01f);                         // c1 / 2
+    p = fmaf(p, a, 1.151000593e+00f);                         // c0 / sqrt 2
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(-(p * a)));
+    return fmaf(-0.5f * fabsf(z), y, fmaxf(z, 0.0f));
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
@@ -65,39 +88,69 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ void cp_async_wait_pending(int n) {
+    if (n <= 0) ptx::cp_async_wait_group<0>();
+    else if (n == 1) ptx::cp_async_wait_group<1>();
+    else ptx::cp_async_wait_group<2>();
+}
+
+// Bounded wait by every lane of a warp; the result is the same in all lanes.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    const bool ok = ptx::mbar_wait(ptx::smem_u32(bar), parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
+}
+// One arrival for the whole warp, after every lane has reached this point.
+__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(bar));
+}
+
+// Four K=16 steps over one 64-wide K block: D (+)= A[128 x 64] . B[N x 64]^T
+__device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr,
+                                           uint32_t idesc, bool overwrite) {
+    const uint64_t ad = ptx::umma_smem_desc_sw128(a_addr);
+    const uint64_t bd = ptx::umma_smem_desc_sw128(b_addr);
+#pragma unroll
+    for (uint32_t ks = 0; ks < 4; ++ks)
+        ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
-              const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, FfnPlan plan,
-              int n_lists, int Tlen, int kc_pad, unsigned int* status) {
+ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2_256,
+              const __grid_constant__ CUtensorMap tm_w2_128, const __nv_bfloat16* __restrict__ X,
+              __nv_bfloat16* __restrict__ Y, FfnPlan plan, int n_lists, int kc_pad,
+              unsigned int* status) {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_u32(smem_raw);
-    const uint32_t base = (raw_addr + 1023u) & ~1023u;   // 1024-byte aligned tile base
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;   // 1024-byte aligned operand blocks
     uint8_t* smem = smem_raw + (base - raw_addr);
     Misc* misc = reinterpret_cast<Misc*>(smem + C::OFF_MISC);
     const uint32_t xs = base, hs = base + C::OFF_H, wsm = base + C::OFF_W;
     volatile int* abort_flag = &misc->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int NC = kc_pad / kChunk;
+    const int NC = kc_pad / C::CH;
     const int total_tiles = plan.tile_start[n_lists];
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::NSTAGES; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(ptx::smem_u32(&misc->w_full[s]), 1);
             ptx::mbar_init(ptx::smem_u32(&misc->w_empty[s]), 1);
         }
-        ptx::mbar_init(ptx::smem_u32(&misc->x_full), kLoaderThreads);
-        ptx::mbar_init(ptx::smem_u32(&misc->x_empty), 1);
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(ptx::smem_u32(&misc->h_full[b]), 1);
-            ptx::mbar_init(ptx::smem_u32(&misc->h_tmem_empty[b]), kEpiThreads);
-            ptx::mbar_init(ptx::smem_u32(&misc->hs_full[b]), kEpiThreads);
+        for (int s = 0; s < 8; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&misc->x_full[s]), kLoaderWarps);
+            ptx::mbar_init(ptx::smem_u32(&misc->x_empty[s]), 1);
+        }
+        ptx::mbar_init(ptx::smem_u32(&misc->h_full), 1);
+        ptx::mbar_init(ptx::smem_u32(&misc->h_tmem_empty), kEpiWarps);
+        for (int b = 0; b < 4; ++b) {
+            ptx::mbar_init(ptx::smem_u32(&misc->hs_full[b]), 4);   // one warp per TMEM lane quarter
             ptx::mbar_init(ptx::smem_u32(&misc->hs_empty[b]), 1);
         }
         ptx::mbar_init(ptx::smem_u32(&misc->y_full), 1);
-        ptx::mbar_init(ptx::smem_u32(&misc->y_empty), kEpiThreads);
+        ptx::mbar_init(ptx::smem_u32(&misc->y_empty), kEpiWarps);
         misc->abort_flag = 0;
         ptx::fence_barrier_init();
     }
@@ -110,166 +163,234 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
     ptx::tc_fence_after_sync();
     const uint32_t tmem = misc->tmem_base;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ weight TMA producer
+    if (warp == 0 || warp == 2) {
+        // ----------------------------------------------------------- weight TMA producers
+        // Both walk the issuer's stage sequence (GEMM1 stages of chunk g, then GEMM2 stages of
+        // chunk g-1); producer p loads the stages with index n = p (mod 2).
         if (lane == 0) {
+            const uint32_t me = (warp == 0) ? 0u : 1u;
             ptx::prefetch_tensormap(&tm_w1);
-            ptx::prefetch_tensormap(&tm_w2);
+            ptx::prefetch_tensormap(&tm_w2_256);
+            ptx::prefetch_tensormap(&tm_w2_128);
             uint32_t n = 0;
             bool ok = true;
-            auto issue = [&](const CUtensorMap* tm, int x, int y) {
-                const uint32_t s = n % C::NSTAGES, use = n / C::NSTAGES;
+            // one stage = one 32 KB box, or two 16 KB boxes (x1 < 0: single box)
+            auto stage = [&](const CUtensorMap* tm, int x0, int x1, int y) {
+                const uint32_t idx = n++;
+                if (!ok || (idx & 1u) != me) return;
+                const uint32_t s = idx % kStages, use = idx / kStages;
                 if (!ptx::mbar_wait(ptx::smem_u32(&misc->w_empty[s]), (use & 1u) ^ 1u, abort_flag)) {
                     ok = false;
                     return;
                 }
                 const uint32_t bar = ptx::smem_u32(&misc->w_full[s]);
                 ptx::mbar_arrive_expect_tx(bar, kStageBytes);
-                ptx::tma_load_2d(wsm + s * kStageBytes, tm, x, y, bar);
-                ++n;
+                ptx::tma_load_2d(wsm + s * kStageBytes, tm, x0, y, bar);
+                if (x1 >= 0) ptx::tma_load_2d(wsm + s * kStageBytes + kBlockBytes, tm, x1, y, bar);
             };
+            auto gemm1_stages = [&](int l, int c) {
+                const int y = l * kc_pad + c * C::CH;
+                if constexpr (D == 384) {
+                    for (int kp = 0; kp < 3; ++kp) stage(&tm_w1, 128 * kp, 128 * kp + 64, y);
+                } else {
+                    for (int kb = 0; kb < C::KB1; ++kb) stage(&tm_w1, 64 * kb, -1, y);
+                }
+            };
+            auto gemm2_stages = [&](int l, int c) {
+                const int x = c * C::CH;
+                if constexpr (D == 256) {
+                    for (int kb2 = 0; kb2 < 4; ++kb2) stage(&tm_w2_256, x + 64 * kb2, -1, l * D);
+                } else if constexpr (D == 128) {
+                    for (int kp = 0; kp < 2; ++kp) stage(&tm_w2_128, x + 128 * kp, x + 128 * kp + 64, l * D);
+                } else {
+                    stage(&tm_w2_256, x, -1, l * D);
+                    stage(&tm_w2_256, x + 64, -1, l * D);
+                    stage(&tm_w2_128, x, x + 64, l * D + 256);
+                }
+            };
+            int prev_l = -1, prev_c = 0;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                int l, slot0, n_rows;
-                ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, slot0, n_rows);
-                for (int c = 0; c <= NC && ok; ++c) {
-                    if (c < NC)
-                        for (int kb = 0; kb < C::KB1 && ok; ++kb)
-                            issue(&tm_w1, kb * 64, l * kc_pad + c * kChunk);
-                    if (c > 0)
-                        for (int nb = 0; nb < C::NB2 && ok; ++nb)
-                            for (int kb2 = 0; kb2 < 2 && ok; ++kb2)
-                                issue(&tm_w2, (c - 1) * kChunk + kb2 * 64, l * D + nb * 128);
+                int l, row0, n_rows;
+                ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
+                for (int c = 0; c < NC && ok; ++c) {
+                    gemm1_stages(l, c);
+                    if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
+                    prev_l = l;
+                    prev_c = c;
                 }
             }
+            if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------- UMMA issuer
         if (lane == 0) {
-            const uint32_t idesc = ptx::umma_idesc_bf16(128, 128);
-            uint32_t n = 0, hc = 0, ti = 0;
+            constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
+            constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
+            const uint32_t tm_h = tmem + C::H_COL0;
+            uint32_t n = 0;   // weight stages consumed
             bool ok = true;
             auto wait = [&](uint64_t* bar, uint32_t parity) {
                 if (ok && !ptx::mbar_wait(ptx::smem_u32(bar), parity, abort_flag)) ok = false;
-                ptx::tc_fence_after_sync();
                 return ok;
             };
-            // one 128x128x64 block: A tile at a_addr, B = current weight stage
-            auto block = [&](uint32_t d_tmem, uint32_t a_addr, bool first) {
-                const uint32_t s = n % C::NSTAGES, use = n / C::NSTAGES;
-                if (!wait(&misc->w_full[s], use & 1u)) return;
-                const uint64_t ad = ptx::umma_smem_desc_sw128(a_addr);
-                const uint64_t bd = ptx::umma_smem_desc_sw128(wsm + s * kStageBytes);
-#pragma unroll
-                for (uint32_t ks = 0; ks < 4; ++ks)
-                    ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!first || ks > 0) ? 1u : 0u);
-                ptx::umma_commit(ptx::smem_u32(&misc->w_empty[s]));
+            auto wait_tmem = [&](uint64_t* bar, uint32_t parity) {   // orders later UMMAs after TMEM reads
+                const bool r = wait(bar, parity);
+                ptx::tc_fence_after_sync();
+                return r;
+            };
+            auto stage_wait = [&](uint32_t& addr) {
+                const uint32_t s = n % kStages, use = n / kStages;
+                addr = wsm + s * kStageBytes;
+                return wait(&misc->w_full[s], use & 1u);
+            };
+            auto stage_done = [&]() {
+                ptx::umma_commit(ptx::smem_u32(&misc->w_empty[n % kStages]));
                 ++n;
             };
-            auto gemm2 = [&](int cc) {
-                const uint32_t g = hc + cc, buf = g % C::NHBUF, use = g / C::NHBUF;
-                if (!wait(&misc->hs_full[buf], use & 1u)) return;
-                if (cc == 0 && !wait(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                for (int nb = 0; nb < C::NB2 && ok; ++nb)
-                    for (int kb2 = 0; kb2 < 2 && ok; ++kb2)
-                        block(tmem + nb * 128, hs + buf * kHBytes + kb2 * 16384, cc == 0 && kb2 == 0);
-                if (ok) ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[buf]));
+            // GEMM1 of global chunk g = chunk c of local tile ti:  H = X . W1c_chunk^T
+            auto gemm1 = [&](uint32_t g, int c, uint32_t ti) {
+                if (!wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
+                uint32_t b = 0;
+                for (int kb = 0; kb < C::KB1 && ok; ++kb) {
+                    const uint32_t gx = ti * C::KB1 + kb, slot = gx % C::NXS;
+                    if (c == 0 && !wait(&misc->x_full[slot], (gx / C::NXS) & 1u)) return;
+                    if constexpr (D == 384) {
+                        if ((kb & 1) == 0 && !stage_wait(b)) return;
+                        mma_kblock(tm_h, xs + slot * kBlockBytes, b + (kb & 1) * kBlockBytes, idesc128, kb == 0);
+                        if (kb & 1) stage_done();
+                    } else {
+                        if (!stage_wait(b)) return;
+                        mma_kblock(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0);
+                        stage_done();
+                    }
+                    if (c == NC - 1) ptx::umma_commit(ptx::smem_u32(&misc->x_empty[slot]));
+                }
+                ptx::umma_commit(ptx::smem_u32(&misc->h_full));
             };
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
-                if (!wait(&misc->x_full, ti & 1u)) break;
-                for (int c = 0; c < NC && ok; ++c) {
-                    const uint32_t g = hc + c, buf = g % C::NHBUF, use = g / C::NHBUF;
-                    if (!wait(&misc->h_tmem_empty[buf], (use & 1u) ^ 1u)) break;
-                    for (int kb = 0; kb < C::KB1 && ok; ++kb)
-                        block(tmem + C::H_COL0 + buf * 128, xs + kb * 16384, kb == 0);
-                    if (!ok) break;
-                    ptx::umma_commit(ptx::smem_u32(&misc->h_full[buf]));
-                    if (c == NC - 1) ptx::umma_commit(ptx::smem_u32(&misc->x_empty));
-                    if (c > 0) gemm2(c - 1);
-                }
-                if (ok) gemm2(NC - 1);
-                if (ok) ptx::umma_commit(ptx::smem_u32(&misc->y_full));
-                hc += NC;
-            }
-        }
-    } else if (warp < 4) {
-        // ------------------------------------------------------------------ X row gather
-        const int t64 = threadIdx.x - 64;
-        constexpr int CH = D / 8;  // 16-byte chunks per row
-        uint32_t ti = 0;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++ti) {
-            int l, slot0, n_rows;
-            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, slot0, n_rows);
-            // x_empty also orders this write after the epilogue's read of the buffer two tiles back
-            if (!ptx::mbar_wait(ptx::smem_u32(&misc->x_empty), (ti & 1u) ^ 1u, abort_flag)) break;
-            int32_t* rowbuf = misc->row[ti & 1u];
-            for (int r = t64; r < kTileRows; r += kLoaderThreads)
-                rowbuf[r] = r < n_rows ? (int32_t)ffn_row_of_slot(plan, l, slot0 + r, Tlen) : -1;
-            asm volatile("bar.sync 1, 64;" ::: "memory");
-            for (int idx = t64; idx < kTileRows * CH; idx += kLoaderThreads) {
-                const int r = idx / CH, ci = idx % CH;
-                const uint32_t dst = xs + (ci >> 3) * 16384 + r * 128 + (((ci & 7) ^ (r & 7)) << 4);
-                const int32_t grow = rowbuf[r];
-                if (grow >= 0) {
-                    ptx::cp_async_16(dst, X + (size_t)grow * D + ci * 8);
+            // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk
+            auto gemm2 = [&](uint32_t g, int c, uint32_t ti) {
+                const bool first = (c == 0);
+                uint32_t b = 0;
+                if constexpr (D == 256) {
+                    for (int kb2 = 0; kb2 < 4 && ok; ++kb2) {
+                        if (!wait(&misc->hs_full[kb2], g & 1u)) return;
+                        if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                        if (!stage_wait(b)) return;
+                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        stage_done();
+                        ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[kb2]));
+                    }
+                } else if constexpr (D == 128) {
+                    for (int kb2 = 0; kb2 < 4 && ok; ++kb2) {
+                        if (!wait(&misc->hs_full[kb2], g & 1u)) return;
+                        if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                        if ((kb2 & 1) == 0 && !stage_wait(b)) return;
+                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b + (kb2 & 1) * kBlockBytes, idesc128, first && kb2 == 0);
+                        if (kb2 & 1) stage_done();
+                        ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[kb2]));
+                    }
                 } else {
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+                    // columns 0..255 of Y from two N=256 stages, columns 256..383 from one N=128 stage
+                    for (int kb2 = 0; kb2 < 2 && ok; ++kb2) {
+                        if (!wait(&misc->hs_full[kb2], g & 1u)) return;
+                        if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                        if (!stage_wait(b)) return;
+                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        stage_done();
+                    }
+                    if (!ok || !stage_wait(b)) return;
+                    mma_kblock(tmem + 256, hs, b, idesc128, first);
+                    mma_kblock(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false);
+                    stage_done();
+                    ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[0]));
+                    ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[1]));
+                }
+                if (ok && c == NC - 1) ptx::umma_commit(ptx::smem_u32(&misc->y_full));
+            };
+            uint32_t g = 0, ti = 0;
+            bool have_prev = false;
+            uint32_t prev_g = 0, prev_ti = 0;
+            int prev_c = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
+                for (int c = 0; c < NC && ok; ++c, ++g) {
+                    gemm1(g, c, ti);
+                    if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
+                    have_prev = true;
+                    prev_g = g; prev_c = c; prev_ti = ti;
                 }
             }
-            ptx::cp_async_wait_all();
-            ptx::fence_proxy_async_smem();
-            ptx::mbar_arrive(ptx::smem_u32(&misc->x_full));
+            if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
         }
-    } else {
-        // ---------------------------------------------------------------------- epilogue
-        const int quarter = warp & 3, half = (warp - 4) >> 2;
-        const int row = quarter * 32 + lane;
-        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-        uint32_t hc = 0, ti = 0;
+    } else if (warp < kEpiWarp0) {
+        // ------------------------------------------------------------------ X row gather
+        // Thread -> 8 (row, 16-byte chunk) pairs of every 128 x 64 block.  Up to three blocks
+        // are in flight per thread; a block is published (x_full, one arrival per warp) once
+        // the copies of all lanes have landed.
+        const int tl = threadIdx.x - kLoaderWarp0 * 32;
+        uint32_t gx = 0, published = 0;   // blocks issued / published by this warp
         bool ok = true;
-        uint32_t r[32];
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
-            int32_t my_row = -1;
-            for (int c = 0; c < NC; ++c) {
-                const uint32_t g = hc + c, buf = g % C::NHBUF, use = g / C::NHBUF;
-                if (!ptx::mbar_wait(ptx::smem_u32(&misc->h_full[buf]), use & 1u, abort_flag)) { ok = false; break; }
-                ptx::tc_fence_after_sync();
-                if (c == 0) my_row = misc->row[ti & 1u][row];
-                if (!ptx::mbar_wait(ptx::smem_u32(&misc->hs_empty[buf]), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        auto publish_oldest = [&]() {
+            cp_async_wait_pending((int)(gx - published) - 1);
+            ptx::fence_proxy_async_smem();
+            warp_arrive(&misc->x_full[published % C::NXS]);
+            ++published;
+        };
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            int l, row0, n_rows;
+            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
+            int32_t rows[8];
 #pragma unroll
-                for (int cb = 0; cb < 2; ++cb) {
-                    const int col0 = half * 64 + cb * 32;
-                    ptx::tmem_ld_32x32(lane_base + C::H_COL0 + buf * 128 + col0, r);
-                    ptx::tmem_ld_wait();
-                    const uint32_t hrow = hs + buf * kHBytes + (col0 >> 6) * 16384 + row * 128;
-                    const int cc0 = (col0 & 63) >> 3;
+            for (int j = 0; j < 8; ++j) {
+                const int r = (tl + j * kLoaderThreads) >> 3;
+                rows[j] = r < n_rows ? plan.rowidx[row0 + r] : -1;
+            }
+            for (int kb = 0; kb < C::KB1 && ok; ++kb) {
+                const uint32_t slot = gx % C::NXS, use = gx / C::NXS;
+                uint64_t* bar = &misc->x_empty[slot];
+                // never block on a slot while holding unpublished blocks the issuer may need
+                while (gx > published &&
+                       !__all_sync(0xffffffffu, ptx::mbar_test_wait(ptx::smem_u32(bar), (use & 1u) ^ 1u)))
+                    publish_oldest();
+                if (!warp_wait(bar, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint32_t p[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            p[q] = pack_bf16x2(gelu_erf(__uint_as_float(r[8 * j + 2 * q])),
-                                               gelu_erf(__uint_as_float(r[8 * j + 2 * q + 1])));
-                        const uint32_t dst = hrow + (((cc0 + j) ^ (row & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p[0]),
-                                     "r"(p[1]), "r"(p[2]), "r"(p[3])
-                                     : "memory");
+                for (int j = 0; j < 8; ++j) {
+                    const int idx = tl + j * kLoaderThreads;
+                    const int r = idx >> 3, ci = idx & 7;
+                    const uint32_t dst = xs + slot * kBlockBytes + r * 128 + ((ci ^ (r & 7)) << 4);
+                    if (rows[j] >= 0) {
+                        ptx::cp_async_16(dst, X + (size_t)rows[j] * D + kb * 64 + ci * 8);
+                    } else {
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
                     }
                 }
-                ptx::tc_fence_before_sync();
-                ptx::fence_proxy_async_smem();
-                ptx::mbar_arrive(ptx::smem_u32(&misc->h_tmem_empty[buf]));
-                ptx::mbar_arrive(ptx::smem_u32(&misc->hs_full[buf]));
+                ptx::cp_async_commit();
+                ++gx;
+                if (gx - published == 3) publish_oldest();
             }
-            if (!ok) break;
-            if (!ptx::mbar_wait(ptx::smem_u32(&misc->y_full), ti & 1u, abort_flag)) { ok = false; break; }
+        }
+        while (ok && gx > published) publish_oldest();
+        ptx::cp_async_wait_all();
+    } else {
+        // ---------------------------------------------------------------------- epilogue
+        const int ew = warp - kEpiWarp0;
+        const int quarter = warp & 3, half = ew >> 2;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        uint32_t g = 0, ti = 0;
+        bool ok = true;
+        int32_t my_row = -1, prev_row = -1;
+        // Y of a finished tile: TMEM -> bf16 -> global, then hand the accumulator back
+        auto drain_y = [&](uint32_t t_idx, int32_t grow) {
+            if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
+            uint32_t r[32];
 #pragma unroll 1
             for (int cb = 0; cb < D / 64; ++cb) {
                 const int col0 = half * (D / 2) + cb * 32;
                 ptx::tmem_ld_32x32(lane_base + col0, r);
                 ptx::tmem_ld_wait();
-                if (my_row >= 0) {
-                    uint4* dst = reinterpret_cast<uint4*>(Y + (size_t)my_row * D + col0);
+                if (grow >= 0) {
+                    uint4* dst = reinterpret_cast<uint4*>(Y + (size_t)grow * D + col0);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 v;
@@ -282,9 +403,59 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 }
             }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(ptx::smem_u32(&misc->y_empty));
-            hc += NC;
+            warp_arrive(&misc->y_empty);
+        };
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
+            int l, row0, n_rows;
+            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
+            prev_row = my_row;
+            my_row = row < n_rows ? plan.rowidx[row0 + row] : -1;
+            for (int c = 0; c < NC && ok; ++c, ++g) {
+                if (!warp_wait(&misc->h_full, g & 1u, abort_flag)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+#pragma unroll 1
+                for (int j = 0; j < C::NBATCH && ok; ++j) {
+                    // 32 rows x 64 columns of the hidden accumulator -> registers
+                    const int blk = half * C::NBATCH + j;        // hidden block = 64 channels
+                    uint32_t h0[32], h1[32];
+                    const uint32_t tcol = lane_base + C::H_COL0 + blk * 64;
+                    ptx::tmem_ld_32x32(tcol, h0);
+                    ptx::tmem_ld_32x32(tcol + 32, h1);
+                    ptx::tmem_ld_wait();
+                    if (j == C::NBATCH - 1) {
+                        // the accumulator is in registers: GEMM1 of the next chunk may start
+                        ptx::tc_fence_before_sync();
+                        warp_arrive(&misc->h_tmem_empty);
+                        // the previous tile's Y is complete about now (its last GEMM2 was queued
+                        // right after this chunk's GEMM1): store it before the arithmetic
+                        if (c == 0 && ti > 0) {
+                            drain_y(ti - 1, prev_row);
+                            if (!ok) break;
+                        }
+                    }
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        pk[i] = pack_bf16x2(gelu_erf_fast(__uint_as_float(h0[2 * i])),
+                                            gelu_erf_fast(__uint_as_float(h0[2 * i + 1])));
+                        pk[16 + i] = pack_bf16x2(gelu_erf_fast(__uint_as_float(h1[2 * i])),
+                                                 gelu_erf_fast(__uint_as_float(h1[2 * i + 1])));
+                    }
+                    if (!warp_wait(&misc->hs_empty[blk], (g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t hrow = hs + blk * kBlockBytes + row * 128;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t dst = hrow + ((i ^ (row & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * i]),
+                                     "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]), "r"(pk[4 * i + 3])
+                                     : "memory");
+                    }
+                    ptx::fence_proxy_async_smem();
+                    warp_arrive(&misc->hs_full[blk]);
+                }
+            }
         }
+        if (ok && ti > 0) drain_y(ti - 1, my_row);
     }
 
     // ---------------------------------------------------------------------------- teardown
@@ -320,13 +491,13 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// bf16 row-major [rows, cols] -> map with a 128-row x 64-column box, 128-byte swizzle.
-bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols) {
+// bf16 row-major [rows, cols] -> map with a box of `box_rows` rows x 64 columns, 128-byte swizzle.
+bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
     EncodeTiledFn fn = get_encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, 128};
+    cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -334,15 +505,21 @@ bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols) {
 }
 
 template <int D>
-int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, const CUtensorMap& m1,
-             const CUtensorMap& m2, int kc_pad, int max_tiles, cudaStream_t st) {
+int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c, int kc_pad,
+             int max_tiles, cudaStream_t st) {
+    const sentry_ffn_desc& d = a.d;
+    CUtensorMap m1, m2a, m2b;
+    const uint64_t r1 = (uint64_t)d.n_lists * kc_pad, r2 = (uint64_t)d.n_lists * D;
+    if (!make_weight_map(&m1, w1c, r1, D, Cfg<D>::CH == 256 ? 256 : 128)) return SENTRY_ERR_CUDA;
+    if (!make_weight_map(&m2a, w2c, r2, kc_pad, D >= 256 ? 256 : 128)) return SENTRY_ERR_CUDA;
+    if (!make_weight_map(&m2b, w2c, r2, kc_pad, 128)) return SENTRY_ERR_CUDA;
     auto kern = ffn_tc_kernel<D>;
     SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::SMEM_BYTES));
     int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;
     if (grid < 1) grid = 1;
     LaunchScope ls(ctx, KS_FFN_MAIN, st);
-    kern<<<grid, kThreads, Cfg<D>::SMEM_BYTES, st>>>(m1, m2, (const __nv_bfloat16*)a.X, (__nv_bfloat16*)a.Y,
-                                                      plan, a.d.n_lists, a.d.T, kc_pad, a.status);
+    kern<<<grid, kThreads, Cfg<D>::SMEM_BYTES, st>>>(m1, m2a, m2b, (const __nv_bfloat16*)a.X,
+                                                      (__nv_bfloat16*)a.Y, plan, d.n_lists, kc_pad, a.status);
     return SENTRY_OK;
 }
 
@@ -352,19 +529,19 @@ bool ffn_tc_supported(const sentry_ffn_desc& d) {
     return d.dtype == SENTRY_BF16 && (d.D == 128 || d.D == 256 || d.D == 384);
 }
 
-int ffn_tc_kc_pad(int k_c) { return (k_c + kChunk - 1) / kChunk * kChunk; }
+// kept channels are padded with zero columns / rows to a whole number of chunks
+int ffn_tc_kc_pad(int D, int k_c) {
+    const int ch = (D == 384) ? 128 : 256;
+    return (k_c + ch - 1) / ch * ch;
+}
 
 int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,
                   int kc_pad, int max_tiles, cudaStream_t st) {
-    const sentry_ffn_desc& d = a.d;
-    CUtensorMap m1, m2;
-    if (!make_weight_map(&m1, w1c, (uint64_t)d.n_lists * kc_pad, (uint64_t)d.D)) return SENTRY_ERR_CUDA;
-    if (!make_weight_map(&m2, w2c, (uint64_t)d.n_lists * d.D, (uint64_t)kc_pad)) return SENTRY_ERR_CUDA;
     int rc;
-    switch (d.D) {
-        case 128: rc = launch_d<128>(ctx, a, plan, m1, m2, kc_pad, max_tiles, st); break;
-        case 256: rc = launch_d<256>(ctx, a, plan, m1, m2, kc_pad, max_tiles, st); break;
-        case 384: rc = launch_d<384>(ctx, a, plan, m1, m2, kc_pad, max_tiles, st); break;
+    switch (a.d.D) {
+        case 128: rc = launch_d<128>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
+        case 256: rc = launch_d<256>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
+        case 384: rc = launch_d<384>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
         default: return SENTRY_ERR_UNSUPPORTED;
     }
     if (rc != SENTRY_OK) return rc;
