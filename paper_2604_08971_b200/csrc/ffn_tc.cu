@@ -21,7 +21,7 @@
 //
 // Warp roles (480 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
 // warp 1 = UMMA issuer, warps 3-6 = X row gather, warps 7-14 = epilogue (two warps per TMEM
-// lane quarter).  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
+// lane quarter).  Producer and issuer warps stay converged and elect one lane per instruction.  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
 // and unwinds.
 #include <cuda.h>
 #include <math.h>
@@ -105,7 +105,8 @@ __device__ __forceinline__ void warp_arrive(uint64_t* bar) {
     if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(bar));
 }
 
-// Four K=16 steps over one 64-wide K block: D (+)= A[128 x 64] . B[N x 64]^T
+// Four K=16 steps over one 64-wide K block: D (+)= A[128 x 64] . B[N x 64]^T.
+// Called by the one elected lane of a converged warp (see the issuer below).
 __device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr,
                                            uint32_t idesc, bool overwrite) {
     const uint64_t ad = ptx::umma_smem_desc_sw128(a_addr);
@@ -113,6 +114,20 @@ __device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uin
 #pragma unroll
     for (uint32_t ks = 0; ks < 4; ++ks)
         ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
+}
+
+// One lane of a fully converged warp.  The single-thread instructions (TMA, UMMA, commit) are
+// issued from inside `if (elect_one())` while the whole warp walks the schedule: operands
+// computed by all lanes stay warp-uniform, which about halves the cost of issuing them
+// compared with a lane-0 branch around the whole loop.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 
 template <int D>
@@ -167,160 +182,200 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         // ----------------------------------------------------------- weight TMA producers
         // Both walk the issuer's stage sequence (GEMM1 stages of chunk g, then GEMM2 stages of
         // chunk g-1); producer p loads the stages with index n = p (mod 2).
-        if (lane == 0) {
-            const uint32_t me = (warp == 0) ? 0u : 1u;
+        const uint32_t me = (warp == 0) ? 0u : 1u;
+        if (elect_one()) {
             ptx::prefetch_tensormap(&tm_w1);
             ptx::prefetch_tensormap(&tm_w2_256);
             ptx::prefetch_tensormap(&tm_w2_128);
-            uint32_t n = 0;
-            bool ok = true;
-            // one stage = one 32 KB box, or two 16 KB boxes (x1 < 0: single box)
-            auto stage = [&](const CUtensorMap* tm, int x0, int x1, int y) {
-                const uint32_t idx = n++;
-                if (!ok || (idx & 1u) != me) return;
-                const uint32_t s = idx % kStages, use = idx / kStages;
-                if (!ptx::mbar_wait(ptx::smem_u32(&misc->w_empty[s]), (use & 1u) ^ 1u, abort_flag)) {
-                    ok = false;
-                    return;
-                }
-                const uint32_t bar = ptx::smem_u32(&misc->w_full[s]);
-                ptx::mbar_arrive_expect_tx(bar, kStageBytes);
-                ptx::tma_load_2d(wsm + s * kStageBytes, tm, x0, y, bar);
-                if (x1 >= 0) ptx::tma_load_2d(wsm + s * kStageBytes + kBlockBytes, tm, x1, y, bar);
-            };
-            auto gemm1_stages = [&](int l, int c) {
-                const int y = l * kc_pad + c * C::CH;
-                if constexpr (D == 384) {
-                    for (int kp = 0; kp < 3; ++kp) stage(&tm_w1, 128 * kp, 128 * kp + 64, y);
-                } else {
-                    for (int kb = 0; kb < C::KB1; ++kb) stage(&tm_w1, 64 * kb, -1, y);
-                }
-            };
-            auto gemm2_stages = [&](int l, int c) {
-                const int x = c * C::CH;
-                if constexpr (D == 256) {
-                    for (int kb2 = 0; kb2 < 4; ++kb2) stage(&tm_w2_256, x + 64 * kb2, -1, l * D);
-                } else if constexpr (D == 128) {
-                    for (int kp = 0; kp < 2; ++kp) stage(&tm_w2_128, x + 128 * kp, x + 128 * kp + 64, l * D);
-                } else {
-                    stage(&tm_w2_256, x, -1, l * D);
-                    stage(&tm_w2_256, x + 64, -1, l * D);
-                    stage(&tm_w2_128, x, x + 64, l * D + 256);
-                }
-            };
-            int prev_l = -1, prev_c = 0;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                int l, row0, n_rows;
-                ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
-                for (int c = 0; c < NC && ok; ++c) {
-                    gemm1_stages(l, c);
-                    if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
-                    prev_l = l;
-                    prev_c = c;
-                }
-            }
-            if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
         }
+        __syncwarp();
+        uint32_t n = 0;
+        bool ok = true;
+        // one stage = one 32 KB box, or two 16 KB boxes (x1 < 0: single box)
+        auto stage = [&](const CUtensorMap* tm, int x0, int x1, int y) {
+            const uint32_t idx = n++;
+            if (!ok || (idx & 1u) != me) return;
+            const uint32_t s = idx % kStages, use = idx / kStages;
+            if (!warp_wait(&misc->w_empty[s], (use & 1u) ^ 1u, abort_flag)) {
+                ok = false;
+                return;
+            }
+            const uint32_t bar = ptx::smem_u32(&misc->w_full[s]);
+            const uint32_t dst = wsm + s * kStageBytes;
+            if (elect_one()) {
+                ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+                ptx::tma_load_2d(dst, tm, x0, y, bar);
+                if (x1 >= 0) ptx::tma_load_2d(dst + kBlockBytes, tm, x1, y, bar);
+            }
+            __syncwarp();
+        };
+        auto gemm1_stages = [&](int l, int c) {
+            const int y = l * kc_pad + c * C::CH;
+            if constexpr (D == 384) {
+                for (int kp = 0; kp < 3; ++kp) stage(&tm_w1, 128 * kp, 128 * kp + 64, y);
+            } else {
+                for (int kb = 0; kb < C::KB1; ++kb) stage(&tm_w1, 64 * kb, -1, y);
+            }
+        };
+        auto gemm2_stages = [&](int l, int c) {
+            const int x = c * C::CH;
+            if constexpr (D == 256) {
+                for (int kb2 = 0; kb2 < 4; ++kb2) stage(&tm_w2_256, x + 64 * kb2, -1, l * D);
+            } else if constexpr (D == 128) {
+                for (int kp = 0; kp < 2; ++kp) stage(&tm_w2_128, x + 128 * kp, x + 128 * kp + 64, l * D);
+            } else {
+                stage(&tm_w2_256, x, -1, l * D);
+                stage(&tm_w2_256, x + 64, -1, l * D);
+                stage(&tm_w2_128, x, x + 64, l * D + 256);
+            }
+        };
+        int prev_l = -1, prev_c = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            int l, row0, n_rows;
+            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
+            for (int c = 0; c < NC && ok; ++c) {
+                gemm1_stages(l, c);
+                if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
+                prev_l = l;
+                prev_c = c;
+            }
+        }
+        if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
     } else if (warp == 1) {
         // ------------------------------------------------------------------- UMMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
-            constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
-            const uint32_t tm_h = tmem + C::H_COL0;
-            uint32_t n = 0;   // weight stages consumed
-            bool ok = true;
-            auto wait = [&](uint64_t* bar, uint32_t parity) {
-                if (ok && !ptx::mbar_wait(ptx::smem_u32(bar), parity, abort_flag)) ok = false;
-                return ok;
-            };
-            auto wait_tmem = [&](uint64_t* bar, uint32_t parity) {   // orders later UMMAs after TMEM reads
-                const bool r = wait(bar, parity);
-                ptx::tc_fence_after_sync();
-                return r;
-            };
-            auto stage_wait = [&](uint32_t& addr) {
-                const uint32_t s = n % kStages, use = n / kStages;
-                addr = wsm + s * kStageBytes;
-                return wait(&misc->w_full[s], use & 1u);
-            };
-            auto stage_done = [&]() {
-                ptx::umma_commit(ptx::smem_u32(&misc->w_empty[n % kStages]));
-                ++n;
-            };
-            // GEMM1 of global chunk g = chunk c of local tile ti:  H = X . W1c_chunk^T
-            auto gemm1 = [&](uint32_t g, int c, uint32_t ti) {
-                if (!wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
-                uint32_t b = 0;
-                for (int kb = 0; kb < C::KB1 && ok; ++kb) {
+        // The whole warp walks the schedule and waits; one elected lane issues the UMMAs and
+        // their commits (a commit tracks the UMMAs of the thread that issues it).
+        constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
+        constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
+        const uint32_t tm_h = tmem + C::H_COL0;
+        uint32_t n = 0;   // weight stages consumed
+        bool ok = true;
+        auto wait = [&](uint64_t* bar, uint32_t parity) {
+            if (ok) ok = warp_wait(bar, parity, abort_flag);
+            return ok;
+        };
+        auto wait_tmem = [&](uint64_t* bar, uint32_t parity) {   // orders later UMMAs after TMEM reads
+            const bool r = wait(bar, parity);
+            ptx::tc_fence_after_sync();
+            return r;
+        };
+        auto stage_wait = [&]() { return wait(&misc->w_full[n % kStages], (n / kStages) & 1u); };
+        auto bar_of = [&](uint64_t* b) { return ptx::smem_u32(b); };
+        // GEMM1 of global chunk g = chunk c of local tile ti:  H = X . W1c_chunk^T
+        auto gemm1 = [&](uint32_t g, int c, uint32_t ti) {
+            if (!wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
+            const bool last = (c == NC - 1);
+            if constexpr (D == 384) {
+                for (int kp = 0; kp < 3; ++kp) {
+                    const uint32_t s0 = 2 * kp, s1 = 2 * kp + 1;   // X slots (NXS = KB1 = 6)
+                    if (c == 0 && (!wait(&misc->x_full[s0], ti & 1u) || !wait(&misc->x_full[s1], ti & 1u))) return;
+                    if (!stage_wait()) return;
+                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) {
+                        mma_kblock(tm_h, xs + s0 * kBlockBytes, b, idesc128, kp == 0);
+                        if (last) ptx::umma_commit(bar_of(&misc->x_empty[s0]));
+                        mma_kblock(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false);
+                        if (last) ptx::umma_commit(bar_of(&misc->x_empty[s1]));
+                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                        if (kp == 2) ptx::umma_commit(bar_of(&misc->h_full));
+                    }
+                    __syncwarp();
+                    ++n;
+                }
+            } else {
+                for (int kb = 0; kb < C::KB1; ++kb) {
                     const uint32_t gx = ti * C::KB1 + kb, slot = gx % C::NXS;
                     if (c == 0 && !wait(&misc->x_full[slot], (gx / C::NXS) & 1u)) return;
-                    if constexpr (D == 384) {
-                        if ((kb & 1) == 0 && !stage_wait(b)) return;
-                        mma_kblock(tm_h, xs + slot * kBlockBytes, b + (kb & 1) * kBlockBytes, idesc128, kb == 0);
-                        if (kb & 1) stage_done();
-                    } else {
-                        if (!stage_wait(b)) return;
+                    if (!stage_wait()) return;
+                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) {
                         mma_kblock(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0);
-                        stage_done();
+                        if (last) ptx::umma_commit(bar_of(&misc->x_empty[slot]));
+                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                        if (kb == C::KB1 - 1) ptx::umma_commit(bar_of(&misc->h_full));
                     }
-                    if (c == NC - 1) ptx::umma_commit(ptx::smem_u32(&misc->x_empty[slot]));
-                }
-                ptx::umma_commit(ptx::smem_u32(&misc->h_full));
-            };
-            // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk
-            auto gemm2 = [&](uint32_t g, int c, uint32_t ti) {
-                const bool first = (c == 0);
-                uint32_t b = 0;
-                if constexpr (D == 256) {
-                    for (int kb2 = 0; kb2 < 4 && ok; ++kb2) {
-                        if (!wait(&misc->hs_full[kb2], g & 1u)) return;
-                        if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                        if (!stage_wait(b)) return;
-                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
-                        stage_done();
-                        ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[kb2]));
-                    }
-                } else if constexpr (D == 128) {
-                    for (int kb2 = 0; kb2 < 4 && ok; ++kb2) {
-                        if (!wait(&misc->hs_full[kb2], g & 1u)) return;
-                        if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                        if ((kb2 & 1) == 0 && !stage_wait(b)) return;
-                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b + (kb2 & 1) * kBlockBytes, idesc128, first && kb2 == 0);
-                        if (kb2 & 1) stage_done();
-                        ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[kb2]));
-                    }
-                } else {
-                    // columns 0..255 of Y from two N=256 stages, columns 256..383 from one N=128 stage
-                    for (int kb2 = 0; kb2 < 2 && ok; ++kb2) {
-                        if (!wait(&misc->hs_full[kb2], g & 1u)) return;
-                        if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                        if (!stage_wait(b)) return;
-                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
-                        stage_done();
-                    }
-                    if (!ok || !stage_wait(b)) return;
-                    mma_kblock(tmem + 256, hs, b, idesc128, first);
-                    mma_kblock(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false);
-                    stage_done();
-                    ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[0]));
-                    ptx::umma_commit(ptx::smem_u32(&misc->hs_empty[1]));
-                }
-                if (ok && c == NC - 1) ptx::umma_commit(ptx::smem_u32(&misc->y_full));
-            };
-            uint32_t g = 0, ti = 0;
-            bool have_prev = false;
-            uint32_t prev_g = 0, prev_ti = 0;
-            int prev_c = 0;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
-                for (int c = 0; c < NC && ok; ++c, ++g) {
-                    gemm1(g, c, ti);
-                    if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
-                    have_prev = true;
-                    prev_g = g; prev_c = c; prev_ti = ti;
+                    __syncwarp();
+                    ++n;
                 }
             }
-            if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
+        };
+        // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk
+        auto gemm2 = [&](uint32_t g, int c, uint32_t ti) {
+            const bool first = (c == 0), last = (c == NC - 1);
+            if constexpr (D == 256) {
+                for (int kb2 = 0; kb2 < 4; ++kb2) {
+                    if (!wait(&misc->hs_full[kb2], g & 1u)) return;
+                    if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                    if (!stage_wait()) return;
+                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) {
+                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                        ptx::umma_commit(bar_of(&misc->hs_empty[kb2]));
+                        if (last && kb2 == 3) ptx::umma_commit(bar_of(&misc->y_full));
+                    }
+                    __syncwarp();
+                    ++n;
+                }
+            } else if constexpr (D == 128) {
+                for (int kp = 0; kp < 2; ++kp) {
+                    const int k0 = 2 * kp, k1 = 2 * kp + 1;
+                    if (!wait(&misc->hs_full[k0], g & 1u) || !wait(&misc->hs_full[k1], g & 1u)) return;
+                    if (first && kp == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                    if (!stage_wait()) return;
+                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) {
+                        mma_kblock(tmem, hs + k0 * kBlockBytes, b, idesc128, first && kp == 0);
+                        ptx::umma_commit(bar_of(&misc->hs_empty[k0]));
+                        mma_kblock(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false);
+                        ptx::umma_commit(bar_of(&misc->hs_empty[k1]));
+                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                        if (last && kp == 1) ptx::umma_commit(bar_of(&misc->y_full));
+                    }
+                    __syncwarp();
+                    ++n;
+                }
+            } else {
+                // columns 0..255 of Y from two N=256 stages, columns 256..383 from one N=128 stage
+                for (int kb2 = 0; kb2 < 2; ++kb2) {
+                    if (!wait(&misc->hs_full[kb2], g & 1u)) return;
+                    if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                    if (!stage_wait()) return;
+                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) {
+                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                    }
+                    __syncwarp();
+                    ++n;
+                }
+                if (!stage_wait()) return;
+                const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                if (elect_one()) {
+                    mma_kblock(tmem + 256, hs, b, idesc128, first);
+                    mma_kblock(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false);
+                    ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                    ptx::umma_commit(bar_of(&misc->hs_empty[0]));
+                    ptx::umma_commit(bar_of(&misc->hs_empty[1]));
+                    if (last) ptx::umma_commit(bar_of(&misc->y_full));
+                }
+                __syncwarp();
+                ++n;
+            }
+        };
+        uint32_t g = 0, ti = 0;
+        bool have_prev = false;
+        uint32_t prev_g = 0, prev_ti = 0;
+        int prev_c = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
+            for (int c = 0; c < NC && ok; ++c, ++g) {
+                gemm1(g, c, ti);
+                if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
+                have_prev = true;
+                prev_g = g; prev_c = c; prev_ti = ti;
+            }
         }
+        if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
     } else if (warp < kEpiWarp0) {
         // ------------------------------------------------------------------ X row gather
         // Thread -> 8 (row, 16-byte chunk) pairs of every 128 x 64 block.  Up to three blocks
@@ -379,28 +434,46 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         uint32_t g = 0, ti = 0;
         bool ok = true;
         int32_t my_row = -1, prev_row = -1;
-        // Y of a finished tile: TMEM -> bf16 -> global, then hand the accumulator back
+        // Y of a finished tile: TMEM -> bf16 -> global, then hand the accumulator back.  Each
+        // lane holds one row; 64 columns at a time go through this warp's 4 KB piece of the
+        // hidden-block buffer (free while Y is complete and this warp has not yet written its
+        // next hidden block there) so that the global stores cover whole 128-byte row segments.
+        constexpr int kDrainBlk = C::NBATCH - 1;
+        const uint32_t stg = hs + (uint32_t)(half * C::NBATCH + kDrainBlk) * kBlockBytes + (uint32_t)quarter * 4096u;
         auto drain_y = [&](uint32_t t_idx, int32_t grow) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
-            uint32_t r[32];
 #pragma unroll 1
-            for (int cb = 0; cb < D / 64; ++cb) {
-                const int col0 = half * (D / 2) + cb * 32;
-                ptx::tmem_ld_32x32(lane_base + col0, r);
-                ptx::tmem_ld_wait();
-                if (grow >= 0) {
-                    uint4* dst = reinterpret_cast<uint4*>(Y + (size_t)grow * D + col0);
+            for (int pass = 0; pass < D / 128; ++pass) {
+                const int col0 = half * (D / 2) + pass * 64;
+#pragma unroll 1
+                for (int sub = 0; sub < 2; ++sub) {
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(lane_base + col0 + sub * 32, r);
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 v;
-                        v.x = pack_bf16x2(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1]));
-                        v.y = pack_bf16x2(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                        v.z = pack_bf16x2(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                        v.w = pack_bf16x2(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                        dst[j] = v;
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t dst = stg + lane * 128 + (((4 * sub + i) ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
+                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1]))),
+                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]))),
+                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]))),
+                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])))
+                                     : "memory");
                     }
                 }
+                __syncwarp();
+#pragma unroll
+                for (int step = 0; step < 8; ++step) {
+                    const int rr = step * 4 + (lane >> 3), ch = lane & 7;
+                    uint4 v;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                 : "r"(stg + rr * 128 + ((ch ^ (rr & 7)) << 4)));
+                    const int32_t gr = __shfl_sync(0xffffffffu, grow, rr);
+                    if (gr >= 0) *reinterpret_cast<uint4*>(Y + (size_t)gr * D + col0 + ch * 8) = v;
+                }
+                __syncwarp();
             }
             ptx::tc_fence_before_sync();
             warp_arrive(&misc->y_empty);
