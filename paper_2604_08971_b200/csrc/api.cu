@@ -95,7 +95,7 @@ int sentry_profile_slots(void) { return KS_COUNT; }
 
 const char* sentry_kernel_name(int slot) {
     static const char* names[KS_COUNT] = {"gate_rows", "gate_expand", "attend_score", "attend_select",
-                                          "attend_core", "ffn_plan", "ffn_prepare", "ffn_main"};
+                                          "attend_core", "ffn_prepare", "ffn_main"};
     return (slot >= 0 && slot < KS_COUNT) ? names[slot] : "?";
 }
 

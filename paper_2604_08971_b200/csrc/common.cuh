@@ -13,7 +13,7 @@
 // Kernel slots for launch accounting and optional per-kernel timing.
 enum KernelSlot {
     KS_GATE_ROWS = 0, KS_GATE_EXPAND, KS_ATT_SCORE, KS_ATT_SELECT, KS_ATT_CORE,
-    KS_FFN_PLAN, KS_FFN_PREPARE, KS_FFN_MAIN, KS_COUNT
+    KS_FFN_PREPARE, KS_FFN_MAIN, KS_COUNT
 };
 
 struct ProfRec { cudaEvent_t start, stop; int slot; };
@@ -119,24 +119,88 @@ __device__ __forceinline__ int block_sum_int(int v, int* red) {
     return t;
 }
 
+// Top-k of n keys by rank counting, for rows short enough that n^2 comparisons are cheaper
+// than 32 rounds of block-wide counting: element i is kept iff fewer than k elements come
+// before it in the order (larger key first, equal keys -> lower index first).  Same contract
+// as block_select_topk.
+__device__ inline void block_select_topk_rank(const uint32_t* keys, int n, int k, int32_t* out,
+                                              const uint16_t* remap, int* red) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    int* wk = red;
+    int base = 0;
+    for (int i0 = 0; i0 < n; i0 += blockDim.x) {
+        const int i = i0 + threadIdx.x;
+        bool keep = false;
+        if (i < n) {
+            const uint32_t mine = keys[i];
+            int before = 0;
+            for (int j = 0; j < i; ++j) before += (keys[j] >= mine);      // earlier index wins ties
+            for (int j = i + 1; j < n; ++j) before += (keys[j] > mine);
+            keep = before < k;
+        }
+        const unsigned km = __ballot_sync(0xffffffffu, keep);
+        __syncthreads();
+        if (lane == 0) wk[wid] = __popc(km);
+        __syncthreads();
+        int pos = base, tot = 0;
+        for (int w = 0; w < nw; ++w) { if (w < wid) pos += wk[w]; tot += wk[w]; }
+        if (keep) out[pos + __popc(km & ((1u << lane) - 1u))] = remap ? (int32_t)remap[i] : i;
+        base += tot;
+    }
+    __syncthreads();
+}
+
 // Top-k of n keys held in shared memory, larger key first, equal keys -> lower
 // index first.  Writes the selected indices to out[0..k) in ASCENDING index
 // order, mapped through `remap` (uint16 list) when given.  All threads of the
 // block must call it.  `red` = 33 ints of smem.  Requires 1 <= k <= n.
 __device__ inline void block_select_topk(const uint32_t* keys, int n, int k, int32_t* out,
                                          const uint16_t* remap, int* red) {
-    // 1. threshold = largest t with |{key >= t}| >= k (bitwise search)
-    uint32_t t = 0;
-    for (int bit = 31; bit >= 0; --bit) {
-        const uint32_t cand = t | (1u << bit);
-        int cnt = 0;
-        for (int i = threadIdx.x; i < n; i += blockDim.x) cnt += (keys[i] >= cand);
-        cnt = block_sum_int(cnt, red);
-        if (cnt >= k) t = cand;
+    if (n <= 256) { block_select_topk_rank(keys, n, k, out, remap, red); return; }
+    // 1. t = the k-th largest key, by radix selection: four passes over 8-bit digits, each a
+    //    shared-memory histogram of the keys that still match the digits fixed so far, scanned
+    //    from the top digit down by one warp.
+    __shared__ int s_hist[256];
+    __shared__ int s_pick[2];   // chosen digit, keys still to take inside it
+    uint32_t prefix = 0, fixed = 0;
+    int want = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const uint32_t key = keys[i];
+            if ((key & fixed) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            // lane L owns digits 255-8L .. 248-8L (descending); inclusive scan over lanes
+            const int top = 255 - 8 * (int)threadIdx.x;
+            int mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mine += s_hist[top - j];
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if ((int)threadIdx.x >= o) incl += v;
+            }
+            const int above = incl - mine;               // keys in digits above this lane's
+            if (above < want && want <= incl) {          // the k-th key falls into this lane's digits
+                int acc = above;
+                for (int j = 0; j < 8; ++j) {
+                    const int c = s_hist[top - j];
+                    if (want <= acc + c) { s_pick[0] = top - j; s_pick[1] = want - acc; break; }
+                    acc += c;
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= (uint32_t)s_pick[0] << shift;
+        fixed |= 255u << shift;
+        want = s_pick[1];
     }
-    int gt = 0;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) gt += (keys[i] > t);
-    gt = block_sum_int(gt, red);
+    const uint32_t t = prefix;
+    const int gt = k - want;     // keys strictly above t; `want` of the keys equal to t are taken
     const int need_eq = k - gt;
     // 2. ordered compaction: everything above t, plus the first need_eq equal to t
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;

@@ -18,100 +18,84 @@ constexpr int kGenericTileRows = 16;
 constexpr int kGenericThreads = 256;
 constexpr int kTcTileRows = 128;
 
-// One CTA.  Present rows per sample (from the per-modality token counts), then per list a
-// stable scan over its samples: where each sample's rows start in the row table, where
-// each list starts, and how many tiles each list needs.
-__global__ void __launch_bounds__(1024)
-ffn_plan_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks,
-                const int32_t* __restrict__ list_of_sample, int B, int T, int n_lists,
-                int tile_rows, FfnPlan p, unsigned int* status) {
-    __shared__ int s_cnt[32];
-    __shared__ int s_warp_rows[32];
-    __shared__ int s_base_rows, s_list_row0;
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    if (threadIdx.x < 32) s_cnt[threadIdx.x] = 0;
-    if (threadIdx.x == 0) { s_list_row0 = 0; p.tile_start[0] = 0; p.list_row0[0] = 0; }
-    __syncthreads();
-    if (ids != nullptr) {
-        for (int t = threadIdx.x; t < T; t += blockDim.x) {
-            const int m = ids[t];
-            if (m >= 0 && m < 32) atomicAdd(&s_cnt[m], 1);
-            else atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
-        }
-        __syncthreads();
-    }
-    auto present_rows = [&](int b) {
-        if (ids == nullptr) return T;
-        uint32_t mask = masks[b];
-        int n = 0;
-        while (mask) { const int m = __ffs(mask) - 1; n += s_cnt[m]; mask &= mask - 1; }
-        return n;
-    };
-    for (int l = 0; l < n_lists; ++l) {
-        if (threadIdx.x == 0) s_base_rows = 0;
-        __syncthreads();
-        for (int b0 = 0; b0 < B; b0 += blockDim.x) {
-            const int b = b0 + threadIdx.x;
-            int rows = 0;
-            bool mine = false;
-            if (b < B) {
-                int lb = list_of_sample ? list_of_sample[b] : 0;
-                if (lb < 0 || lb >= n_lists) {
-                    if (l == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
-                    lb = 0;
-                }
-                mine = (lb == l);
-                if (mine) {
-                    rows = present_rows(b);
-                    if (rows == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
-                }
-            }
-            int r = rows;  // inclusive warp scan
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int r2 = __shfl_up_sync(0xffffffffu, r, o);
-                if (lane >= o) r += r2;
-            }
-            if (lane == 31) s_warp_rows[wid] = r;
-            __syncthreads();
-            int before = s_base_rows, tot = 0;
-            for (int w = 0; w < nw; ++w) {
-                if (w < wid) before += s_warp_rows[w];
-                tot += s_warp_rows[w];
-            }
-            if (mine) p.sample_row0[b] = s_list_row0 + before + r - rows;
-            __syncthreads();
-            if (threadIdx.x == 0) s_base_rows += tot;
-            __syncthreads();
-        }
-        if (threadIdx.x == 0) {
-            s_list_row0 += s_base_rows;
-            p.list_row0[l + 1] = s_list_row0;
-            p.tile_start[l + 1] = p.tile_start[l] + (s_base_rows + tile_rows - 1) / tile_rows;
-        }
-        __syncthreads();
-    }
-}
-
-// Blocks [0, B): row table entries of sample b (its present tokens, ascending) and zero rows
-// of Y for its absent tokens.  Blocks [B, B + prepack blocks): the weight gather, which
-// "materialises" the pruned W1', W2' of every kept list.
-//   layout 0 (plain-ALU kernel): W1g [l][D][kc_pad], W2g [l][kc_pad][D]
-//   layout 1 (tensor-core kernel, both K-major): W1c [l][kc_pad][D], W2c [l][D][kc_pad]
-// Columns / rows n >= k_c are zero.
+// One launch prepares everything the main kernel needs.  Block ranges:
+//   [0, B)              row table of sample b: every block finds by itself where its sample's
+//                       rows start (a scan over all samples' lists and present-row counts, so no
+//                       separate planning launch is needed); block 0 also writes the per-list
+//                       offsets and tile counts
+//   [B, B + B*zsplit)   zero rows of Y for the absent tokens of a sample (slices of its rows)
+//   [.., + prepack)     the weight gather, which "materialises" the pruned W1', W2' per list:
+//     layout 0 (plain-ALU kernel): W1g [l][D][kc_pad], W2g [l][kc_pad][D]
+//     layout 1 (tensor-core kernel, both K-major): W1c [l][kc_pad][D], W2c [l][D][kc_pad]
+//     columns / rows n >= k_c are zero.
 template <typename T>
 __global__ void __launch_bounds__(256)
-ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks, int B,
-                   int Tlen, FfnPlan p, uint8_t* __restrict__ Y,
+ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks,
+                   const int32_t* __restrict__ list_of_sample, int B, int Tlen, int zsplit,
+                   int tile_rows, FfnPlan p, uint8_t* __restrict__ Y,
                    const T* __restrict__ W1, const T* __restrict__ W2,
                    const int32_t* __restrict__ kept, int n_lists, int D, int F, int k_c, int kc_pad,
                    int layout, T* __restrict__ out1, T* __restrict__ out2, unsigned int* status) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     if ((int)blockIdx.x < B) {
-        __shared__ int red[33];
+        __shared__ int s_cnt[32];
+        __shared__ int red[66];
         const int b = blockIdx.x;
+        if (threadIdx.x < 32) s_cnt[threadIdx.x] = 0;
+        __syncthreads();
+        if (ids != nullptr) {
+            for (int t = threadIdx.x; t < Tlen; t += blockDim.x) {
+                const int m = ids[t];
+                if (m >= 0 && m < 32) atomicAdd(&s_cnt[m], 1);
+                else if (b == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+            }
+            __syncthreads();
+        }
+        auto present_rows = [&](int bb) {
+            if (ids == nullptr) return Tlen;
+            uint32_t mask = masks[bb];
+            int n = 0;
+            while (mask) { const int m = __ffs(mask) - 1; n += s_cnt[m]; mask &= mask - 1; }
+            return n;
+        };
+        auto list_of = [&](int bb) {
+            int l = list_of_sample ? list_of_sample[bb] : 0;
+            if (l < 0 || l >= n_lists) {
+                if (b == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+                l = 0;
+            }
+            return l;
+        };
+        // rows of all samples in earlier lists, and of earlier samples in this sample's list
+        const int my_list = list_of(b);
+        int before = 0;
+        for (int bb = threadIdx.x; bb < B; bb += blockDim.x) {
+            const int l = list_of(bb);
+            if (l < my_list || (l == my_list && bb < b)) before += present_rows(bb);
+        }
+        before = block_sum_int(before, red);
+        if (threadIdx.x == 0) p.sample_row0[b] = before;
+        if (b == 0) {
+            // per-list totals -> list offsets and tile counts (lists are few: one pass each)
+            int row0 = 0, tile0 = 0;
+            for (int l = 0; l < n_lists; ++l) {
+                int rows = 0;
+                for (int bb = threadIdx.x; bb < B; bb += blockDim.x)
+                    if (list_of(bb) == l) {
+                        const int r = present_rows(bb);
+                        rows += r;
+                        if (r == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
+                    }
+                rows = block_sum_int(rows, red);
+                if (threadIdx.x == 0) { p.list_row0[l] = row0; p.tile_start[l] = tile0; }
+                row0 += rows;
+                tile0 += (rows + tile_rows - 1) / tile_rows;
+            }
+            if (threadIdx.x == 0) { p.list_row0[n_lists] = row0; p.tile_start[n_lists] = tile0; }
+        }
+        // present tokens of this sample, ascending -> row table
         const uint32_t mask = (ids != nullptr) ? masks[b] : 0xffffffffu;
-        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-        int32_t* rows = p.rowidx + p.sample_row0[b];
+        int32_t* rows = p.rowidx + before;
         int base = 0;
         for (int t0 = 0; t0 < Tlen; t0 += blockDim.x) {
             const int t = t0 + threadIdx.x;
@@ -129,20 +113,29 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
             if (ok) rows[pos + __popc(bm & ((1u << lane) - 1u))] = b * Tlen + t;
             base += tot;
         }
-        if (ids == nullptr || base == Tlen) return;
-        // zero the rows of absent tokens, 16 bytes per store, all threads busy
+        return;
+    }
+    size_t pb = (size_t)blockIdx.x - B;
+    const size_t zero_blocks = (ids != nullptr) ? (size_t)B * zsplit : 0;
+    if (pb < zero_blocks) {
+        // zero the rows of absent tokens, 16 bytes per store
+        const int b = (int)(pb / zsplit), part = (int)(pb % zsplit);
+        const uint32_t mask = masks[b];
         const int vpr = D * (int)sizeof(T) / 16;
+        const int total = Tlen * vpr;
+        const int per = (total + zsplit - 1) / zsplit;
+        const int end = min(total, (part + 1) * per);
         uint4* Yb = reinterpret_cast<uint4*>(Y + (size_t)b * Tlen * D * sizeof(T));
-        for (int i = threadIdx.x; i < Tlen * vpr; i += blockDim.x) {
+        for (int i = part * per + threadIdx.x; i < end; i += blockDim.x) {
             const int m = ids[i / vpr];
             const bool present = (m >= 0 && m < 32) && ((mask >> m) & 1u);
             if (!present) Yb[i] = make_uint4(0, 0, 0, 0);
         }
         return;
     }
+    pb -= zero_blocks;
     const size_t per = (size_t)kc_pad * D;
     const size_t blocks_per = (per + 255) / 256;
-    size_t pb = (size_t)blockIdx.x - B;
     const int which = (int)(pb / (blocks_per * n_lists));
     pb -= (size_t)which * blocks_per * n_lists;
     const int l = (int)(pb / blocks_per);
@@ -290,25 +283,24 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cud
     const int tile_rows = tc ? kTcTileRows : kGenericTileRows;
 
     {
-        LaunchScope ls(ctx, KS_FFN_PLAN, st);
-        ffn_plan_kernel<<<1, 1024, 0, st>>>(a.ids, a.masks, a.list_of_sample, d.B, d.T, d.n_lists,
-                                             tile_rows, w.plan, a.status);
-    }
-    SENTRY_CUDA_TRY(cudaGetLastError());
-    {
         const size_t per = (size_t)kc_pad * d.D;
-        const size_t grid = (size_t)d.B + 2 * (size_t)d.n_lists * ((per + 255) / 256);
+        // enough zero-fill blocks to cover the GPU a few times over when the batch is small
+        int zsplit = (4 * ctx->sm_count + d.B - 1) / d.B;
+        if (zsplit < 1) zsplit = 1;
+        if (zsplit > 32) zsplit = 32;
+        const size_t grid = (size_t)d.B + (a.ids != nullptr ? (size_t)d.B * zsplit : 0) +
+                            2 * (size_t)d.n_lists * ((per + 255) / 256);
         LaunchScope ls(ctx, KS_FFN_PREPARE, st);
         if (d.dtype == SENTRY_F32)
             ffn_prepare_kernel<float><<<(unsigned)grid, 256, 0, st>>>(
-                a.ids, a.masks, d.B, d.T, w.plan, (uint8_t*)a.Y, (const float*)a.W1,
-                (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, (float*)w.w1p,
-                (float*)w.w2p, a.status);
+                a.ids, a.masks, a.list_of_sample, d.B, d.T, zsplit, tile_rows, w.plan, (uint8_t*)a.Y,
+                (const float*)a.W1, (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0,
+                (float*)w.w1p, (float*)w.w2p, a.status);
         else
             ffn_prepare_kernel<__nv_bfloat16><<<(unsigned)grid, 256, 0, st>>>(
-                a.ids, a.masks, d.B, d.T, w.plan, (uint8_t*)a.Y, (const __nv_bfloat16*)a.W1,
-                (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, tc ? 1 : 0,
-                (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
+                a.ids, a.masks, a.list_of_sample, d.B, d.T, zsplit, tile_rows, w.plan, (uint8_t*)a.Y,
+                (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F,
+                d.k_c, kc_pad, tc ? 1 : 0, (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
     const long long rows = (long long)d.B * d.T;

@@ -130,6 +130,7 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2_256,

@@ -8,10 +8,16 @@
 
 namespace {
 
-constexpr int kGateThreads = 128;
+constexpr int kGateMaxThreads = 1024;
+
+// Block size of the per-row selection: one key per thread up to 1024 threads.
+inline int gate_threads(int n_units) {
+    int t = (n_units + 31) / 32 * 32;
+    return t < 64 ? 64 : (t > kGateMaxThreads ? kGateMaxThreads : t);
+}
 
 // One block per score-table row s: rows[s, 0..k) and groups[s].
-__global__ void __launch_bounds__(kGateThreads)
+__global__ void __launch_bounds__(kGateMaxThreads)
 gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
                  int32_t* __restrict__ rows, uint32_t* __restrict__ groups,
                  int heads_per_group) {
@@ -68,7 +74,7 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
         LaunchScope ls(ctx, KS_GATE_ROWS, st);
-        gate_rows_kernel<<<S, kGateThreads, smem, st>>>(scores, n_units, k, ws_rows,
+        gate_rows_kernel<<<S, gate_threads(n_units), smem, st>>>(scores, n_units, k, ws_rows,
                                                          kv_groups ? ws_groups : nullptr,
                                                          heads_per_group > 0 ? heads_per_group : 1);
     }
@@ -173,7 +179,7 @@ extern "C" int sentry_gate_select_static(int device, const float* scores, int S,
     // The array keeps whatever the previous call left.  rows/groups are rewritten in full for
     // all S score rows before the fan-out reads them; only the status word must start at zero.
     SENTRY_CUDA_TRY(cudaMemsetAsync(own_status, 0, sizeof(unsigned int), st));
-    gate_rows_kernel<<<S, kGateThreads, (size_t)n_units * sizeof(uint32_t), st>>>(
+    gate_rows_kernel<<<S, gate_threads(n_units), (size_t)n_units * sizeof(uint32_t), st>>>(
         scores, n_units, k, rows, kv_groups ? groups : nullptr, heads_per_group > 0 ? heads_per_group : 1);
     SENTRY_CUDA_TRY(cudaGetLastError());
     const size_t total = (size_t)n_masks * k;
