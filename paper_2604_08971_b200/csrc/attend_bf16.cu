@@ -570,9 +570,466 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     }
 }
 
+// ------------------------------------------------------------------------------------ fused
+// One CTA per (sample, KV group) does the whole of SentryAttend for the group's kept heads
+// when the group's present K and V rows fit in shared memory (T up to ~1.5 k at d = 32):
+//   stage K, V (gathered present rows, once) -> sparsity scores from shared memory ->
+//   top-U per head (one warp per head, radix selection) -> Eq. 6 on the active rows with the
+//   warp-level tensor-core MMA straight from the resident K/V -> context rows and zero rows.
+// Q, K, V are read from HBM once and O is written once: the algorithmic traffic.
+
+// Warp-level top-k by radix selection over n order keys in shared memory (larger key first,
+// ties -> lower index).  Writes remap[index] of the selected entries to out[0..k) in ascending
+// index order.  `hist` = 256 ints of shared memory owned by this warp.
+__device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k, int32_t* out,
+                                              const uint16_t* remap, int* hist) {
+    const int lane = threadIdx.x & 31;
+    uint32_t prefix = 0, fixed = 0;
+    int want = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = lane; i < 256; i += 32) hist[i] = 0;
+        __syncwarp();
+        for (int i = lane; i < n; i += 32) {
+            const uint32_t key = keys[i];
+            if ((key & fixed) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+        }
+        __syncwarp();
+        const int top = 255 - 8 * lane;      // this lane's digits, descending
+        int mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine += hist[top - j];
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int above = incl - mine;
+        const bool here = above < want && want <= incl;
+        int digit = 0, rem = 0;
+        if (here) {
+            int acc = above;
+            for (int j = 0; j < 8; ++j) {
+                const int cdig = hist[top - j];
+                if (want <= acc + cdig) { digit = top - j; rem = want - acc; break; }
+                acc += cdig;
+            }
+        }
+        const unsigned who = __ballot_sync(0xffffffffu, here);
+        const int src = __ffs(who) - 1;
+        digit = __shfl_sync(0xffffffffu, digit, src);
+        rem = __shfl_sync(0xffffffffu, rem, src);
+        prefix |= (uint32_t)digit << shift;
+        fixed |= 255u << shift;
+        want = rem;
+        __syncwarp();
+    }
+    const uint32_t t = prefix;
+    const int need_eq = want;
+    int base = 0, eq_seen = 0;
+    for (int i0 = 0; i0 < n; i0 += 32) {
+        const int i = i0 + lane;
+        const uint32_t key = i < n ? keys[i] : 0u;
+        const bool is_eq = i < n && key == t, is_gt = i < n && key > t;
+        const unsigned em = __ballot_sync(0xffffffffu, is_eq);
+        const bool keep = is_gt || (is_eq && eq_seen + __popc(em & ((1u << lane) - 1u)) < need_eq);
+        const unsigned km = __ballot_sync(0xffffffffu, keep);
+        if (keep) out[base + __popc(km & ((1u << lane) - 1u))] = (int32_t)remap[i];
+        base += __popc(km);
+        eq_seen += __popc(em);
+    }
+    __syncwarp();
+}
+
+// Sparsity scores of NH heads of the group at once for the queries of this thread:
+// M_i = max_j s_ij - mean_j s_ij over the sampled (or all) present keys, K rows from shared
+// memory.  The order keys of the scores go to keys_out[h][p].
+template <int D, int NH>
+__device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict__ Q, size_t q_head_stride,
+                                                 const size_t* q_base, const uint16_t* s_valid,
+                                                 uint32_t ks_addr, int Tv,
+                                                 const int32_t* __restrict__ tbl, int n_s, int cnt,
+                                                 int score_mode, uint32_t* const* keys_out,
+                                                 unsigned int* status) {
+    using S = Sw<D>;
+    const float scale = rsqrtf((float)D);
+    const float inv_cnt = 1.0f / (float)cnt;
+    for (int p = threadIdx.x; p < Tv; p += blockDim.x) {
+        const int tok = s_valid[p];
+        float q[NH][D];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            const uint4* src = reinterpret_cast<const uint4*>(Q + q_base[h] + (size_t)tok * D);
+#pragma unroll
+            for (int cc = 0; cc < S::CPR; ++cc) {
+                float f[8];
+                unpack8(__ldg(src + cc), f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) q[h][8 * cc + e] = f[e];
+            }
+        }
+        float mx[NH], sum[NH];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) { mx[h] = -INFINITY; sum[h] = 0.f; }
+        const int32_t* row = score_mode == 0 ? tbl + (size_t)p * n_s : nullptr;
+        int pj_next = score_mode == 0 ? __ldg(row) : 0;
+        for (int a = 0; a < cnt; ++a) {
+            int pj = pj_next;
+            if (a + 1 < cnt) pj_next = score_mode == 0 ? __ldg(row + a + 1) : a + 1;
+            if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
+            float dot[NH];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) dot[h] = 0.f;
+#pragma unroll
+            for (int cc = 0; cc < S::CPR; ++cc) {
+                float f[8];
+                unpack8(lds128(ks_addr + S::off(pj, cc)), f);
+#pragma unroll
+                for (int h = 0; h < NH; ++h)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) dot[h] = fmaf(q[h][8 * cc + e], f[e], dot[h]);
+            }
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                const float sc = dot[h] * scale;
+                mx[h] = fmaxf(mx[h], sc);
+                sum[h] += sc;
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < NH; ++h) keys_out[h][p] = sentry_order_key(mx[h] - sum[h] * inv_cnt);
+    }
+}
+
+// grid B*Hk, 256 or 512 threads.  Dynamic smem: valid[T] u16 | kind[T] u8 | actbits[4][T/32] u32 |
+// keys[4][T] u32 | hist[4][256] | K[Tpad][D] | V[Tpad][D]   (Tpad = T rounded up to 64).
+template <int D>
+__global__ void __launch_bounds__(512, 1)
+attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
+                         const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ kept_heads,
+                         const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks,
+                         const int32_t* __restrict__ table, const int64_t* __restrict__ offsets,
+                         int n_subsets, const int32_t* __restrict__ active_in,
+                         int32_t* __restrict__ active_out, int Tlen, int Hq, int Hk, int k_h, int c,
+                         int score_mode, int U_max, __nv_bfloat16* __restrict__ O, unsigned int* status) {
+    using S = Sw<D>;
+    constexpr int NT = D / 8;        // n-tiles of the output (8 dims each)
+    constexpr int KS = D / 16;       // k-steps of q.k
+    constexpr int TILE_BYTES = kKeyTile * D * 2;
+    extern __shared__ __align__(128) uint8_t s_raw[];
+    __shared__ int red[66];
+    __shared__ int32_t s_act[kMaxRK][kMaxActive];
+    __shared__ float s_vpart[512 / (D / 2)][D];
+    __shared__ __align__(16) __nv_bfloat16 s_mean[D];
+
+    const int words = (Tlen + 31) / 32;
+    const int Tpad = (Tlen + kKeyTile - 1) / kKeyTile * kKeyTile;
+    size_t o = 0;
+    uint16_t* s_valid = reinterpret_cast<uint16_t*>(s_raw + o); o += (((size_t)Tlen * 2 + 127) / 128) * 128;
+    uint8_t* s_kind = s_raw + o;                                o += (((size_t)Tlen + 127) / 128) * 128;
+    uint32_t* s_abits = reinterpret_cast<uint32_t*>(s_raw + o); o += (((size_t)kMaxRK * words * 4 + 127) / 128) * 128;
+    uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_raw + o);  o += (((size_t)kMaxRK * Tlen * 4 + 127) / 128) * 128;
+    int* s_hist = reinterpret_cast<int*>(s_raw + o);            o += (size_t)kMaxRK * 256 * 4;
+    const uint32_t ks_addr = ptx::smem_u32(s_raw + o);          o += (size_t)Tpad * D * 2;
+    const uint32_t vs_addr = ptx::smem_u32(s_raw + o);
+
+    const int b = blockIdx.x / Hk, g = blockIdx.x % Hk;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const uint32_t mask = masks[b];
+    const int Tv = block_build_valid(ids, Tlen, mask, s_valid, red);
+    int hs[kMaxRK], khs[kMaxRK];
+    bool bad;
+    const int rk = group_heads(kept_heads + (size_t)b * k_h, k_h, Hq / Hk, g, Hq, hs, khs, bad);
+    if (bad && threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+    if (rk == 0) return;
+    if (Tv == 0) {  // no modality present: zero rows, flag
+        for (int hh = 0; hh < rk; ++hh) {
+            uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D);
+            for (int i = threadIdx.x; i < Tlen * S::CPR; i += blockDim.x) dst[i] = make_uint4(0, 0, 0, 0);
+            if (active_out != nullptr && active_in == nullptr)
+                for (int i = threadIdx.x; i < U_max; i += blockDim.x)
+                    active_out[((size_t)b * k_h + khs[hh]) * U_max + i] = -1;
+        }
+        if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_EMPTY_MASK);
+        return;
+    }
+    const int U = sentry_num_active(Tv, c);
+
+    // ---- stage the group's present K rows, then V rows (two copy groups), zero the padding
+    const __nv_bfloat16* Kg = K + ((size_t)b * Hk + g) * Tlen * D;
+    const __nv_bfloat16* Vg = V + ((size_t)b * Hk + g) * Tlen * D;
+    const int n_kt = (Tv + kKeyTile - 1) / kKeyTile;
+    const int rows_staged = n_kt * kKeyTile;
+    for (int i = threadIdx.x; i < rows_staged * S::CPR; i += blockDim.x) {
+        const int row = i / S::CPR, cc = i % S::CPR;
+        if (row < Tv) ptx::cp_async_16(ks_addr + S::off(row, cc), Kg + (size_t)s_valid[row] * D + cc * 8);
+        else asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(ks_addr + S::off(row, cc)), "r"(0) : "memory");
+    }
+    ptx::cp_async_commit();
+    for (int i = threadIdx.x; i < rows_staged * S::CPR; i += blockDim.x) {
+        const int row = i / S::CPR, cc = i % S::CPR;
+        if (row < Tv) ptx::cp_async_16(vs_addr + S::off(row, cc), Vg + (size_t)s_valid[row] * D + cc * 8);
+        else asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs_addr + S::off(row, cc)), "r"(0) : "memory");
+    }
+    ptx::cp_async_commit();
+
+    for (int t = threadIdx.x; t < Tlen; t += blockDim.x) s_kind[t] = 0;
+    for (int i = threadIdx.x; i < kMaxRK * words; i += blockDim.x) s_abits[i] = 0u;
+    for (int i = threadIdx.x; i < kMaxRK * kMaxActive; i += blockDim.x) (&s_act[0][0])[i] = -1;
+    __syncthreads();
+    for (int p = threadIdx.x; p < Tv; p += blockDim.x) s_kind[s_valid[p]] = 1;
+
+    if (active_in == nullptr) {
+        // ---- sparsity scores (Section 4.4) from the resident K rows
+        const int n_s = U;
+        const int cnt = score_mode == 0 ? n_s : Tv;
+        const int32_t* tbl = nullptr;
+        bool table_ok = true;
+        if (score_mode == 0) {
+            if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) table_ok = false;
+            else tbl = table + offsets[mask];
+        }
+        ptx::cp_async_wait_group<1>();   // K has landed (V may still be in flight)
+        __syncthreads();
+        if (table_ok) {
+            constexpr int HPP = (D == 64) ? 1 : 2;   // heads per pass: q rows live in registers
+            for (int h0 = 0; h0 < rk; h0 += HPP) {
+                const int nh = min(HPP, rk - h0);
+                size_t q_base[2];
+                uint32_t* keys_out[2];
+                for (int j = 0; j < 2; ++j) {
+                    const int hh = min(h0 + j, rk - 1);
+                    q_base[j] = ((size_t)b * Hq + hs[hh]) * Tlen * D;
+                    keys_out[j] = s_keys + (size_t)hh * Tlen;
+                }
+                if (HPP == 2 && nh == 2)
+                    fused_score_pass<D, (D == 64 ? 1 : 2)>(Q, 0, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+                else
+                    fused_score_pass<D, 1>(Q, 0, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+            }
+        } else {
+            if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+            for (int i = threadIdx.x; i < rk * Tlen; i += blockDim.x) s_keys[i] = 0u;
+        }
+        __syncthreads();
+        // ---- the U present queries with the largest score are active: one warp per head
+        if (warp < rk) warp_select_topk_radix(s_keys + (size_t)warp * Tlen, Tv, U, s_act[warp], s_valid, s_hist + warp * 256);
+        __syncthreads();
+        if (active_out != nullptr)
+            for (int i = threadIdx.x; i < rk * U_max; i += blockDim.x) {
+                const int hh = i / U_max, a = i % U_max;
+                active_out[((size_t)b * k_h + khs[hh]) * U_max + a] = a < U ? s_act[hh][a] : -1;
+            }
+    } else {
+        __syncthreads();
+        for (int i = threadIdx.x; i < rk * kMaxActive; i += blockDim.x) {
+            const int hh = i / kMaxActive, a = i % kMaxActive;
+            int t = a < U_max ? active_in[((size_t)b * k_h + khs[hh]) * U_max + a] : -1;
+            if (t >= 0 && (t >= Tlen || s_kind[t] == 0)) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); t = -1; }
+            s_act[hh][a] = t;
+        }
+        __syncthreads();
+    }
+    for (int i = threadIdx.x; i < rk * kMaxActive; i += blockDim.x) {
+        const int hh = i / kMaxActive, t = s_act[hh][i % kMaxActive];
+        if (t >= 0) atomicOr(&s_abits[hh * words + (t >> 5)], 1u << (t & 31));
+    }
+    ptx::cp_async_wait_group<0>();       // V has landed
+    __syncthreads();
+
+    // ---- context vector = mean of V_g over the present keys (padding rows are zero)
+    {
+        constexpr int DP = D / 2;
+        const int vs_dp = threadIdx.x % DP, vs_k0 = threadIdx.x / DP;
+        const int stride = blockDim.x / DP;
+        float v0 = 0.f, v1 = 0.f;
+        for (int row = vs_k0; row < rows_staged; row += stride) {
+            uint32_t w;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(vs_addr + S::off(row, vs_dp >> 2) + (vs_dp & 3) * 4));
+            v0 += __uint_as_float(w << 16);
+            v1 += __uint_as_float(w & 0xffff0000u);
+        }
+        s_vpart[vs_k0][2 * vs_dp] = v0;
+        s_vpart[vs_k0][2 * vs_dp + 1] = v1;
+        __syncthreads();
+        if (threadIdx.x < D) {
+            float t = 0.f;
+            for (int i = 0; i < stride; ++i) t += s_vpart[i][threadIdx.x];
+            s_mean[threadIdx.x] = __float2bfloat16_rn(t / (float)Tv);
+        }
+    }
+
+    // ---- Eq. 6 on the active rows: row tiles (head slot, 16 rows) over the warps
+    const int WT = (min(U, kMaxActive) + 15) / 16;
+    const int n_tiles = rk * WT;
+    const int gq = lane >> 2, tq = lane & 3;
+    const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;  // scale * log2(e)
+    for (int tt = warp; tt < n_tiles; tt += nwarps) {
+        const int hh = tt / WT, row0 = (tt % WT) * 16;
+        uint32_t qf[KS][4];
+        float acc[NT][4];
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[n][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) qf[ks][e] = 0u;
+        const __nv_bfloat16* Qh = Q + ((size_t)b * Hq + hs[hh]) * Tlen * D;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int a = row0 + gq + half * 8;
+            const int t = a < kMaxActive ? s_act[hh][a] : -1;
+            if (t >= 0) {
+                const uint32_t* qrow = reinterpret_cast<const uint32_t*>(Qh + (size_t)t * D);
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    qf[ks][half] = __ldg(qrow + ks * 8 + tq);          // cols 16ks + 2t, +1
+                    qf[ks][half + 2] = __ldg(qrow + ks * 8 + 4 + tq);  // cols 16ks + 8 + 2t, +1
+                }
+            }
+        }
+        for (int kt = 0; kt < n_kt; ++kt) {
+            const uint32_t kbase = ks_addr + kt * TILE_BYTES;
+            const uint32_t vbase = vs_addr + kt * TILE_BYTES;
+            const int key0 = kt * kKeyTile;
+            float sc[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
+                const int krow = nt * 8 + (lane & 7);
+                if constexpr (D == 32) {
+                    uint32_t bfr[4];
+                    ldmatrix_x4(kbase + S::off(krow, lane >> 3), bfr);
+                    mma_bf16_16816(sc[nt], qf[0], bfr[0], bfr[1]);
+                    mma_bf16_16816(sc[nt], qf[1], bfr[2], bfr[3]);
+                } else if constexpr (D == 16) {
+                    uint32_t bfr[2];
+                    ldmatrix_x2(kbase + S::off(krow, (lane >> 3) & 1), bfr);
+                    mma_bf16_16816(sc[nt], qf[0], bfr[0], bfr[1]);
+                } else {
+                    uint32_t bfr[4];
+                    ldmatrix_x4(kbase + S::off(krow, lane >> 3), bfr);
+                    mma_bf16_16816(sc[nt], qf[0], bfr[0], bfr[1]);
+                    mma_bf16_16816(sc[nt], qf[1], bfr[2], bfr[3]);
+                    ldmatrix_x4(kbase + S::off(krow, 4 + (lane >> 3)), bfr);
+                    mma_bf16_16816(sc[nt], qf[2], bfr[0], bfr[1]);
+                    mma_bf16_16816(sc[nt], qf[3], bfr[2], bfr[3]);
+                }
+            }
+            float mt[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int key = key0 + nt * 8 + tq * 2 + (e & 1);
+                    sc[nt][e] = key < Tv ? sc[nt][e] * sl2 : -INFINITY;
+                    mt[e >> 1] = fmaxf(mt[e >> 1], sc[nt][e]);
+                }
+            float corr[2];
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+                mt[h2] = fmaxf(mt[h2], __shfl_xor_sync(0xffffffffu, mt[h2], 1));
+                mt[h2] = fmaxf(mt[h2], __shfl_xor_sync(0xffffffffu, mt[h2], 2));
+                const float m_new = fmaxf(m_run[h2], mt[h2]);
+                corr[h2] = fast_exp2(m_run[h2] - m_new);   // 0 on the first tile
+                m_run[h2] = m_new;
+                l_run[h2] *= corr[h2];
+            }
+            float lsum[2] = {0.f, 0.f};
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    sc[nt][e] = fast_exp2(sc[nt][e] - m_run[e >> 1]);
+                    lsum[e >> 1] += sc[nt][e];
+                }
+            l_run[0] += lsum[0];
+            l_run[1] += lsum[1];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                acc[n][0] *= corr[0]; acc[n][1] *= corr[0];
+                acc[n][2] *= corr[1]; acc[n][3] *= corr[1];
+            }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t pa[4];
+                pa[0] = pack2(sc[2 * ks][0], sc[2 * ks][1]);
+                pa[1] = pack2(sc[2 * ks][2], sc[2 * ks][3]);
+                pa[2] = pack2(sc[2 * ks + 1][0], sc[2 * ks + 1][1]);
+                pa[3] = pack2(sc[2 * ks + 1][2], sc[2 * ks + 1][3]);
+                const int vrow = ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                for (int n2 = 0; n2 < NT / 2; ++n2) {
+                    uint32_t bfr[4];
+                    ldmatrix_x4_trans(vbase + S::off(vrow, 2 * n2 + (lane >> 4)), bfr);
+                    mma_bf16_16816(acc[2 * n2], pa, bfr[0], bfr[1]);
+                    mma_bf16_16816(acc[2 * n2 + 1], pa, bfr[2], bfr[3]);
+                }
+            }
+        }
+        // normalise and store this tile's rows
+        __nv_bfloat16* Oh = O + ((size_t)b * k_h + khs[hh]) * Tlen * D;
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+            float l = l_run[h2];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int a = row0 + gq + h2 * 8;
+            const int t = a < kMaxActive ? s_act[hh][a] : -1;
+            if (t < 0) continue;
+            const float inv = 1.0f / l;
+            uint32_t* orow = reinterpret_cast<uint32_t*>(Oh + (size_t)t * D);
+#pragma unroll
+            for (int n = 0; n < NT; ++n)
+                orow[n * 4 + tq] = pack2(acc[n][2 * h2] * inv, acc[n][2 * h2 + 1] * inv);
+        }
+    }
+    __syncthreads();   // s_mean is complete
+    // ---- context rows and zero rows, 16 bytes per store
+    const uint4* mean4 = reinterpret_cast<const uint4*>(s_mean);
+    for (int hh = 0; hh < rk; ++hh) {
+        uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D);
+        const uint32_t* bits = s_abits + hh * words;
+        for (int i = threadIdx.x; i < Tlen * S::CPR; i += blockDim.x) {
+            const int t = i / S::CPR, cc = i % S::CPR;
+            if ((bits[t >> 5] >> (t & 31)) & 1u) continue;
+            dst[i] = s_kind[t] ? mean4[cc] : make_uint4(0, 0, 0, 0);
+        }
+    }
+}
+
+template <int D>
+size_t fused_smem_bytes(int T) {
+    const int words = (T + 31) / 32;
+    const int Tpad = (T + kKeyTile - 1) / kKeyTile * kKeyTile;
+    size_t o = (((size_t)T * 2 + 127) / 128) * 128 + (((size_t)T + 127) / 128) * 128 +
+               (((size_t)kMaxRK * words * 4 + 127) / 128) * 128 + (((size_t)kMaxRK * T * 4 + 127) / 128) * 128 +
+               (size_t)kMaxRK * 256 * 4;
+    return o + 2 * (size_t)Tpad * D * 2;
+}
+
 template <int D>
 int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
     const sentry_attend_desc& d = a.d;
+    const size_t fused_bytes = fused_smem_bytes<D>(d.T);
+    if (fused_bytes <= 200 * 1024) {
+        // the group's K and V fit in shared memory: one kernel does everything
+        auto kern = attend_fused_bf16_kernel<D>;
+        SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused_bytes));
+        const int threads = fused_bytes > 100 * 1024 ? 512 : 256;   // one big CTA or two per SM
+        LaunchScope ls(ctx, KS_ATT_CORE, st);
+        kern<<<d.B * d.Hk, threads, fused_bytes, st>>>(
+            (const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, a.kept_heads,
+            a.ids, a.masks, a.sample_table, a.sample_offsets, a.n_subsets,
+            a.selection_given ? a.active : nullptr, a.selection_given ? nullptr : a.active_out_user, d.T,
+            d.Hq, d.Hk, d.k_h, d.c, d.score_mode, a.U_max, (__nv_bfloat16*)a.O, a.status);
+        SENTRY_CUDA_TRY(cudaGetLastError());
+        return SENTRY_OK;
+    }
     const size_t valid_bytes = (((size_t)d.T * 2 + 127) / 128) * 128;
     if (!a.selection_given) {
         // K segment: as many rows as fit in ~64 KB (one pass for T <= 1024 at d = 32)
