@@ -134,6 +134,56 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
         return;
     }
     pb -= zero_blocks;
+    if (layout == 1) {
+        // K-major copies for the tensor-core kernel, one 32-channel x 64-column tile per block,
+        // transposed through shared memory so that both the gather and the store touch whole
+        // sectors:  W1c[l][n][e] = W1[e][N[n]],  W2c[l][e][n] = W2[N[n]][e].
+        __shared__ T s_tile[64][33];
+        __shared__ int s_ch[32];
+        const int tiles_n = kc_pad / 32, tiles_e = D / 64;
+        const size_t per_list = (size_t)tiles_n * tiles_e;
+        const int which = (int)(pb / (per_list * n_lists));
+        pb -= (size_t)which * per_list * n_lists;
+        const int l = (int)(pb / per_list);
+        const int tn = (int)((pb % per_list) / tiles_e), te = (int)(pb % tiles_e);
+        const int n0 = tn * 32, e0 = te * 64;
+        const int tx = threadIdx.x & 31, wy = threadIdx.x >> 5;   // 8 warps
+        if (threadIdx.x < 32) {
+            const int n = n0 + threadIdx.x;
+            int ch = -1;
+            if (n < k_c) {
+                ch = kept[(size_t)l * k_c + n];
+                if (ch < 0 || ch >= F) {
+                    if (which == 0 && te == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+                    ch = -1;
+                }
+            }
+            s_ch[threadIdx.x] = ch;
+        }
+        __syncthreads();
+        const T zero = from_f32<T>(0.f);
+        if (which == 0) {
+            const int ch = s_ch[tx];
+            for (int ee = wy; ee < 64; ee += 8)
+                s_tile[ee][tx] = ch >= 0 ? W1[(size_t)(e0 + ee) * F + ch] : zero;
+            __syncthreads();
+            T* dst = out1 + ((size_t)l * kc_pad + n0) * D + e0;
+            for (int nn = wy; nn < 32; nn += 8) {
+                dst[(size_t)nn * D + tx] = s_tile[tx][nn];
+                dst[(size_t)nn * D + 32 + tx] = s_tile[32 + tx][nn];
+            }
+        } else {
+            for (int nn = wy; nn < 32; nn += 8) {
+                const int ch = s_ch[nn];
+                s_tile[tx][nn] = ch >= 0 ? W2[(size_t)ch * D + e0 + tx] : zero;
+                s_tile[32 + tx][nn] = ch >= 0 ? W2[(size_t)ch * D + e0 + 32 + tx] : zero;
+            }
+            __syncthreads();
+            T* dst = out2 + ((size_t)l * D + e0) * kc_pad + n0;
+            for (int ee = wy; ee < 64; ee += 8) dst[(size_t)ee * kc_pad + tx] = s_tile[ee][tx];
+        }
+        return;
+    }
     const size_t per = (size_t)kc_pad * D;
     const size_t blocks_per = (per + 255) / 256;
     const int which = (int)(pb / (blocks_per * n_lists));
@@ -288,8 +338,9 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cud
         int zsplit = (4 * ctx->sm_count + d.B - 1) / d.B;
         if (zsplit < 1) zsplit = 1;
         if (zsplit > 32) zsplit = 32;
-        const size_t grid = (size_t)d.B + (a.ids != nullptr ? (size_t)d.B * zsplit : 0) +
-                            2 * (size_t)d.n_lists * ((per + 255) / 256);
+        const size_t pack_blocks = tc ? 2 * (size_t)d.n_lists * (kc_pad / 32) * (d.D / 64)
+                                      : 2 * (size_t)d.n_lists * ((per + 255) / 256);
+        const size_t grid = (size_t)d.B + (a.ids != nullptr ? (size_t)d.B * zsplit : 0) + pack_blocks;
         LaunchScope ls(ctx, KS_FFN_PREPARE, st);
         if (d.dtype == SENTRY_F32)
             ffn_prepare_kernel<float><<<(unsigned)grid, 256, 0, st>>>(

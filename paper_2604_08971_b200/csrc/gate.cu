@@ -16,11 +16,15 @@ inline int gate_threads(int n_units) {
     return t < 64 ? 64 : (t > kGateMaxThreads ? kGateMaxThreads : t);
 }
 
-// One block per score-table row s: rows[s, 0..k) and groups[s].
+// One block per score-table row s: rows[s, 0..k) and groups[s].  With fan_masks given (a small
+// fan-out), the block also copies its row to every sample whose mask selects it, which saves
+// the second launch: kept[m, :] = rows[s, :] for masks[m] == s.
 __global__ void __launch_bounds__(kGateMaxThreads)
 gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
                  int32_t* __restrict__ rows, uint32_t* __restrict__ groups,
-                 int heads_per_group) {
+                 int heads_per_group, const uint32_t* __restrict__ fan_masks = nullptr,
+                 int n_masks = 0, int S = 0, int32_t* __restrict__ kept = nullptr,
+                 uint32_t* __restrict__ kv_groups = nullptr, unsigned int* status = nullptr) {
     extern __shared__ uint32_t s_keys[];
     __shared__ int red[66];
     __shared__ uint32_t s_bits;
@@ -39,6 +43,19 @@ gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
         if ((threadIdx.x & 31) == 0 && bits) atomicOr(&s_bits, bits);
         __syncthreads();
         if (threadIdx.x == 0) groups[s] = s_bits;
+    }
+    if (fan_masks == nullptr) return;
+    __syncthreads();   // out[] (global, written by this block) is complete
+    const long long total = (long long)n_masks * k;
+    for (long long i = threadIdx.x; i < total; i += blockDim.x) {
+        const int m = (int)(i / k), j = (int)(i % k);
+        const uint32_t ms = fan_masks[m];
+        if (ms == (uint32_t)s) {
+            kept[i] = out[j];
+            if (j == 0 && kv_groups != nullptr) kv_groups[m] = s_bits;
+        } else if (s == 0 && j == 0 && ms >= (uint32_t)S) {
+            atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+        }
     }
 }
 
@@ -72,6 +89,15 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
     if (smem > 48 * 1024)
         SENTRY_CUDA_TRY(cudaFuncSetAttribute(gate_rows_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const size_t total = (size_t)n_masks * k;
+    if (total <= 16384) {   // small fan-out: one launch does both steps
+        LaunchScope ls(ctx, KS_GATE_ROWS, st);
+        gate_rows_kernel<<<S, gate_threads(n_units), smem, st>>>(
+            scores, n_units, k, ws_rows, kv_groups ? ws_groups : nullptr,
+            heads_per_group > 0 ? heads_per_group : 1, masks, n_masks, S, kept, kv_groups, ctx->d_status);
+        SENTRY_CUDA_TRY(cudaGetLastError());
+        return SENTRY_OK;
+    }
     {
         LaunchScope ls(ctx, KS_GATE_ROWS, st);
         gate_rows_kernel<<<S, gate_threads(n_units), smem, st>>>(scores, n_units, k, ws_rows,
@@ -79,7 +105,6 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                                                          heads_per_group > 0 ? heads_per_group : 1);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
-    const size_t total = (size_t)n_masks * k;
     int blocks = (int)((total + 255) / 256);
     const int cap = ctx->sm_count * 8;
     if (blocks > cap) blocks = cap;
