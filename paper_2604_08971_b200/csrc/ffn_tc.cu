@@ -116,6 +116,18 @@ __device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uin
         ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
 }
 
+// K=16 steps ks0 .. ks1-1 of a 64-wide K block (the stage's last step is issued after the
+// issuer has looked at the next stage's barrier, see below).
+__device__ __forceinline__ void mma_ksteps(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr,
+                                           uint32_t idesc, bool overwrite, uint32_t ks0, uint32_t ks1) {
+    const uint64_t ad = ptx::umma_smem_desc_sw128(a_addr);
+    const uint64_t bd = ptx::umma_smem_desc_sw128(b_addr);
+#pragma unroll
+    for (uint32_t ks = 0; ks < 4; ++ks)
+        if (ks >= ks0 && ks < ks1)
+            ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
+}
+
 // One lane of a fully converged warp.  The single-thread instructions (TMA, UMMA, commit) are
 // issued from inside `if (elect_one())` while the whole warp walks the schedule: operands
 // computed by all lanes stay warp-uniform, which about halves the cost of issuing them
@@ -245,12 +257,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------------------------- UMMA issuer
         // The whole warp walks the schedule and waits; one elected lane issues the UMMAs and
-        // their commits (a commit tracks the UMMAs of the thread that issues it).
+        // their commits (a commit tracks the UMMAs of the thread that issues it).  The tensor
+        // pipe queues only a few instructions, so the barrier of the NEXT weight stage is waited
+        // for before the current stage's last UMMA is issued: the wait then overlaps queued work
+        // instead of draining the pipe.
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
         const uint32_t tm_h = tmem + C::H_COL0;
         uint32_t n = 0;   // weight stages consumed
-        bool ok = true;
+        bool ok = true, peeked = false;
         auto wait = [&](uint64_t* bar, uint32_t parity) {
             if (ok) ok = warp_wait(bar, parity, abort_flag);
             return ok;
@@ -260,7 +275,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             ptx::tc_fence_after_sync();
             return r;
         };
-        auto stage_wait = [&]() { return wait(&misc->w_full[n % kStages], (n / kStages) & 1u); };
+        auto stage_wait = [&]() {
+            if (peeked) { peeked = false; return ok; }
+            return wait(&misc->w_full[n % kStages], (n / kStages) & 1u);
+        };
+        auto peek_next = [&](bool more) {   // stage n+1 (if there is one) has landed
+            if (more && wait(&misc->w_full[(n + 1) % kStages], ((n + 1) / kStages) & 1u)) peeked = true;
+            return ok;
+        };
         auto bar_of = [&](uint64_t* b) { return ptx::smem_u32(b); };
         // GEMM1 of global chunk g = chunk c of local tile ti:  H = X . W1c_chunk^T
         auto gemm1 = [&](uint32_t g, int c, uint32_t ti) {
@@ -275,7 +297,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (elect_one()) {
                         mma_kblock(tm_h, xs + s0 * kBlockBytes, b, idesc128, kp == 0);
                         if (last) ptx::umma_commit(bar_of(&misc->x_empty[s0]));
-                        mma_kblock(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false);
+                        mma_ksteps(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false, 0, 3);
+                    }
+                    __syncwarp();
+                    if (!peek_next(true)) return;
+                    if (elect_one()) {
+                        mma_ksteps(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false, 3, 4);
                         if (last) ptx::umma_commit(bar_of(&misc->x_empty[s1]));
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         if (kp == 2) ptx::umma_commit(bar_of(&misc->h_full));
@@ -289,8 +316,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (c == 0 && !wait(&misc->x_full[slot], (gx / C::NXS) & 1u)) return;
                     if (!stage_wait()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) mma_ksteps(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0, 0, 3);
+                    __syncwarp();
+                    if (!peek_next(true)) return;
                     if (elect_one()) {
-                        mma_kblock(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0);
+                        mma_ksteps(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0, 3, 4);
                         if (last) ptx::umma_commit(bar_of(&misc->x_empty[slot]));
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         if (kb == C::KB1 - 1) ptx::umma_commit(bar_of(&misc->h_full));
@@ -300,8 +330,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 }
             }
         };
-        // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk
-        auto gemm2 = [&](uint32_t g, int c, uint32_t ti) {
+        // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk   (`final`: nothing follows it)
+        auto gemm2 = [&](uint32_t g, int c, uint32_t ti, bool final) {
             const bool first = (c == 0), last = (c == NC - 1);
             if constexpr (D == 256) {
                 for (int kb2 = 0; kb2 < 4; ++kb2) {
@@ -309,8 +339,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
                     if (!stage_wait()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 0, 3);
+                    __syncwarp();
+                    if (!peek_next(!(final && kb2 == 3))) return;
                     if (elect_one()) {
-                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 3, 4);
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         ptx::umma_commit(bar_of(&misc->hs_empty[kb2]));
                         if (last && kb2 == 3) ptx::umma_commit(bar_of(&misc->y_full));
@@ -328,7 +361,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (elect_one()) {
                         mma_kblock(tmem, hs + k0 * kBlockBytes, b, idesc128, first && kp == 0);
                         ptx::umma_commit(bar_of(&misc->hs_empty[k0]));
-                        mma_kblock(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false);
+                        mma_ksteps(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false, 0, 3);
+                    }
+                    __syncwarp();
+                    if (!peek_next(!(final && kp == 1))) return;
+                    if (elect_one()) {
+                        mma_ksteps(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false, 3, 4);
                         ptx::umma_commit(bar_of(&misc->hs_empty[k1]));
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         if (last && kp == 1) ptx::umma_commit(bar_of(&misc->y_full));
@@ -343,8 +381,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
                     if (!stage_wait()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
+                    if (elect_one()) mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 0, 3);
+                    __syncwarp();
+                    if (!peek_next(true)) return;
                     if (elect_one()) {
-                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 3, 4);
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                     }
                     __syncwarp();
@@ -354,7 +395,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 const uint32_t b = wsm + (n % kStages) * kStageBytes;
                 if (elect_one()) {
                     mma_kblock(tmem + 256, hs, b, idesc128, first);
-                    mma_kblock(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false);
+                    mma_ksteps(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false, 0, 3);
+                }
+                __syncwarp();
+                if (!peek_next(!final)) return;
+                if (elect_one()) {
+                    mma_ksteps(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false, 3, 4);
                     ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                     ptx::umma_commit(bar_of(&misc->hs_empty[0]));
                     ptx::umma_commit(bar_of(&misc->hs_empty[1]));
@@ -371,12 +417,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
             for (int c = 0; c < NC && ok; ++c, ++g) {
                 gemm1(g, c, ti);
-                if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
+                if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti, false);
                 have_prev = true;
                 prev_g = g; prev_c = c; prev_ti = ti;
             }
         }
-        if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
+        if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti, true);
     } else if (warp < kEpiWarp0) {
         // ------------------------------------------------------------------ X row gather
         // Thread -> 8 (row, 16-byte chunk) pairs of every 128 x 64 block.  Up to three blocks
