@@ -145,7 +145,7 @@ def test_config4_full_layer_all_subsets(sn):
 
 
 @pytest.mark.parametrize("B,T", [(1, 64), (16, 64), (16, 256), (1, 1024), (16, 1024), (1, 4096),
-                                 (256, 256), (14, 4096)])
+                                 (256, 256), (14, 4096), (256, 1024), (4096, 64)])
 def test_config5_sweep_cells(sn, B, T):
     _run_workload(sn, synth.config5(B, T), "strat", "strat")
 
