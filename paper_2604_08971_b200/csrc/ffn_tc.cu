@@ -19,9 +19,9 @@
 // next chunk (or of the next tile's first chunk) before GEMM2 of the current one, so GEMM2
 // never waits for the GELU epilogue with nothing else queued.
 //
-// Warp roles (480 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
-// warp 1 = UMMA issuer, warps 3-6 = X row gather, warps 7-14 = epilogue (two warps per TMEM
-// lane quarter).  Producer and issuer warps stay converged and elect one lane per instruction.  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
+// Warp roles (512 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
+// warps 1 and 15 = UMMA issuers (alternate stages), warps 3-6 = X row gather, warps 7-14 =
+// epilogue (two warps per TMEM lane quarter).  Producer and issuer warps stay converged and elect one lane per instruction.  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
 // and unwinds.
 #include <cuda.h>
 #include <math.h>
@@ -36,9 +36,10 @@ constexpr int kTileRows = 128;
 constexpr int kBlockBytes = 128 * 128;   // 128 rows x 64 bf16: one X block, one hidden block
 constexpr int kStageBytes = 2 * kBlockBytes;
 constexpr int kStages = 3;
-constexpr int kThreads = 480;
+constexpr int kThreads = 512;
 constexpr int kLoaderWarp0 = 3, kLoaderWarps = 4, kLoaderThreads = kLoaderWarps * 32;
 constexpr int kEpiWarp0 = 7, kEpiWarps = 8;
+constexpr int kIssuerB = 15;   // second UMMA issuer warp (the first is warp 1)
 constexpr int kTmemCols = 512;
 
 template <int D>
@@ -64,6 +65,7 @@ struct Misc {
     uint64_t y_full, y_empty;
     uint32_t tmem_base;
     int abort_flag;
+    uint32_t issued;   // weight stages whose UMMAs have been issued (turn counter of the two issuers)
 };
 static_assert(sizeof(Misc) <= 2048, "misc block too large");
 
@@ -72,15 +74,40 @@ static_assert(sizeof(Misc) <= 2048, "misc block too large");
 // (weighted least squares pushed towards minimax on |z| <= 4 sqrt 2, where erfc is below 2e-8;
 // beyond, |z| is clamped).  Largest error of gelu over all z: 7e-7, far below the resolution
 // of the bf16 value that is stored.  One special-function operation per element.
-__device__ __forceinline__ float gelu_erf_fast(float z) {
-    const float a = fminf(fabsf(z), 5.65685424949f);
-    float p = fmaf(4.880980979e-04f, a, -7.198737003e-03f);   // c4/4sqrt2, c3/4
-    p = fmaf(p, a, 5.214667618e-02f);                         // c2 / 2 sqrt 2
-    p = fmaf(p, a, 4.595957994e-01f);                         // c1 / 2
-    p = fmaf(p, a, 1.151000593e+00f);                         // c0 / sqrt 2
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(-(p * a)));
-    return fmaf(-0.5f * fabsf(z), y, fmaxf(z, 0.0f));
+// Coefficients of the quartic, highest power first: 4.880980979e-04, -7.198737003e-03,
+// 5.214667618e-02, 4.595957994e-01, 1.151000593e+00.
+// Evaluated on two values at once with the packed fp32 instructions of sm_100 (two lanes of a
+// 64-bit register per instruction), result rounded to a bf16 pair: 7 instead of 11 issue slots
+// per element, which matters because the GELU epilogue competes with the UMMA issuers for them.
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t gelu_erf_fast_bf16x2(float z0, float z1) {
+    const float a0 = fminf(fabsf(z0), 5.65685424949f), a1 = fminf(fabsf(z1), 5.65685424949f);
+    const uint64_t A = f32x2(a0, a1);
+    uint64_t P = fma_f32x2(f32x2(4.880980979e-04f, 4.880980979e-04f), A, f32x2(-7.198737003e-03f, -7.198737003e-03f));
+    P = fma_f32x2(P, A, f32x2(5.214667618e-02f, 5.214667618e-02f));
+    P = fma_f32x2(P, A, f32x2(4.595957994e-01f, 4.595957994e-01f));
+    P = fma_f32x2(P, A, f32x2(1.151000593e+00f, 1.151000593e+00f));
+    const uint64_t Qn = fma_f32x2(P, A, f32x2(0.f, 0.f));            // q = p * a
+    float q0, q1, y0, y1;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(q0), "=f"(q1) : "l"(Qn));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y0) : "f"(-q0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y1) : "f"(-q1));
+    // relu(z) - (a/2) * erfc: beyond the clamp erfc < 2e-8, so a stands in for |z|
+    const uint64_t H = fma_f32x2(A, f32x2(-0.5f, -0.5f), f32x2(0.f, 0.f));
+    const uint64_t G = fma_f32x2(H, f32x2(y0, y1), f32x2(fmaxf(z0, 0.0f), fmaxf(z1, 0.0f)));
+    float g0, g1;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(g0), "=f"(g1) : "l"(G));
+    __nv_bfloat162 v = __floats2bfloat162_rn(g0, g1);
+    return *reinterpret_cast<uint32_t*>(&v);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
@@ -114,18 +141,6 @@ __device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uin
 #pragma unroll
     for (uint32_t ks = 0; ks < 4; ++ks)
         ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
-}
-
-// K=16 steps ks0 .. ks1-1 of a 64-wide K block (the stage's last step is issued after the
-// issuer has looked at the next stage's barrier, see below).
-__device__ __forceinline__ void mma_ksteps(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr,
-                                           uint32_t idesc, bool overwrite, uint32_t ks0, uint32_t ks1) {
-    const uint64_t ad = ptx::umma_smem_desc_sw128(a_addr);
-    const uint64_t bd = ptx::umma_smem_desc_sw128(b_addr);
-#pragma unroll
-    for (uint32_t ks = 0; ks < 4; ++ks)
-        if (ks >= ks0 && ks < ks1)
-            ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
 }
 
 // One lane of a fully converged warp.  The single-thread instructions (TMA, UMMA, commit) are
@@ -180,6 +195,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         ptx::mbar_init(ptx::smem_u32(&misc->y_full), 1);
         ptx::mbar_init(ptx::smem_u32(&misc->y_empty), kEpiWarps);
         misc->abort_flag = 0;
+        misc->issued = 0;
         ptx::fence_barrier_init();
     }
     if (warp == 0) {
@@ -254,18 +270,23 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             }
         }
         if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------- UMMA issuer
-        // The whole warp walks the schedule and waits; one elected lane issues the UMMAs and
-        // their commits (a commit tracks the UMMAs of the thread that issues it).  The tensor
-        // pipe queues only a few instructions, so the barrier of the NEXT weight stage is waited
-        // for before the current stage's last UMMA is issued: the wait then overlaps queued work
-        // instead of draining the pipe.
+    } else if (warp == 1 || warp == kIssuerB) {
+        // ------------------------------------------------------------------ UMMA issuers
+        // Two warps take the weight stages of the schedule in turn (even / odd stage index).
+        // Each walks the whole schedule converged, waits for its own stage's operands, then for
+        // its turn (all earlier stages issued: the tensor pipe executes in issue order), and
+        // one elected lane issues the stage's UMMAs and commits (a commit tracks the UMMAs of the
+        // thread that issues it; since the pipe is in order, a commit after the last stage of a
+        // GEMM also covers the other issuer's earlier stages).  While one issuer is blocked
+        // issuing into the short UMMA queue, the other does its waiting and bookkeeping, so the
+        // queue does not run dry between stages.
+        const uint32_t me = (warp == 1) ? 0u : 1u;
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
         const uint32_t tm_h = tmem + C::H_COL0;
-        uint32_t n = 0;   // weight stages consumed
-        bool ok = true, peeked = false;
+        volatile uint32_t* issued = &misc->issued;
+        uint32_t n = 0;   // weight stages walked
+        bool ok = true;
         auto wait = [&](uint64_t* bar, uint32_t parity) {
             if (ok) ok = warp_wait(bar, parity, abort_flag);
             return ok;
@@ -275,139 +296,127 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             ptx::tc_fence_after_sync();
             return r;
         };
-        auto stage_wait = [&]() {
-            if (peeked) { peeked = false; return ok; }
-            return wait(&misc->w_full[n % kStages], (n / kStages) & 1u);
-        };
-        auto peek_next = [&](bool more) {   // stage n+1 (if there is one) has landed
-            if (more && wait(&misc->w_full[(n + 1) % kStages], ((n + 1) / kStages) & 1u)) peeked = true;
-            return ok;
+        // this stage's weights have landed and every earlier stage has been issued
+        auto stage_ready = [&]() {
+            if (!wait(&misc->w_full[n % kStages], (n / kStages) & 1u)) return false;
+            for (uint32_t spins = 0; !__all_sync(0xffffffffu, *issued >= n); ++spins) {
+                if (spins > (1u << 22) || *abort_flag) { *abort_flag = 1; ok = false; return false; }
+            }
+            return true;
         };
         auto bar_of = [&](uint64_t* b) { return ptx::smem_u32(b); };
         // GEMM1 of global chunk g = chunk c of local tile ti:  H = X . W1c_chunk^T
         auto gemm1 = [&](uint32_t g, int c, uint32_t ti) {
-            if (!wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
             const bool last = (c == NC - 1);
             if constexpr (D == 384) {
-                for (int kp = 0; kp < 3; ++kp) {
+                for (int kp = 0; kp < 3 && ok; ++kp, ++n) {
+                    if ((n & 1u) != me) continue;
+                    if (kp == 0 && !wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
                     const uint32_t s0 = 2 * kp, s1 = 2 * kp + 1;   // X slots (NXS = KB1 = 6)
                     if (c == 0 && (!wait(&misc->x_full[s0], ti & 1u) || !wait(&misc->x_full[s1], ti & 1u))) return;
-                    if (!stage_wait()) return;
+                    if (!stage_ready()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
                     if (elect_one()) {
                         mma_kblock(tm_h, xs + s0 * kBlockBytes, b, idesc128, kp == 0);
-                        if (last) ptx::umma_commit(bar_of(&misc->x_empty[s0]));
-                        mma_ksteps(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false, 0, 3);
-                    }
-                    __syncwarp();
-                    if (!peek_next(true)) return;
-                    if (elect_one()) {
-                        mma_ksteps(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false, 3, 4);
-                        if (last) ptx::umma_commit(bar_of(&misc->x_empty[s1]));
+                        mma_kblock(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false);
+                        *issued = n + 1;
+                        if (last) {
+                            ptx::umma_commit(bar_of(&misc->x_empty[s0]));
+                            ptx::umma_commit(bar_of(&misc->x_empty[s1]));
+                        }
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         if (kp == 2) ptx::umma_commit(bar_of(&misc->h_full));
                     }
                     __syncwarp();
-                    ++n;
                 }
             } else {
-                for (int kb = 0; kb < C::KB1; ++kb) {
+                for (int kb = 0; kb < C::KB1 && ok; ++kb, ++n) {
+                    if ((n & 1u) != me) continue;
+                    if (kb == 0 && !wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
                     const uint32_t gx = ti * C::KB1 + kb, slot = gx % C::NXS;
                     if (c == 0 && !wait(&misc->x_full[slot], (gx / C::NXS) & 1u)) return;
-                    if (!stage_wait()) return;
+                    if (!stage_ready()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) mma_ksteps(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0, 0, 3);
-                    __syncwarp();
-                    if (!peek_next(true)) return;
                     if (elect_one()) {
-                        mma_ksteps(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0, 3, 4);
+                        mma_kblock(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0);
+                        *issued = n + 1;
                         if (last) ptx::umma_commit(bar_of(&misc->x_empty[slot]));
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         if (kb == C::KB1 - 1) ptx::umma_commit(bar_of(&misc->h_full));
                     }
                     __syncwarp();
-                    ++n;
                 }
             }
         };
-        // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk   (`final`: nothing follows it)
-        auto gemm2 = [&](uint32_t g, int c, uint32_t ti, bool final) {
+        // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk
+        auto gemm2 = [&](uint32_t g, int c, uint32_t ti) {
             const bool first = (c == 0), last = (c == NC - 1);
             if constexpr (D == 256) {
-                for (int kb2 = 0; kb2 < 4; ++kb2) {
+                for (int kb2 = 0; kb2 < 4 && ok; ++kb2, ++n) {
+                    if ((n & 1u) != me) continue;
                     if (!wait(&misc->hs_full[kb2], g & 1u)) return;
                     if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                    if (!stage_wait()) return;
+                    if (!stage_ready()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 0, 3);
-                    __syncwarp();
-                    if (!peek_next(!(final && kb2 == 3))) return;
                     if (elect_one()) {
-                        mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 3, 4);
+                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
+                        *issued = n + 1;
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         ptx::umma_commit(bar_of(&misc->hs_empty[kb2]));
                         if (last && kb2 == 3) ptx::umma_commit(bar_of(&misc->y_full));
                     }
                     __syncwarp();
-                    ++n;
                 }
             } else if constexpr (D == 128) {
-                for (int kp = 0; kp < 2; ++kp) {
+                for (int kp = 0; kp < 2 && ok; ++kp, ++n) {
+                    if ((n & 1u) != me) continue;
                     const int k0 = 2 * kp, k1 = 2 * kp + 1;
                     if (!wait(&misc->hs_full[k0], g & 1u) || !wait(&misc->hs_full[k1], g & 1u)) return;
                     if (first && kp == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                    if (!stage_wait()) return;
+                    if (!stage_ready()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
                     if (elect_one()) {
                         mma_kblock(tmem, hs + k0 * kBlockBytes, b, idesc128, first && kp == 0);
+                        mma_kblock(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false);
+                        *issued = n + 1;
                         ptx::umma_commit(bar_of(&misc->hs_empty[k0]));
-                        mma_ksteps(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false, 0, 3);
-                    }
-                    __syncwarp();
-                    if (!peek_next(!(final && kp == 1))) return;
-                    if (elect_one()) {
-                        mma_ksteps(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false, 3, 4);
                         ptx::umma_commit(bar_of(&misc->hs_empty[k1]));
                         ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
                         if (last && kp == 1) ptx::umma_commit(bar_of(&misc->y_full));
                     }
                     __syncwarp();
-                    ++n;
                 }
             } else {
                 // columns 0..255 of Y from two N=256 stages, columns 256..383 from one N=128 stage
-                for (int kb2 = 0; kb2 < 2; ++kb2) {
-                    if (!wait(&misc->hs_full[kb2], g & 1u)) return;
-                    if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                    if (!stage_wait()) return;
+                for (int st3 = 0; st3 < 3 && ok; ++st3, ++n) {
+                    if ((n & 1u) != me) continue;
+                    if (st3 < 2) {
+                        if (!wait(&misc->hs_full[st3], g & 1u)) return;
+                        if (first && st3 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                    } else {
+                        // both hidden blocks (and, on the first chunk, Y's release) are needed here too
+                        if (!wait(&misc->hs_full[0], g & 1u) || !wait(&misc->hs_full[1], g & 1u)) return;
+                        if (first && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                    }
+                    if (!stage_ready()) return;
                     const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 0, 3);
-                    __syncwarp();
-                    if (!peek_next(true)) return;
                     if (elect_one()) {
-                        mma_ksteps(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0, 3, 4);
-                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                        if (st3 < 2) {
+                            mma_kblock(tmem, hs + st3 * kBlockBytes, b, idesc256, first && st3 == 0);
+                            *issued = n + 1;
+                            ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                        } else {
+                            mma_kblock(tmem + 256, hs, b, idesc128, first);
+                            mma_kblock(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false);
+                            *issued = n + 1;
+                            ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                            ptx::umma_commit(bar_of(&misc->hs_empty[0]));
+                            ptx::umma_commit(bar_of(&misc->hs_empty[1]));
+                            if (last) ptx::umma_commit(bar_of(&misc->y_full));
+                        }
                     }
                     __syncwarp();
-                    ++n;
                 }
-                if (!stage_wait()) return;
-                const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                if (elect_one()) {
-                    mma_kblock(tmem + 256, hs, b, idesc128, first);
-                    mma_ksteps(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false, 0, 3);
-                }
-                __syncwarp();
-                if (!peek_next(!final)) return;
-                if (elect_one()) {
-                    mma_ksteps(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false, 3, 4);
-                    ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
-                    ptx::umma_commit(bar_of(&misc->hs_empty[0]));
-                    ptx::umma_commit(bar_of(&misc->hs_empty[1]));
-                    if (last) ptx::umma_commit(bar_of(&misc->y_full));
-                }
-                __syncwarp();
-                ++n;
             }
         };
         uint32_t g = 0, ti = 0;
@@ -417,13 +426,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
             for (int c = 0; c < NC && ok; ++c, ++g) {
                 gemm1(g, c, ti);
-                if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti, false);
+                if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
                 have_prev = true;
                 prev_g = g; prev_c = c; prev_ti = ti;
             }
         }
-        if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti, true);
-    } else if (warp < kEpiWarp0) {
+        if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
+    } else if (warp >= kLoaderWarp0 && warp < kEpiWarp0) {
         // ------------------------------------------------------------------ X row gather
         // Thread -> 8 (row, 16-byte chunk) pairs of every 128 x 64 block.  Up to three blocks
         // are in flight per thread; a block is published (x_full, one arrival per warp) once
@@ -472,7 +481,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         }
         while (ok && gx > published) publish_oldest();
         ptx::cp_async_wait_all();
-    } else {
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
         // ---------------------------------------------------------------------- epilogue
         const int ew = warp - kEpiWarp0;
         const int quarter = warp & 3, half = ew >> 2;
@@ -556,10 +565,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     uint32_t pk[32];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        pk[i] = pack_bf16x2(gelu_erf_fast(__uint_as_float(h0[2 * i])),
-                                            gelu_erf_fast(__uint_as_float(h0[2 * i + 1])));
-                        pk[16 + i] = pack_bf16x2(gelu_erf_fast(__uint_as_float(h1[2 * i])),
-                                                 gelu_erf_fast(__uint_as_float(h1[2 * i + 1])));
+                        pk[i] = gelu_erf_fast_bf16x2(__uint_as_float(h0[2 * i]), __uint_as_float(h0[2 * i + 1]));
+                        pk[16 + i] = gelu_erf_fast_bf16x2(__uint_as_float(h1[2 * i]), __uint_as_float(h1[2 * i + 1]));
                     }
                     if (!warp_wait(&misc->hs_empty[blk], (g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t hrow = hs + blk * kBlockBytes + row * 128;
