@@ -641,11 +641,24 @@ __device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k
     __syncwarp();
 }
 
+// acc_lo += a.lo * b.lo, acc_hi += a.hi * b.hi for two bf16 pairs, in fp32: the mixed-precision
+// FMA of sm_100 takes the bf16 operands as they are (exact products, fp32 accumulate), so
+// neither the query nor the key row has to be unpacked to fp32 first.
+__device__ __forceinline__ void fma_bf16_pair(float& acc_lo, float& acc_hi, uint32_t a, uint32_t b) {
+    asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
+        "mov.b32 {al, ah}, %2;\n\tmov.b32 {bl, bh}, %3;\n\t"
+        "fma.rn.f32.bf16 %0, al, bl, %0;\n\tfma.rn.f32.bf16 %1, ah, bh, %1;\n\t}"
+        : "+f"(acc_lo), "+f"(acc_hi)
+        : "r"(a), "r"(b));
+}
+
 // Sparsity scores of NH heads of the group at once for the queries of this thread:
 // M_i = max_j s_ij - mean_j s_ij over the sampled (or all) present keys, K rows from shared
-// memory.  The order keys of the scores go to keys_out[h][p].
+// memory.  The order keys of the scores go to keys_out[h][p].  The query rows stay in
+// registers as packed bf16 (D/2 words per head), so all kept heads of a group fit in one pass
+// and a sampled key row is fetched once per group.
 template <int D, int NH>
-__device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict__ Q, size_t q_head_stride,
+__device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict__ Q,
                                                  const size_t* q_base, const uint16_t* s_valid,
                                                  uint32_t ks_addr, int Tv,
                                                  const int32_t* __restrict__ tbl, int n_s, int cnt,
@@ -656,16 +669,14 @@ __device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict
     const float inv_cnt = 1.0f / (float)cnt;
     for (int p = threadIdx.x; p < Tv; p += blockDim.x) {
         const int tok = s_valid[p];
-        float q[NH][D];
+        uint32_t qw[NH][D / 2];
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
             const uint4* src = reinterpret_cast<const uint4*>(Q + q_base[h] + (size_t)tok * D);
 #pragma unroll
             for (int cc = 0; cc < S::CPR; ++cc) {
-                float f[8];
-                unpack8(__ldg(src + cc), f);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) q[h][8 * cc + e] = f[e];
+                const uint4 v = __ldg(src + cc);
+                qw[h][4 * cc] = v.x; qw[h][4 * cc + 1] = v.y; qw[h][4 * cc + 2] = v.z; qw[h][4 * cc + 3] = v.w;
             }
         }
         float mx[NH], sum[NH];
@@ -677,21 +688,23 @@ __device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict
             int pj = pj_next;
             if (a + 1 < cnt) pj_next = score_mode == 0 ? __ldg(row + a + 1) : a + 1;
             if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
-            float dot[NH];
+            float acc[NH][4];
 #pragma unroll
-            for (int h = 0; h < NH; ++h) dot[h] = 0.f;
+            for (int h = 0; h < NH; ++h) acc[h][0] = acc[h][1] = acc[h][2] = acc[h][3] = 0.f;
 #pragma unroll
             for (int cc = 0; cc < S::CPR; ++cc) {
-                float f[8];
-                unpack8(lds128(ks_addr + S::off(pj, cc)), f);
+                const uint4 v = lds128(ks_addr + S::off(pj, cc));
 #pragma unroll
-                for (int h = 0; h < NH; ++h)
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) dot[h] = fmaf(q[h][8 * cc + e], f[e], dot[h]);
+                for (int h = 0; h < NH; ++h) {
+                    fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc], v.x);
+                    fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 1], v.y);
+                    fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc + 2], v.z);
+                    fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 3], v.w);
+                }
             }
 #pragma unroll
             for (int h = 0; h < NH; ++h) {
-                const float sc = dot[h] * scale;
+                const float sc = ((acc[h][0] + acc[h][1]) + (acc[h][2] + acc[h][3])) * scale;
                 mx[h] = fmaxf(mx[h], sc);
                 sum[h] += sc;
             }
@@ -792,20 +805,22 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         ptx::cp_async_wait_group<1>();   // K has landed (V may still be in flight)
         __syncthreads();
         if (table_ok) {
-            constexpr int HPP = (D == 64) ? 1 : 2;   // heads per pass: q rows live in registers
+            constexpr int HPP = (D == 64) ? 2 : 4;   // heads per pass: packed q rows live in registers
             for (int h0 = 0; h0 < rk; h0 += HPP) {
                 const int nh = min(HPP, rk - h0);
-                size_t q_base[2];
-                uint32_t* keys_out[2];
-                for (int j = 0; j < 2; ++j) {
+                size_t q_base[4];
+                uint32_t* keys_out[4];
+                for (int j = 0; j < 4; ++j) {
                     const int hh = min(h0 + j, rk - 1);
                     q_base[j] = ((size_t)b * Hq + hs[hh]) * Tlen * D;
                     keys_out[j] = s_keys + (size_t)hh * Tlen;
                 }
-                if (HPP == 2 && nh == 2)
-                    fused_score_pass<D, (D == 64 ? 1 : 2)>(Q, 0, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
-                else
-                    fused_score_pass<D, 1>(Q, 0, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+                if (nh == 1) fused_score_pass<D, 1>(Q, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+                else if (nh == 2) fused_score_pass<D, 2>(Q, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+                else if constexpr (HPP == 4) {
+                    if (nh == 3) fused_score_pass<D, 3>(Q, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+                    else fused_score_pass<D, 4>(Q, q_base, s_valid, ks_addr, Tv, tbl, n_s, cnt, score_mode, keys_out, status);
+                }
             }
         } else {
             if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
