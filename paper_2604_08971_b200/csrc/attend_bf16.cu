@@ -26,7 +26,7 @@
 namespace {
 
 constexpr int kMaxRK = 4;          // kept heads of one KV group handled per CTA
-constexpr int kScoreThreads = 128;
+constexpr int kScoreThreads = 256;
 constexpr int kCoreThreads = 256;
 constexpr int kCoreWarps = kCoreThreads / 32;
 constexpr int kKeyTile = 64;
@@ -43,15 +43,6 @@ struct Sw {
         return (uint32_t)row * RB + (uint32_t)((c ^ ((row / RPL) & (CPR - 1))) << 4);
     }
 };
-
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        f[2 * j] = __uint_as_float(w[j] << 16);
-        f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
-    }
-}
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
@@ -73,36 +64,102 @@ __device__ __forceinline__ int group_heads(const int32_t* kept, int k_h, int r, 
 }
 
 // ------------------------------------------------------------------------------------ score
-template <int D, int RK>
-__device__ __forceinline__ void score_pass(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
-                                           const uint16_t* s_valid, uint32_t ks_addr, int seg_rows,
-                                           int Tv, int Tlen, int b, int g, int Hq, int Hk,
-                                           const int* hs, const int* khs,
-                                           const int32_t* tbl_row, int cnt, int score_mode, int p,
-                                           int k_h, float* __restrict__ mscore, unsigned int* status) {
+// acc_lo += a.lo * b.lo, acc_hi += a.hi * b.hi for two bf16 pairs, in fp32: the mixed-precision
+// FMA of sm_100 takes the bf16 operands as they are (exact products, fp32 accumulate), so
+// neither the query nor the key row has to be unpacked to fp32 first.
+__device__ __forceinline__ void fma_bf16_pair(float& acc_lo, float& acc_hi, uint32_t a, uint32_t b) {
+    asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
+        "mov.b32 {al, ah}, %2;\n\tmov.b32 {bl, bh}, %3;\n\t"
+        "fma.rn.f32.bf16 %0, al, bl, %0;\n\tfma.rn.f32.bf16 %1, ah, bh, %1;\n\t}"
+        : "+f"(acc_lo), "+f"(acc_hi)
+        : "r"(a), "r"(b));
+}
+
+// s = q . k / sqrt(d) for NH heads against one key row in shared memory; updates max and sum.
+template <int D, int NH>
+__device__ __forceinline__ void score_one_key(const uint32_t (&qw)[NH][D / 2], uint32_t row_addr_base, int row,
+                                              float scale, float (&mx)[NH], float (&sum)[NH]) {
+    using S = Sw<D>;
+    float acc[NH][4];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) acc[h][0] = acc[h][1] = acc[h][2] = acc[h][3] = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < S::CPR; ++cc) {
+        const uint4 v = lds128(row_addr_base + S::off(row, cc));
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc], v.x);
+            fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 1], v.y);
+            fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc + 2], v.z);
+            fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 3], v.w);
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+        const float sc = ((acc[h][0] + acc[h][1]) + (acc[h][2] + acc[h][3])) * scale;
+        mx[h] = fmaxf(mx[h], sc);
+        sum[h] += sc;
+    }
+}
+
+// Score pass for sequences whose K does not fit in shared memory at once: the group's present
+// K rows pass through shared memory in segments of seg_rows (a power of two).  Each thread owns
+// one query; it first sorts its sampled keys by segment into a per-thread list in shared memory
+// (counting sort, counts packed in one 64-bit register), so that during a segment every lane
+// walks only its own keys of that segment instead of skipping through the whole list.
+template <int D, int NH>
+__device__ __forceinline__ void long_score_pass(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ Kg,
+                                                const uint16_t* s_valid, uint16_t* s_list, uint32_t ks_addr,
+                                                int seg_shift, int Tv, int Tlen, const size_t* q_base,
+                                                const int* khs, const int32_t* tbl_row, int cnt,
+                                                int score_mode, int p, int b, int k_h,
+                                                float* __restrict__ mscore, unsigned int* status) {
     using S = Sw<D>;
     const bool act = p < Tv;
-    float q[RK][D];
-    float mx[RK], sum[RK];
+    const int seg_rows = 1 << seg_shift;
+    uint32_t qw[NH][D / 2];
+    float mx[NH], sum[NH];
 #pragma unroll
-    for (int h = 0; h < RK; ++h) { mx[h] = -INFINITY; sum[h] = 0.f; }
+    for (int h = 0; h < NH; ++h) { mx[h] = -INFINITY; sum[h] = 0.f; }
+    unsigned long long starts = 0ull;   // byte s = first list slot of segment s (8 segments at most)
     if (act) {
         const int tok = s_valid[p];
 #pragma unroll
-        for (int h = 0; h < RK; ++h) {
-            const uint4* src = reinterpret_cast<const uint4*>(Q + (((size_t)b * Hq + hs[h]) * Tlen + tok) * D);
+        for (int h = 0; h < NH; ++h) {
+            const uint4* src = reinterpret_cast<const uint4*>(Q + q_base[h] + (size_t)tok * D);
 #pragma unroll
-            for (int c = 0; c < S::CPR; ++c) {
-                float f[8];
-                unpack8(__ldg(src + c), f);
+            for (int cc = 0; cc < S::CPR; ++cc) {
+                const uint4 v = __ldg(src + cc);
+                qw[h][4 * cc] = v.x; qw[h][4 * cc + 1] = v.y; qw[h][4 * cc + 2] = v.z; qw[h][4 * cc + 3] = v.w;
+            }
+        }
+        if (score_mode == 0) {
+            unsigned long long counts = 0ull;
+            for (int a = 0; a < cnt; ++a) {
+                int pj = __ldg(tbl_row + a);
+                if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
+                counts += 1ull << (8 * (pj >> seg_shift));
+            }
+            unsigned long long run = 0ull;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) q[h][8 * c + e] = f[e];
+            for (int sgm = 0; sgm < 8; ++sgm) {
+                starts |= run << (8 * sgm);
+                run += (counts >> (8 * sgm)) & 255ull;
+            }
+            unsigned long long fill = starts;
+            for (int a = 0; a < cnt; ++a) {
+                int pj = __ldg(tbl_row + a);
+                if (pj < 0 || pj >= Tv) pj = 0;
+                const int sgm = pj >> seg_shift;
+                const int pos = (int)((fill >> (8 * sgm)) & 255ull);
+                fill += 1ull << (8 * sgm);
+                s_list[pos * blockDim.x + threadIdx.x] = (uint16_t)pj;
             }
         }
     }
     const float scale = rsqrtf((float)D);
-    const __nv_bfloat16* Kg = K + ((size_t)b * Hk + g) * Tlen * D;
-    for (int seg0 = 0; seg0 < Tv; seg0 += seg_rows) {
+    int sgm = 0;
+    for (int seg0 = 0; seg0 < Tv; seg0 += seg_rows, ++sgm) {
         const int seg_n = min(seg_rows, Tv - seg0);
         __syncthreads();  // the previous segment is no longer being read
         for (int i = threadIdx.x; i < seg_n * S::CPR; i += blockDim.x) {
@@ -111,53 +168,41 @@ __device__ __forceinline__ void score_pass(const __nv_bfloat16* __restrict__ Q, 
         }
         ptx::cp_async_wait_all();
         __syncthreads();
-        if (act) {
-            for (int a = 0; a < cnt; ++a) {
-                int pj = score_mode == 0 ? tbl_row[a] : a;
-                if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
-                const int row = pj - seg0;
-                if (row < 0 || row >= seg_n) continue;
-                float dot[RK];
-#pragma unroll
-                for (int h = 0; h < RK; ++h) dot[h] = 0.f;
-#pragma unroll
-                for (int c = 0; c < S::CPR; ++c) {
-                    float f[8];
-                    unpack8(lds128(ks_addr + S::off(row, c)), f);
-#pragma unroll
-                    for (int h = 0; h < RK; ++h)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) dot[h] = fmaf(q[h][8 * c + e], f[e], dot[h]);
-                }
-#pragma unroll
-                for (int h = 0; h < RK; ++h) {
-                    const float s = dot[h] * scale;
-                    mx[h] = fmaxf(mx[h], s);
-                    sum[h] += s;
-                }
+        if (!act) continue;
+        if (score_mode == 0) {
+            const int i0 = (int)((starts >> (8 * sgm)) & 255ull);
+            const int i1 = sgm == 7 ? cnt : (seg0 + seg_rows >= Tv ? cnt : (int)((starts >> (8 * (sgm + 1))) & 255ull));
+            for (int i = i0; i < i1; ++i) {
+                const int pj = s_list[i * blockDim.x + threadIdx.x];
+                score_one_key<D, NH>(qw, ks_addr, pj - seg0, scale, mx, sum);
             }
+        } else {
+            for (int row = 0; row < seg_n; ++row) score_one_key<D, NH>(qw, ks_addr, row, scale, mx, sum);
         }
     }
     if (act) {
 #pragma unroll
-        for (int h = 0; h < RK; ++h)
+        for (int h = 0; h < NH; ++h)
             mscore[((size_t)b * k_h + khs[h]) * Tlen + p] = mx[h] - sum[h] / (float)cnt;
     }
 }
 
-// grid (ceil(T/threads), B*Hk).  Dynamic smem: valid list (2T bytes, 16-aligned) + K segment.
+// grid (ceil(T/threads), B*Hk).  Dynamic smem: valid list (2T bytes, 128-aligned) | per-thread key
+// lists [kMaxActive][threads] u16 | K segment.
 template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 attend_score_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                          const int32_t* __restrict__ kept_heads, const int32_t* __restrict__ ids,
                          const uint32_t* __restrict__ masks, const int32_t* __restrict__ table,
                          const int64_t* __restrict__ offsets, int n_subsets, int Tlen, int Hq, int Hk,
-                         int k_h, int c, int score_mode, int seg_rows, float* __restrict__ mscore,
+                         int k_h, int c, int score_mode, int seg_shift, float* __restrict__ mscore,
                          unsigned int* status) {
     extern __shared__ __align__(128) uint8_t s_raw[];
     __shared__ int red[66];
     uint16_t* s_valid = reinterpret_cast<uint16_t*>(s_raw);
-    const uint32_t ks_addr = ptx::smem_u32(s_raw) + (uint32_t)((((size_t)Tlen * 2 + 127) / 128) * 128);
+    const size_t valid_bytes = (((size_t)Tlen * 2 + 127) / 128) * 128;
+    uint16_t* s_list = reinterpret_cast<uint16_t*>(s_raw + valid_bytes);
+    const uint32_t ks_addr = ptx::smem_u32(s_raw) + (uint32_t)(valid_bytes + (size_t)kMaxActive * kScoreThreads * 2);
     const int b = blockIdx.y / Hk, g = blockIdx.y % Hk;
     const uint32_t mask = masks[b];
     const int Tv = block_build_valid(ids, Tlen, mask, s_valid, red);
@@ -178,28 +223,28 @@ attend_score_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         }
         tbl_row = table + offsets[mask] + (size_t)min(p, Tv - 1) * n_s;
     }
-    // The q rows of a pass live in registers: up to 4 heads x 32 dims, or 2 heads x 64 dims.
-#define SCORE_PASS(N, H0, H1, H2, H3)                                                              \
-    {                                                                                              \
-        const int hs_[kMaxRK] = {hs[H0], hs[H1], hs[H2], hs[H3]};                                  \
-        const int khs_[kMaxRK] = {khs[H0], khs[H1], khs[H2], khs[H3]};                             \
-        score_pass<D, N>(Q, K, s_valid, ks_addr, seg_rows, Tv, Tlen, b, g, Hq, Hk, hs_, khs_,      \
-                         tbl_row, cnt, score_mode, p, k_h, mscore, status);                        \
-    }
-    if constexpr (D == 64) {
-        if (rk == 1) SCORE_PASS(1, 0, 0, 0, 0)
-        else SCORE_PASS(2, 0, 1, 0, 0)
-        if (rk == 3) SCORE_PASS(1, 2, 2, 2, 2)
-        else if (rk == 4) SCORE_PASS(2, 2, 3, 2, 2)
-    } else {
-        switch (rk) {
-            case 1: SCORE_PASS(1, 0, 0, 0, 0) break;
-            case 2: SCORE_PASS(2, 0, 1, 0, 0) break;
-            case 3: SCORE_PASS(3, 0, 1, 2, 0) break;
-            default: SCORE_PASS(4, 0, 1, 2, 3) break;
+    const __nv_bfloat16* Kg = K + ((size_t)b * Hk + g) * Tlen * D;
+    constexpr int HPP = (D == 64) ? 1 : (D == 32 ? 2 : 4);   // heads per pass: packed q rows live in registers
+    for (int h0 = 0; h0 < rk; h0 += HPP) {
+        const int nh = min(HPP, rk - h0);
+        size_t q_base[4];
+        int khs_[4];
+        for (int j = 0; j < 4; ++j) {
+            const int hh = min(h0 + j, rk - 1);
+            q_base[j] = ((size_t)b * Hq + hs[hh]) * Tlen * D;
+            khs_[j] = khs[hh];
         }
+#define LONG_PASS(N) long_score_pass<D, N>(Q, Kg, s_valid, s_list, ks_addr, seg_shift, Tv, Tlen, q_base, khs_, \
+                                           tbl_row, cnt, score_mode, p, b, k_h, mscore, status)
+        if (nh == 1) LONG_PASS(1);
+        else if (nh == 2) LONG_PASS(2);
+        else if constexpr (HPP == 4) {
+            if (nh == 3) LONG_PASS(3);
+            else LONG_PASS(4);
+        }
+#undef LONG_PASS
+        __syncthreads();
     }
-#undef SCORE_PASS
 }
 
 // ------------------------------------------------------------------------------------- core
@@ -641,17 +686,6 @@ __device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k
     __syncwarp();
 }
 
-// acc_lo += a.lo * b.lo, acc_hi += a.hi * b.hi for two bf16 pairs, in fp32: the mixed-precision
-// FMA of sm_100 takes the bf16 operands as they are (exact products, fp32 accumulate), so
-// neither the query nor the key row has to be unpacked to fp32 first.
-__device__ __forceinline__ void fma_bf16_pair(float& acc_lo, float& acc_hi, uint32_t a, uint32_t b) {
-    asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
-        "mov.b32 {al, ah}, %2;\n\tmov.b32 {bl, bh}, %3;\n\t"
-        "fma.rn.f32.bf16 %0, al, bl, %0;\n\tfma.rn.f32.bf16 %1, ah, bh, %1;\n\t}"
-        : "+f"(acc_lo), "+f"(acc_hi)
-        : "r"(a), "r"(b));
-}
-
 // Sparsity scores of NH heads of the group at once for the queries of this thread:
 // M_i = max_j s_ij - mean_j s_ij over the sampled (or all) present keys, K rows from shared
 // memory.  The order keys of the scores go to keys_out[h][p].  The query rows stay in
@@ -1047,10 +1081,12 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
     }
     const size_t valid_bytes = (((size_t)d.T * 2 + 127) / 128) * 128;
     if (!a.selection_given) {
-        // K segment: as many rows as fit in ~64 KB (one pass for T <= 1024 at d = 32)
-        int seg_rows = (64 * 1024) / (D * 2);
-        if (seg_rows > d.T) seg_rows = (d.T + 7) / 8 * 8;
-        const size_t smem = valid_bytes + (size_t)seg_rows * D * 2;
+        // K segment: 64 KB worth of rows, a power of two (at most 8 segments for T <= 8192)
+        int seg_shift = 0;
+        while ((2 << seg_shift) * D * 2 <= 64 * 1024) ++seg_shift;
+        while ((8 << seg_shift) < d.T) ++seg_shift;
+        const int seg_rows = 1 << seg_shift;
+        const size_t smem = valid_bytes + (size_t)kMaxActive * kScoreThreads * 2 + (size_t)seg_rows * D * 2;
         auto kern = attend_score_bf16_kernel<D>;
         SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid((d.T + kScoreThreads - 1) / kScoreThreads, d.B * d.Hk);
@@ -1058,7 +1094,7 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
         kern<<<grid, kScoreThreads, smem, st>>>((const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K,
                                                  a.kept_heads, a.ids, a.masks, a.sample_table,
                                                  a.sample_offsets, a.n_subsets, d.T, d.Hq, d.Hk, d.k_h,
-                                                 d.c, d.score_mode, seg_rows, a.mscore, a.status);
+                                                 d.c, d.score_mode, seg_shift, a.mscore, a.status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
     {
