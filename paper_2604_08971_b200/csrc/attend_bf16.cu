@@ -30,7 +30,8 @@ constexpr int kScoreThreads = 256;
 constexpr int kCoreThreads = 256;
 constexpr int kCoreWarps = kCoreThreads / 32;
 constexpr int kKeyTile = 64;
-constexpr int kMaxActive = 48;     // U <= 45 for T <= 8103 with c = 5 (checked on the host)
+constexpr int kMaxActive = 48;
+constexpr int kOrderMaxBatch = 1024; // batches up to this size are walked heaviest-sample-first     // U <= 45 for T <= 8103 with c = 5 (checked on the host)
 
 // Row layout in shared memory: rows of D bf16, 16-byte chunks XOR-swizzled so that both
 // 8-consecutive-row matrix loads and random row gathers spread over the banks.
@@ -780,7 +781,48 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     const uint32_t ks_addr = ptx::smem_u32(s_raw + o);          o += (size_t)Tpad * D * 2;
     const uint32_t vs_addr = ptx::smem_u32(s_raw + o);
 
-    const int b = blockIdx.x / Hk, g = blockIdx.x % Hk;
+    // Samples with more modalities present take longer; in small batches the CTAs take them
+    // heaviest first (every CTA finds the sample of its rank by itself with a counting sort on
+    // the number of present modalities), so that the long ones do not end up alone in the tail
+    // of the launch.
+    int b = blockIdx.x / Hk;
+    const int g = blockIdx.x % Hk;
+    const int Bn = gridDim.x / Hk;
+    if (Bn > 1 && Bn <= kOrderMaxBatch) {
+        __shared__ int s_hist[33];
+        __shared__ int s_wcnt[16];
+        __shared__ int s_pick[2];
+        const int lane_ = threadIdx.x & 31, wid_ = threadIdx.x >> 5, nw_ = blockDim.x >> 5;
+        if (threadIdx.x < 33) s_hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (int bb = threadIdx.x; bb < Bn; bb += blockDim.x) atomicAdd(&s_hist[__popc(masks[bb])], 1);
+        __syncthreads();
+        if (threadIdx.x == 0) {   // class (present modalities, descending) that holds rank b, and the offset in it
+            int left = b, cls = 32;
+            while (cls > 0 && left >= s_hist[cls]) { left -= s_hist[cls]; --cls; }
+            s_pick[0] = cls;
+            s_pick[1] = left;
+        }
+        __syncthreads();
+        const int cls = s_pick[0];
+        int need = s_pick[1];      // the need-th sample of that class, in index order
+        __syncthreads();
+        for (int b0 = 0; b0 < Bn; b0 += blockDim.x) {
+            const int bb = b0 + threadIdx.x;
+            const bool hit = bb < Bn && __popc(masks[bb]) == cls;
+            const unsigned bm = __ballot_sync(0xffffffffu, hit);
+            if (lane_ == 0) s_wcnt[wid_] = __popc(bm);
+            __syncthreads();
+            int before = 0, tot = 0;
+            for (int w = 0; w < nw_; ++w) { if (w < wid_) before += s_wcnt[w]; tot += s_wcnt[w]; }
+            if (hit && before + __popc(bm & ((1u << lane_) - 1u)) == need) s_pick[0] = bb;
+            __syncthreads();
+            if (need < tot) break;
+            need -= tot;
+        }
+        __syncthreads();
+        b = s_pick[0];
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const uint32_t mask = masks[b];
     const int Tv = block_build_valid(ids, Tlen, mask, s_valid, red);
