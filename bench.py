@@ -279,6 +279,10 @@ def run_ours(args, w: synth.Workload):
         dist.init_process_group("nccl", device_id=torch.device(dev))
     sentry.build()
     sn = sentry.Sentry(local_rank)
+    # the attention branch (gate for heads -> attend) and the FFN branch (gate for channels -> ffn) are
+    # independent: a second context with its own workspace lets them run on two streams of one graph
+    sn2 = sentry.Sentry(local_rank) if not args.no_overlap else sn
+    branch = torch.cuda.Stream() if not args.no_overlap else None
     n_s_of = lambda tv: sentry.num_active_queries(tv, w.c)
 
     sampler = ClockSampler(local_rank)
@@ -300,23 +304,35 @@ def run_ours(args, w: synth.Workload):
     hpg = w.Hq // w.Hk
     launches = [0]
 
-    def step(s: DeviceSet, count=False):
+    def ffn_branch(s: DeviceSet, ctx):
+        ctx.gate_select(sc, subsets, w.k_c, kept=s.kept_c)
+        n = ctx.last_launch_count()
+        ctx.ffn_fwd(s.X, W1, W2, s.kept_c, los, ids, masks, Y=s.Y)
+        return n + ctx.last_launch_count()
+
+    def step(s: DeviceSet, count=False, fork=True):
         n = 0
+        two = fork and branch is not None
+        if two:
+            cur = torch.cuda.current_stream()
+            branch.wait_stream(cur)
+            with torch.cuda.stream(branch):
+                n += ffn_branch(s, sn2)
         sn.gate_select(sh, masks, w.k_h, kept=s.kept_h)
-        n += sn.last_launch_count()
-        sn.gate_select(sc, subsets, w.k_c, kept=s.kept_c)
         n += sn.last_launch_count()
         sn.attend_fwd(s.Q, s.K, s.V, s.kept_h, ids, masks, tbl, offs, c=w.c, O=s.O)
         n += sn.last_launch_count()
-        sn.ffn_fwd(s.X, W1, W2, s.kept_c, los, ids, masks, Y=s.Y)
-        n += sn.last_launch_count()
+        if two:
+            torch.cuda.current_stream().wait_stream(branch)
+        else:
+            n += ffn_branch(s, sn)
         if count:
             launches[0] = n
 
     # workspace sized once, before any capture
     step(sets[0], count=True)
     torch.cuda.synchronize()
-    assert sn.last_status() == 0, "device status word set during warm-up"
+    assert sn.last_status() == 0 and sn2.last_status() == 0, "device status word set during warm-up"
 
     graphs = None
     if not args.no_graph:
@@ -358,11 +374,11 @@ def run_ours(args, w: synth.Workload):
     # ---- per-kernel pass (same steps, events around every kernel, no graph)
     sn.profile_enable(True)
     for i in range(3):
-        step(sets[i % n_sets])
+        step(sets[i % n_sets], fork=False)
     sn.profile_read()
     n_prof = min(args.steps, 50)
     for i in range(n_prof):
-        step(sets[i % n_sets])
+        step(sets[i % n_sets], fork=False)
     prof = sn.profile_read()
     sn.profile_enable(False)
 
@@ -395,7 +411,7 @@ def run_ours(args, w: synth.Workload):
     ev1.record()
     barrier_sync()
     e2e_tokens, e2e_ms = aggregate(float(wm["tokens"]) * n_e2e, ev0.elapsed_time(ev1), dev)
-    status = sn.last_status()
+    status = sn.last_status() | sn2.last_status()
     sampler.stop_flag = True
 
     if rank != 0:
@@ -459,7 +475,9 @@ def run_ours(args, w: synth.Workload):
                    "present_tokens_per_step_per_gpu": wm["tokens"], "parallelism": "replicas x%d" % world,
                    "l2_policy": "rotating %d resident buffer sets, %.0f MB in total (> 126 MB L2)"
                                 % (n_sets, n_sets * set_bytes / 1e6),
-                   "cuda_graph": graphs is not None},
+                   "cuda_graph": graphs is not None,
+                   "streams": "attention branch and FFN branch forked inside the step" if branch is not None
+                              else "one stream"},
         "useful_tflops": (wm["att_flops"] + wm["ffn_flops"]) * world * args.steps / (ms * 1e-3) / 1e12,
         "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": n_e2e},
@@ -479,6 +497,8 @@ def main():
                     help="1, 2, 3a|3b|3c, 4 (default: the full pruned encoder layer), 5:BxT")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="run the attention branch and the FFN branch of a step on one stream")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
