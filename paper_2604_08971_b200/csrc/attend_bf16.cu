@@ -278,23 +278,54 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Warp-level top-k over n order keys in shared memory (larger key first, ties -> lower index).
-// Writes remap[index] of the selected entries to out[0..k) in ascending index order.
-__device__ inline void warp_select_topk(const uint32_t* keys, int n, int k, int32_t* out,
-                                        const uint16_t* remap) {
+// Warp-level top-k by radix selection over n order keys in shared memory (larger key first,
+// ties -> lower index).  Writes remap[index] of the selected entries to out[0..k) in ascending
+// index order.  `hist` = 256 ints of shared memory owned by this warp.
+__device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k, int32_t* out,
+                                              const uint16_t* remap, int* hist) {
     const int lane = threadIdx.x & 31;
-    uint32_t t = 0;
-    for (int bit = 31; bit >= 0; --bit) {
-        const uint32_t cand = t | (1u << bit);
-        int cnt = 0;
-        for (int i = lane; i < n; i += 32) cnt += (keys[i] >= cand);
-        cnt = __reduce_add_sync(0xffffffffu, cnt);
-        if (cnt >= k) t = cand;
+    uint32_t prefix = 0, fixed = 0;
+    int want = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = lane; i < 256; i += 32) hist[i] = 0;
+        __syncwarp();
+        for (int i = lane; i < n; i += 32) {
+            const uint32_t key = keys[i];
+            if ((key & fixed) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+        }
+        __syncwarp();
+        const int top = 255 - 8 * lane;      // this lane's digits, descending
+        int mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine += hist[top - j];
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int above = incl - mine;
+        const bool here = above < want && want <= incl;
+        int digit = 0, rem = 0;
+        if (here) {
+            int acc = above;
+            for (int j = 0; j < 8; ++j) {
+                const int cdig = hist[top - j];
+                if (want <= acc + cdig) { digit = top - j; rem = want - acc; break; }
+                acc += cdig;
+            }
+        }
+        const unsigned who = __ballot_sync(0xffffffffu, here);
+        const int src = __ffs(who) - 1;
+        digit = __shfl_sync(0xffffffffu, digit, src);
+        rem = __shfl_sync(0xffffffffu, rem, src);
+        prefix |= (uint32_t)digit << shift;
+        fixed |= 255u << shift;
+        want = rem;
+        __syncwarp();
     }
-    int gt = 0;
-    for (int i = lane; i < n; i += 32) gt += (keys[i] > t);
-    gt = __reduce_add_sync(0xffffffffu, gt);
-    const int need_eq = k - gt;
+    const uint32_t t = prefix;
+    const int need_eq = want;
     int base = 0, eq_seen = 0;
     for (int i0 = 0; i0 < n; i0 += 32) {
         const int i = i0 + lane;
@@ -319,7 +350,7 @@ struct CoreSmem {
 
 // grid B*Hk.  Dynamic smem: valid[T] u16 | kind[T] u8 | actbits[4][T/32] u32 | union{keys, KV pipe}
 template <int D>
-__global__ void __launch_bounds__(kCoreThreads)
+__global__ void __launch_bounds__(kCoreThreads, 2)
 attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                         const __nv_bfloat16* __restrict__ V, const int32_t* __restrict__ kept_heads,
                         const int32_t* __restrict__ ids, const uint32_t* __restrict__ masks,
@@ -334,6 +365,7 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     __shared__ int red[66];
     __shared__ int32_t s_act[kMaxRK][kMaxActive];
     __shared__ float s_vpart[kCoreThreads / (D / 2)][D];   // partial column sums of V
+    __shared__ int s_hist[kMaxRK][256];                    // radix-selection histograms, one per head
     __shared__ __align__(16) __nv_bfloat16 s_mean[D];
 
     const int words = (Tlen + 31) / 32;
@@ -378,7 +410,7 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
             for (int p = threadIdx.x; p < Tv; p += blockDim.x) s_keys[(size_t)hh * Tv + p] = sentry_order_key(m[p]);
         }
         __syncthreads();
-        if (warp < rk) warp_select_topk(s_keys + (size_t)warp * Tv, Tv, U, s_act[warp], s_valid);
+        if (warp < rk) warp_select_topk_radix(s_keys + (size_t)warp * Tv, Tv, U, s_act[warp], s_valid, s_hist[warp]);
         __syncthreads();
         if (active_out != nullptr)
             for (int i = threadIdx.x; i < rk * U_max; i += blockDim.x) {
@@ -623,69 +655,6 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
 //   top-U per head (one warp per head, radix selection) -> Eq. 6 on the active rows with the
 //   warp-level tensor-core MMA straight from the resident K/V -> context rows and zero rows.
 // Q, K, V are read from HBM once and O is written once: the algorithmic traffic.
-
-// Warp-level top-k by radix selection over n order keys in shared memory (larger key first,
-// ties -> lower index).  Writes remap[index] of the selected entries to out[0..k) in ascending
-// index order.  `hist` = 256 ints of shared memory owned by this warp.
-__device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k, int32_t* out,
-                                              const uint16_t* remap, int* hist) {
-    const int lane = threadIdx.x & 31;
-    uint32_t prefix = 0, fixed = 0;
-    int want = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = lane; i < 256; i += 32) hist[i] = 0;
-        __syncwarp();
-        for (int i = lane; i < n; i += 32) {
-            const uint32_t key = keys[i];
-            if ((key & fixed) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
-        }
-        __syncwarp();
-        const int top = 255 - 8 * lane;      // this lane's digits, descending
-        int mine = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) mine += hist[top - j];
-        int incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        const int above = incl - mine;
-        const bool here = above < want && want <= incl;
-        int digit = 0, rem = 0;
-        if (here) {
-            int acc = above;
-            for (int j = 0; j < 8; ++j) {
-                const int cdig = hist[top - j];
-                if (want <= acc + cdig) { digit = top - j; rem = want - acc; break; }
-                acc += cdig;
-            }
-        }
-        const unsigned who = __ballot_sync(0xffffffffu, here);
-        const int src = __ffs(who) - 1;
-        digit = __shfl_sync(0xffffffffu, digit, src);
-        rem = __shfl_sync(0xffffffffu, rem, src);
-        prefix |= (uint32_t)digit << shift;
-        fixed |= 255u << shift;
-        want = rem;
-        __syncwarp();
-    }
-    const uint32_t t = prefix;
-    const int need_eq = want;
-    int base = 0, eq_seen = 0;
-    for (int i0 = 0; i0 < n; i0 += 32) {
-        const int i = i0 + lane;
-        const uint32_t key = i < n ? keys[i] : 0u;
-        const bool is_eq = i < n && key == t, is_gt = i < n && key > t;
-        const unsigned em = __ballot_sync(0xffffffffu, is_eq);
-        const bool keep = is_gt || (is_eq && eq_seen + __popc(em & ((1u << lane) - 1u)) < need_eq);
-        const unsigned km = __ballot_sync(0xffffffffu, keep);
-        if (keep) out[base + __popc(km & ((1u << lane) - 1u))] = (int32_t)remap[i];
-        base += __popc(km);
-        eq_seen += __popc(em);
-    }
-    __syncwarp();
-}
 
 // Sparsity scores of NH heads of the group at once for the queries of this thread:
 // M_i = max_j s_ij - mean_j s_ij over the sampled (or all) present keys, K rows from shared
