@@ -50,6 +50,7 @@ struct Cfg {
     static constexpr int NXS = (D == 128) ? 4 : KB1;   // X block slots (D = 128: two tiles' worth)
     static constexpr int NHS = CH / 64;                // hidden blocks per chunk (64 channels each)
     static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
+    static constexpr int SPG = (D == 384) ? 3 : KB1;   // weight stages per chunk of GEMM1 (= of GEMM2)
     static constexpr int OFF_H = NXS * kBlockBytes;
     static constexpr int OFF_W = OFF_H + NHS * kBlockBytes;
     static constexpr int OFF_MISC = OFF_W + kStages * kStageBytes;
@@ -132,15 +133,49 @@ __device__ __forceinline__ void warp_arrive(uint64_t* bar) {
     if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(bar));
 }
 
-// Four K=16 steps over one 64-wide K block: D (+)= A[128 x 64] . B[N x 64]^T.
-// Called by the one elected lane of a converged warp (see the issuer below).
-__device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr,
-                                           uint32_t idesc, bool overwrite) {
-    const uint64_t ad = ptx::umma_smem_desc_sw128(a_addr);
-    const uint64_t bd = ptx::umma_smem_desc_sw128(b_addr);
-#pragma unroll
-    for (uint32_t ks = 0; ks < 4; ++ks)
-        ptx::umma_bf16(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (!overwrite || ks > 0) ? 1u : 0u);
+// ---- lean forms for the single-thread roles -------------------------------------------------
+// A warp that walks a chain of dependent scalar instructions with shared-memory round trips in
+// it (an mbarrier probe, a flag poll, a vote) advances at 8 to 15 cycles per instruction here,
+// so what the producers and issuers execute per stage is counted in instructions: barrier
+// addresses are one add from a base, descriptors are a 32-bit add and a register pair, all the
+// probes of a stage are issued back to back and voted on once.
+#define MISC_BAR(base, field) ((base) + (uint32_t)offsetof(Misc, field))
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // upper word of umma_smem_desc_sw128
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3fffu) | (1u << 16); }
+// D (+)= A . B^T for one 64-wide K block = four K=16 steps; descriptors from their low words
+__device__ __forceinline__ void mma_kblock_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t accumulate_first) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+        "setp.ne.b32 p, 1, 0;\n\t"
+        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        :
+        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(kDescHi), "r"(accumulate_first)
+        : "memory");
+}
+// Slow path of a stage's combined wait: the barriers one after the other, bounded (0 = none).
+static __device__ __noinline__ bool wait_each_slow(uint32_t b0, uint32_t p0, uint32_t b1, uint32_t p1, uint32_t b2,
+                                                   uint32_t p2, uint32_t b3, uint32_t p3, volatile int* abort_flag) {
+    bool ok = ptx::mbar_wait(b0, p0, abort_flag);
+    if (ok && b1 != 0u) ok = ptx::mbar_wait(b1, p1, abort_flag);
+    if (ok && b2 != 0u) ok = ptx::mbar_wait(b2, p2, abort_flag);
+    if (ok && b3 != 0u) ok = ptx::mbar_wait(b3, p3, abort_flag);
+    return ok;
+}
+// Slow path of the issuers' turn: poll until `n` stages have been issued, bounded.
+static __device__ __noinline__ bool turn_wait_slow(volatile uint32_t* issued, uint32_t n, volatile int* abort_flag) {
+    for (uint32_t spins = 0; *issued < n; ++spins) {
+        if (spins > (1u << 22) || *abort_flag) { *abort_flag = 1; return false; }
+    }
+    return true;
 }
 
 // One lane of a fully converged warp.  The single-thread instructions (TMA, UMMA, commit) are
@@ -207,10 +242,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
     ptx::tc_fence_after_sync();
     const uint32_t tmem = misc->tmem_base;
 
+    constexpr int SPG = C::SPG;
+    const uint32_t mb = ptx::smem_u32(misc);
+    const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const uint32_t n_chunks = (uint32_t)(my_tiles * NC);
+    // Ring order: GEMM1 of chunk 0; then, per chunk q >= 1, GEMM1 of q and GEMM2 of q-1; at the
+    // end GEMM2 of the last chunk.  Producers and issuers walk it as "group q = GEMM1(q), GEMM2(q-1)"
+    // for q = 0 .. n_chunks, skipping the halves that do not exist; SPG stages per GEMM.
     if (warp == 0 || warp == 2) {
         // ----------------------------------------------------------- weight TMA producers
-        // Both walk the issuer's stage sequence (GEMM1 stages of chunk g, then GEMM2 stages of
-        // chunk g-1); producer p loads the stages with index n = p (mod 2).
+        // Producer p loads the stages with ring position n = p (mod 2).
         const uint32_t me = (warp == 0) ? 0u : 1u;
         if (elect_one()) {
             ptx::prefetch_tensormap(&tm_w1);
@@ -218,220 +259,184 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             ptx::prefetch_tensormap(&tm_w2_128);
         }
         __syncwarp();
-        uint32_t n = 0;
-        bool ok = true;
         // one stage = one 32 KB box, or two 16 KB boxes (x1 < 0: single box)
-        auto stage = [&](const CUtensorMap* tm, int x0, int x1, int y) {
-            const uint32_t idx = n++;
-            if (!ok || (idx & 1u) != me) return;
-            const uint32_t s = idx % kStages, use = idx / kStages;
-            if (!warp_wait(&misc->w_empty[s], (use & 1u) ^ 1u, abort_flag)) {
-                ok = false;
-                return;
-            }
-            const uint32_t bar = ptx::smem_u32(&misc->w_full[s]);
-            const uint32_t dst = wsm + s * kStageBytes;
+        auto stage = [&](uint32_t n, const CUtensorMap* tm, int x0, int x1, int y) -> bool {
+            const uint32_t sl = n % kStages, use = n / kStages;
+            const uint32_t we = MISC_BAR(mb, w_empty) + 8u * sl;
+            if (!__all_sync(0xffffffffu, ptx::mbar_try_wait(we, (use & 1u) ^ 1u)) &&
+                !__all_sync(0xffffffffu, ptx::mbar_wait_slow(we, (use & 1u) ^ 1u, abort_flag)))
+                return false;
             if (elect_one()) {
+                const uint32_t bar = MISC_BAR(mb, w_full) + 8u * sl;
+                const uint32_t dst = wsm + sl * kStageBytes;
                 ptx::mbar_arrive_expect_tx(bar, kStageBytes);
                 ptx::tma_load_2d(dst, tm, x0, y, bar);
                 if (x1 >= 0) ptx::tma_load_2d(dst + kBlockBytes, tm, x1, y, bar);
             }
             __syncwarp();
+            return true;
         };
-        auto gemm1_stages = [&](int l, int c) {
-            const int y = l * kc_pad + c * C::CH;
-            if constexpr (D == 384) {
-                for (int kp = 0; kp < 3; ++kp) stage(&tm_w1, 128 * kp, 128 * kp + 64, y);
-            } else {
-                for (int kb = 0; kb < C::KB1; ++kb) stage(&tm_w1, 64 * kb, -1, y);
+        uint32_t n = 0;
+        bool ok = true;
+        int l_cur = 0, l_last = 0, c = 0;
+        uint32_t ti = 0;
+#pragma unroll 1
+        for (uint32_t q = 0; q <= n_chunks && ok; ++q) {
+            if (c == 0) {
+                l_last = l_cur;
+                if (q < n_chunks) {
+                    int row0, n_rows;
+                    ffn_tile_lookup(plan, n_lists, (int)blockIdx.x + (int)ti * (int)gridDim.x, kTileRows, l_cur, row0, n_rows);
+                }
             }
-        };
-        auto gemm2_stages = [&](int l, int c) {
-            const int x = c * C::CH;
-            if constexpr (D == 256) {
-                for (int kb2 = 0; kb2 < 4; ++kb2) stage(&tm_w2_256, x + 64 * kb2, -1, l * D);
-            } else if constexpr (D == 128) {
-                for (int kp = 0; kp < 2; ++kp) stage(&tm_w2_128, x + 128 * kp, x + 128 * kp + 64, l * D);
-            } else {
-                stage(&tm_w2_256, x, -1, l * D);
-                stage(&tm_w2_256, x + 64, -1, l * D);
-                stage(&tm_w2_128, x, x + 64, l * D + 256);
+            if (q < n_chunks) {
+                const int y = l_cur * kc_pad + c * C::CH;
+#pragma unroll
+                for (int i = 0; i < SPG; ++i) {
+                    if (ok && ((n + i) & 1u) == me) {
+                        if constexpr (D == 384) ok = stage(n + i, &tm_w1, 128 * i, 128 * i + 64, y);
+                        else ok = stage(n + i, &tm_w1, 64 * i, -1, y);
+                    }
+                }
+                n += SPG;
             }
-        };
-        int prev_l = -1, prev_c = 0;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            int l, row0, n_rows;
-            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
-            for (int c = 0; c < NC && ok; ++c) {
-                gemm1_stages(l, c);
-                if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
-                prev_l = l;
-                prev_c = c;
+            if (q > 0) {
+                const int pl = c ? l_cur : l_last, x = (c ? c - 1 : NC - 1) * C::CH, y = pl * D;
+#pragma unroll
+                for (int i = 0; i < SPG; ++i) {
+                    if (ok && ((n + i) & 1u) == me) {
+                        if constexpr (D == 256) {
+                            ok = stage(n + i, &tm_w2_256, x + 64 * i, -1, y);
+                        } else if constexpr (D == 128) {
+                            ok = stage(n + i, &tm_w2_128, x + 128 * i, x + 128 * i + 64, y);
+                        } else {
+                            // columns 0..255 of Y from two N=256 stages, 256..383 from one N=128 stage
+                            if (i < 2) ok = stage(n + i, &tm_w2_256, x + 64 * i, -1, y);
+                            else ok = stage(n + i, &tm_w2_128, x, x + 64, y + 256);
+                        }
+                    }
+                }
+                n += SPG;
             }
+            if (++c == NC) { c = 0; ++ti; }
         }
-        if (prev_l >= 0) gemm2_stages(prev_l, prev_c);
     } else if (warp == 1 || warp == kIssuerB) {
         // ------------------------------------------------------------------ UMMA issuers
-        // Two warps take the weight stages of the schedule in turn (even / odd stage index).
-        // Each walks the whole schedule converged, waits for its own stage's operands, then for
-        // its turn (all earlier stages issued: the tensor pipe executes in issue order), and
-        // one elected lane issues the stage's UMMAs and commits (a commit tracks the UMMAs of the
-        // thread that issues it; since the pipe is in order, a commit after the last stage of a
-        // GEMM also covers the other issuer's earlier stages).  While one issuer is blocked
-        // issuing into the short UMMA queue, the other does its waiting and bookkeeping, so the
-        // queue does not run dry between stages.
+        // Two warps take the weight stages in turn (even / odd ring position).  Each waits for
+        // its own stage's operands, then for its turn (all earlier stages issued: the tensor
+        // pipe executes in issue order, and the ring's phase parities need in-order use), and
+        // one elected lane issues the stage's UMMAs, passes the turn on and commits.  A commit
+        // tracks the UMMAs of the thread that issues it; since the pipe is in order, a commit
+        // after the last stage of a GEMM also covers the other issuer's earlier stages.  While
+        // one issuer is blocked issuing into the short UMMA queue, the other does its waiting
+        // and bookkeeping, so the queue does not run dry between stages.
         const uint32_t me = (warp == 1) ? 0u : 1u;
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
+        constexpr uint32_t kBlkLo = kBlockBytes >> 4, kStageLo = kStageBytes >> 4;
         const uint32_t tm_h = tmem + C::H_COL0;
+        const uint32_t xs_lo = desc_lo(xs), hs_lo = desc_lo(hs), w_lo = desc_lo(wsm);
         volatile uint32_t* issued = &misc->issued;
-        uint32_t n = 0;   // weight stages walked
-        bool ok = true;
-        auto wait = [&](uint64_t* bar, uint32_t parity) {
-            if (ok) ok = warp_wait(bar, parity, abort_flag);
-            return ok;
-        };
-        auto wait_tmem = [&](uint64_t* bar, uint32_t parity) {   // orders later UMMAs after TMEM reads
-            const bool r = wait(bar, parity);
-            ptx::tc_fence_after_sync();
-            return r;
-        };
-        // this stage's weights have landed and every earlier stage has been issued
-        auto stage_ready = [&]() {
-            if (!wait(&misc->w_full[n % kStages], (n / kStages) & 1u)) return false;
-            for (uint32_t spins = 0; !__all_sync(0xffffffffu, *issued >= n); ++spins) {
-                if (spins > (1u << 22) || *abort_flag) { *abort_flag = 1; ok = false; return false; }
+        // One stage: probe every barrier it needs at once, take the turn, issue, pass the turn
+        // on, commit.  wb*: barriers to wait on besides the weights (0 = none), cb*: barriers to
+        // commit to besides w_empty (0 = none); a_lo1 != 0: the stage holds two K blocks.
+        auto stage = [&](uint32_t n, uint32_t d_tm, uint32_t a_lo0, uint32_t a_lo1, uint32_t idesc, bool overwrite,
+                         uint32_t wb0, uint32_t wp0, uint32_t wb1, uint32_t wp1, uint32_t wb2, uint32_t wp2,
+                         bool tmem_guard, uint32_t cb0, uint32_t cb1, uint32_t cb2) -> bool {
+            const uint32_t sl = n % kStages, ph = (n / kStages) & 1u;
+            const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
+            bool p = ptx::mbar_try_wait(wf, ph);
+            if (wb0 != 0u) p &= ptx::mbar_try_wait(wb0, wp0);
+            if (wb1 != 0u) p &= ptx::mbar_try_wait(wb1, wp1);
+            if (wb2 != 0u) p &= ptx::mbar_try_wait(wb2, wp2);
+            if (!__all_sync(0xffffffffu, p) &&
+                !__all_sync(0xffffffffu, wait_each_slow(wf, ph, wb0, wp0, wb1, wp1, wb2, wp2, abort_flag)))
+                return false;
+            if (tmem_guard) ptx::tc_fence_after_sync();   // orders the UMMAs after the epilogue's TMEM reads
+            if (!__all_sync(0xffffffffu, *issued >= n) &&
+                !__all_sync(0xffffffffu, turn_wait_slow(issued, n, abort_flag)))
+                return false;
+            if (elect_one()) {
+                const uint32_t b_lo = w_lo + sl * kStageLo;
+                mma_kblock_lo(d_tm, a_lo0, b_lo, idesc, overwrite ? 0u : 1u);
+                if (a_lo1 != 0u) mma_kblock_lo(d_tm, a_lo1, b_lo + kBlkLo, idesc, 1u);
+                *issued = n + 1;
+                if (cb0 != 0u) ptx::umma_commit(cb0);
+                if (cb1 != 0u) ptx::umma_commit(cb1);
+                ptx::umma_commit(MISC_BAR(mb, w_empty) + 8u * sl);
+                if (cb2 != 0u) ptx::umma_commit(cb2);
             }
+            __syncwarp();
             return true;
         };
-        auto bar_of = [&](uint64_t* b) { return ptx::smem_u32(b); };
-        // GEMM1 of global chunk g = chunk c of local tile ti:  H = X . W1c_chunk^T
-        auto gemm1 = [&](uint32_t g, int c, uint32_t ti) {
-            const bool last = (c == NC - 1);
-            if constexpr (D == 384) {
-                for (int kp = 0; kp < 3 && ok; ++kp, ++n) {
-                    if ((n & 1u) != me) continue;
-                    if (kp == 0 && !wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
-                    const uint32_t s0 = 2 * kp, s1 = 2 * kp + 1;   // X slots (NXS = KB1 = 6)
-                    if (c == 0 && (!wait(&misc->x_full[s0], ti & 1u) || !wait(&misc->x_full[s1], ti & 1u))) return;
-                    if (!stage_ready()) return;
-                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) {
-                        mma_kblock(tm_h, xs + s0 * kBlockBytes, b, idesc128, kp == 0);
-                        mma_kblock(tm_h, xs + s1 * kBlockBytes, b + kBlockBytes, idesc128, false);
-                        *issued = n + 1;
-                        if (last) {
-                            ptx::umma_commit(bar_of(&misc->x_empty[s0]));
-                            ptx::umma_commit(bar_of(&misc->x_empty[s1]));
-                        }
-                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
-                        if (kp == 2) ptx::umma_commit(bar_of(&misc->h_full));
-                    }
-                    __syncwarp();
-                }
-            } else {
-                for (int kb = 0; kb < C::KB1 && ok; ++kb, ++n) {
-                    if ((n & 1u) != me) continue;
-                    if (kb == 0 && !wait_tmem(&misc->h_tmem_empty, (g & 1u) ^ 1u)) return;
-                    const uint32_t gx = ti * C::KB1 + kb, slot = gx % C::NXS;
-                    if (c == 0 && !wait(&misc->x_full[slot], (gx / C::NXS) & 1u)) return;
-                    if (!stage_ready()) return;
-                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) {
-                        mma_kblock(tm_h, xs + slot * kBlockBytes, b, idesc256, kb == 0);
-                        *issued = n + 1;
-                        if (last) ptx::umma_commit(bar_of(&misc->x_empty[slot]));
-                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
-                        if (kb == C::KB1 - 1) ptx::umma_commit(bar_of(&misc->h_full));
-                    }
-                    __syncwarp();
-                }
-            }
-        };
-        // GEMM2 of global chunk g:  Y (+)= gelu(H) . W2c_chunk
-        auto gemm2 = [&](uint32_t g, int c, uint32_t ti) {
-            const bool first = (c == 0), last = (c == NC - 1);
-            if constexpr (D == 256) {
-                for (int kb2 = 0; kb2 < 4 && ok; ++kb2, ++n) {
-                    if ((n & 1u) != me) continue;
-                    if (!wait(&misc->hs_full[kb2], g & 1u)) return;
-                    if (first && kb2 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                    if (!stage_ready()) return;
-                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) {
-                        mma_kblock(tmem, hs + kb2 * kBlockBytes, b, idesc256, first && kb2 == 0);
-                        *issued = n + 1;
-                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
-                        ptx::umma_commit(bar_of(&misc->hs_empty[kb2]));
-                        if (last && kb2 == 3) ptx::umma_commit(bar_of(&misc->y_full));
-                    }
-                    __syncwarp();
-                }
-            } else if constexpr (D == 128) {
-                for (int kp = 0; kp < 2 && ok; ++kp, ++n) {
-                    if ((n & 1u) != me) continue;
-                    const int k0 = 2 * kp, k1 = 2 * kp + 1;
-                    if (!wait(&misc->hs_full[k0], g & 1u) || !wait(&misc->hs_full[k1], g & 1u)) return;
-                    if (first && kp == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
-                    if (!stage_ready()) return;
-                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) {
-                        mma_kblock(tmem, hs + k0 * kBlockBytes, b, idesc128, first && kp == 0);
-                        mma_kblock(tmem, hs + k1 * kBlockBytes, b + kBlockBytes, idesc128, false);
-                        *issued = n + 1;
-                        ptx::umma_commit(bar_of(&misc->hs_empty[k0]));
-                        ptx::umma_commit(bar_of(&misc->hs_empty[k1]));
-                        ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
-                        if (last && kp == 1) ptx::umma_commit(bar_of(&misc->y_full));
-                    }
-                    __syncwarp();
-                }
-            } else {
-                // columns 0..255 of Y from two N=256 stages, columns 256..383 from one N=128 stage
-                for (int st3 = 0; st3 < 3 && ok; ++st3, ++n) {
-                    if ((n & 1u) != me) continue;
-                    if (st3 < 2) {
-                        if (!wait(&misc->hs_full[st3], g & 1u)) return;
-                        if (first && st3 == 0 && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+        uint32_t n = 0, ti = 0;
+        bool ok = true;
+        int c = 0;
+#pragma unroll 1
+        for (uint32_t q = 0; q <= n_chunks && ok; ++q) {
+            if (q < n_chunks) {
+                // GEMM1 of chunk q = chunk c of local tile ti:  H = X . W1c_chunk^T
+                const bool last = (c == NC - 1), first = (c == 0);
+                const uint32_t hp = (q & 1u) ^ 1u;
+#pragma unroll
+                for (int i = 0; i < SPG; ++i) {
+                    if (!ok || ((n + i) & 1u) != me) continue;
+                    const uint32_t he = (i == 0) ? MISC_BAR(mb, h_tmem_empty) : 0u;
+                    const uint32_t hf = (i == SPG - 1) ? MISC_BAR(mb, h_full) : 0u;
+                    if constexpr (D == 384) {
+                        const uint32_t s0 = 2 * i, s1 = 2 * i + 1;   // X slots (NXS = KB1 = 6)
+                        ok = stage(n + i, tm_h, xs_lo + s0 * kBlkLo, xs_lo + s1 * kBlkLo, idesc128, i == 0,
+                                   first ? MISC_BAR(mb, x_full) + 8u * s0 : 0u, ti & 1u,
+                                   first ? MISC_BAR(mb, x_full) + 8u * s1 : 0u, ti & 1u, he, hp, i == 0,
+                                   last ? MISC_BAR(mb, x_empty) + 8u * s0 : 0u,
+                                   last ? MISC_BAR(mb, x_empty) + 8u * s1 : 0u, hf);
                     } else {
-                        // both hidden blocks (and, on the first chunk, Y's release) are needed here too
-                        if (!wait(&misc->hs_full[0], g & 1u) || !wait(&misc->hs_full[1], g & 1u)) return;
-                        if (first && !wait_tmem(&misc->y_empty, (ti & 1u) ^ 1u)) return;
+                        const uint32_t gx = ti * C::KB1 + i, slot = gx % C::NXS;
+                        ok = stage(n + i, tm_h, xs_lo + slot * kBlkLo, 0u, idesc256, i == 0,
+                                   first ? MISC_BAR(mb, x_full) + 8u * slot : 0u, (gx / C::NXS) & 1u, 0u, 0u, he, hp,
+                                   i == 0, last ? MISC_BAR(mb, x_empty) + 8u * slot : 0u, 0u, hf);
                     }
-                    if (!stage_ready()) return;
-                    const uint32_t b = wsm + (n % kStages) * kStageBytes;
-                    if (elect_one()) {
-                        if (st3 < 2) {
-                            mma_kblock(tmem, hs + st3 * kBlockBytes, b, idesc256, first && st3 == 0);
-                            *issued = n + 1;
-                            ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
+                }
+                n += SPG;
+            }
+            if (q > 0 && ok) {
+                // GEMM2 of chunk q-1 = chunk pc of local tile pti:  Y (+)= gelu(H) . W2c_chunk
+                const int pc = c ? c - 1 : NC - 1;
+                const uint32_t pti = c ? ti : ti - 1, gp = (q - 1) & 1u;
+                const bool first = (pc == 0), last = (pc == NC - 1);
+                const uint32_t ye = first ? MISC_BAR(mb, y_empty) : 0u, yp = (pti & 1u) ^ 1u;
+                const uint32_t yf = last ? MISC_BAR(mb, y_full) : 0u;
+#pragma unroll
+                for (int i = 0; i < SPG; ++i) {
+                    if (!ok || ((n + i) & 1u) != me) continue;
+                    if constexpr (D == 256) {
+                        ok = stage(n + i, tmem, hs_lo + i * kBlkLo, 0u, idesc256, first && i == 0,
+                                   MISC_BAR(mb, hs_full) + 8u * i, gp, 0u, 0u, i == 0 ? ye : 0u, yp, first && i == 0,
+                                   MISC_BAR(mb, hs_empty) + 8u * i, 0u, i == SPG - 1 ? yf : 0u);
+                    } else if constexpr (D == 128) {
+                        const int k0 = 2 * i, k1 = 2 * i + 1;
+                        ok = stage(n + i, tmem, hs_lo + k0 * kBlkLo, hs_lo + k1 * kBlkLo, idesc128, first && i == 0,
+                                   MISC_BAR(mb, hs_full) + 8u * k0, gp, MISC_BAR(mb, hs_full) + 8u * k1, gp,
+                                   i == 0 ? ye : 0u, yp, first && i == 0, MISC_BAR(mb, hs_empty) + 8u * k0,
+                                   MISC_BAR(mb, hs_empty) + 8u * k1, i == SPG - 1 ? yf : 0u);
+                    } else {
+                        // columns 0..255 of Y from two N=256 stages, columns 256..383 from one N=128
+                        // stage that needs both hidden blocks (and, on the first chunk, Y's release)
+                        if (i < 2) {
+                            ok = stage(n + i, tmem, hs_lo + i * kBlkLo, 0u, idesc256, first && i == 0,
+                                       MISC_BAR(mb, hs_full) + 8u * i, gp, 0u, 0u, i == 0 ? ye : 0u, yp,
+                                       first && i == 0, 0u, 0u, 0u);
                         } else {
-                            mma_kblock(tmem + 256, hs, b, idesc128, first);
-                            mma_kblock(tmem + 256, hs + kBlockBytes, b + kBlockBytes, idesc128, false);
-                            *issued = n + 1;
-                            ptx::umma_commit(bar_of(&misc->w_empty[n % kStages]));
-                            ptx::umma_commit(bar_of(&misc->hs_empty[0]));
-                            ptx::umma_commit(bar_of(&misc->hs_empty[1]));
-                            if (last) ptx::umma_commit(bar_of(&misc->y_full));
+                            ok = stage(n + i, tmem + 256, hs_lo, hs_lo + kBlkLo, idesc128, first,
+                                       MISC_BAR(mb, hs_full), gp, MISC_BAR(mb, hs_full) + 8u, gp, ye, yp, first,
+                                       MISC_BAR(mb, hs_empty), MISC_BAR(mb, hs_empty) + 8u, yf);
                         }
                     }
-                    __syncwarp();
                 }
+                n += SPG;
             }
-        };
-        uint32_t g = 0, ti = 0;
-        bool have_prev = false;
-        uint32_t prev_g = 0, prev_ti = 0;
-        int prev_c = 0;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
-            for (int c = 0; c < NC && ok; ++c, ++g) {
-                gemm1(g, c, ti);
-                if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
-                have_prev = true;
-                prev_g = g; prev_c = c; prev_ti = ti;
-            }
+            if (++c == NC) { c = 0; ++ti; }
         }
-        if (ok && have_prev) gemm2(prev_g, prev_c, prev_ti);
     } else if (warp >= kLoaderWarp0 && warp < kEpiWarp0) {
         // ------------------------------------------------------------------ X row gather
         // Thread -> 8 (row, 16-byte chunk) pairs of every 128 x 64 block.  Up to three blocks
