@@ -341,6 +341,78 @@ __device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k
     __syncwarp();
 }
 
+// The same selection for the rk <= kMaxRK heads of a group at once, by the whole block: all
+// threads count digits for every head (the long part), warp hh then picks head hh's digit, and
+// at the end compacts head hh's selection.  keys: [rk][stride] order keys, n per head;
+// hist: kMaxRK * 256 ints of shared memory.
+__device__ inline void block_select_topk_heads(const uint32_t* keys, int stride, int n, int k, int rk,
+                                               int32_t (*out)[kMaxActive], const uint16_t* remap, int* hist) {
+    __shared__ uint32_t s_sel[2 * kMaxRK];   // per head: fixed key prefix, entries still wanted
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x < rk) { s_sel[2 * threadIdx.x] = 0u; s_sel[2 * threadIdx.x + 1] = (uint32_t)k; }
+    uint32_t fixed = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < rk * 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        for (int hh = 0; hh < rk; ++hh) {
+            const uint32_t prefix = s_sel[2 * hh];
+            const uint32_t* kh = keys + (size_t)hh * stride;
+            int* hh_hist = hist + hh * 256;
+            for (int i = threadIdx.x; i < n; i += blockDim.x) {
+                const uint32_t key = kh[i];
+                if ((key & fixed) == prefix) atomicAdd(&hh_hist[(key >> shift) & 255u], 1);
+            }
+        }
+        __syncthreads();
+        if (warp < rk) {
+            const int* h = hist + warp * 256;
+            const int want = (int)s_sel[2 * warp + 1];
+            const int top = 255 - 8 * lane;      // this lane's digits, descending
+            int mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mine += h[top - j];
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const int above = incl - mine;
+            if (above < want && want <= incl) {   // exactly one lane
+                int acc = above;
+                for (int j = 0; j < 8; ++j) {
+                    const int cdig = h[top - j];
+                    if (want <= acc + cdig) {
+                        s_sel[2 * warp] |= (uint32_t)(top - j) << shift;
+                        s_sel[2 * warp + 1] = (uint32_t)(want - acc);
+                        break;
+                    }
+                    acc += cdig;
+                }
+            }
+        }
+        fixed |= 255u << shift;
+        __syncthreads();
+    }
+    if (warp < rk) {
+        const uint32_t* kh = keys + (size_t)warp * stride;
+        const uint32_t t = s_sel[2 * warp];
+        const int need_eq = (int)s_sel[2 * warp + 1];
+        int base = 0, eq_seen = 0;
+        for (int i0 = 0; i0 < n; i0 += 32) {
+            const int i = i0 + lane;
+            const uint32_t key = i < n ? kh[i] : 0u;
+            const bool is_eq = i < n && key == t, is_gt = i < n && key > t;
+            const unsigned em = __ballot_sync(0xffffffffu, is_eq);
+            const bool keep = is_gt || (is_eq && eq_seen + __popc(em & ((1u << lane) - 1u)) < need_eq);
+            const unsigned km = __ballot_sync(0xffffffffu, keep);
+            if (keep) out[warp][base + __popc(km & ((1u << lane) - 1u))] = (int32_t)remap[i];
+            base += __popc(km);
+            eq_seen += __popc(em);
+        }
+    }
+}
+
 template <int D>
 struct CoreSmem {
     static constexpr int TILE_BYTES = kKeyTile * D * 2;      // one K or V tile
@@ -872,8 +944,8 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
             for (int i = threadIdx.x; i < rk * Tlen; i += blockDim.x) s_keys[i] = 0u;
         }
         __syncthreads();
-        // ---- the U present queries with the largest score are active: one warp per head
-        if (warp < rk) warp_select_topk_radix(s_keys + (size_t)warp * Tlen, Tv, U, s_act[warp], s_valid, s_hist + warp * 256);
+        // ---- the U present queries with the largest score are active
+        block_select_topk_heads(s_keys, Tlen, Tv, U, rk, s_act, s_valid, s_hist);
         __syncthreads();
         if (active_out != nullptr)
             for (int i = threadIdx.x; i < rk * U_max; i += blockDim.x) {
