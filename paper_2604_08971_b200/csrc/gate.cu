@@ -46,6 +46,21 @@ gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
     }
     if (fan_masks == nullptr) return;
     __syncthreads();   // out[] (global, written by this block) is complete
+    if (k <= 32) {
+        // short lists (heads): one thread per mask -- one independent load of the mask per
+        // thread instead of a chain of dependent loads down an element loop
+        for (int m = threadIdx.x; m < n_masks; m += blockDim.x) {
+            const uint32_t ms = fan_masks[m];
+            if (ms == (uint32_t)s) {
+                int32_t* dst = kept + (size_t)m * k;
+                for (int j = 0; j < k; ++j) dst[j] = out[j];
+                if (kv_groups != nullptr) kv_groups[m] = s_bits;
+            } else if (s == 0 && ms >= (uint32_t)S) {
+                atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+            }
+        }
+        return;
+    }
     const long long total = (long long)n_masks * k;
     for (long long i = threadIdx.x; i < total; i += blockDim.x) {
         const int m = (int)(i / k), j = (int)(i % k);
@@ -91,8 +106,12 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const size_t total = (size_t)n_masks * k;
     if (total <= 16384) {   // small fan-out: one launch does both steps
+        // enough threads for the fan-out as well as for the selection
+        int threads = gate_threads(n_units);
+        const int fan = k <= 32 ? n_masks : (int)(total < 1024 ? total : 1024);
+        while (threads < 256 && threads < fan) threads *= 2;
         LaunchScope ls(ctx, KS_GATE_ROWS, st);
-        gate_rows_kernel<<<S, gate_threads(n_units), smem, st>>>(
+        gate_rows_kernel<<<S, threads, smem, st>>>(
             scores, n_units, k, ws_rows, kv_groups ? ws_groups : nullptr,
             heads_per_group > 0 ? heads_per_group : 1, masks, n_masks, S, kept, kv_groups, ctx->d_status);
         SENTRY_CUDA_TRY(cudaGetLastError());
