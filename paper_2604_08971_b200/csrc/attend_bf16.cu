@@ -31,6 +31,7 @@ constexpr int kCoreThreads = 256;
 constexpr int kCoreWarps = kCoreThreads / 32;
 constexpr int kKeyTile = 64;
 constexpr int kMaxActive = 48;
+constexpr int kSmallT = 256;   // fused attention: sequences up to this length run in 128-thread CTAs
 constexpr int kOrderMaxBatch = 1024; // batches up to this size are walked heaviest-sample-first     // U <= 45 for T <= 8103 with c = 5 (checked on the host)
 
 // Row layout in shared memory: rows of D bf16, 16-byte chunks XOR-swizzled so that both
@@ -1152,7 +1153,9 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
         // the group's K and V fit in shared memory: one kernel does everything
         auto kern = attend_fused_bf16_kernel<D>;
         SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused_bytes));
-        const int threads = fused_bytes > 100 * 1024 ? 512 : 256;   // one big CTA or two per SM
+        // one big CTA, or two per SM; short sequences get small CTAs (more of them per SM: their
+        // phases are a few barrier-separated microseconds each, so concurrency is what helps)
+        const int threads = fused_bytes > 100 * 1024 ? 512 : (d.T <= kSmallT ? 128 : 256);
         LaunchScope ls(ctx, KS_ATT_CORE, st);
         kern<<<d.B * d.Hk, threads, fused_bytes, st>>>(
             (const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, a.kept_heads,
