@@ -28,6 +28,7 @@
 
 #include "common.cuh"
 #include "ffn_plan.cuh"
+#include "ffn_tc_common.cuh"
 #include "ptx/sm100.cuh"
 
 namespace {
@@ -69,69 +70,6 @@ struct Misc {
     uint32_t issued;   // weight stages whose UMMAs have been issued (turn counter of the two issuers)
 };
 static_assert(sizeof(Misc) <= 2048, "misc block too large");
-
-// gelu(z) = z/2 (1 + erf(z / sqrt 2)) = relu(z) - |z|/2 * erfc(|z| / sqrt 2).
-// erfc(x) = 2^(-q(x)), q = -log2(erfc): q(|z|/sqrt 2) is fitted by |z| times a quartic in |z|
-// (weighted least squares pushed towards minimax on |z| <= 4 sqrt 2, where erfc is below 2e-8;
-// beyond, |z| is clamped).  Largest error of gelu over all z: 7e-7, far below the resolution
-// of the bf16 value that is stored.  One special-function operation per element.
-// Coefficients of the quartic, highest power first: 4.880980979e-04, -7.198737003e-03,
-// 5.214667618e-02, 4.595957994e-01, 1.151000593e+00.
-// Evaluated on two values at once with the packed fp32 instructions of sm_100 (two lanes of a
-// 64-bit register per instruction), result rounded to a bf16 pair: 7 instead of 11 issue slots
-// per element, which matters because the GELU epilogue competes with the UMMA issuers for them.
-__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint32_t gelu_erf_fast_bf16x2(float z0, float z1) {
-    const float a0 = fminf(fabsf(z0), 5.65685424949f), a1 = fminf(fabsf(z1), 5.65685424949f);
-    const uint64_t A = f32x2(a0, a1);
-    uint64_t P = fma_f32x2(f32x2(4.880980979e-04f, 4.880980979e-04f), A, f32x2(-7.198737003e-03f, -7.198737003e-03f));
-    P = fma_f32x2(P, A, f32x2(5.214667618e-02f, 5.214667618e-02f));
-    P = fma_f32x2(P, A, f32x2(4.595957994e-01f, 4.595957994e-01f));
-    P = fma_f32x2(P, A, f32x2(1.151000593e+00f, 1.151000593e+00f));
-    const uint64_t Qn = fma_f32x2(P, A, f32x2(0.f, 0.f));            // q = p * a
-    float q0, q1, y0, y1;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(q0), "=f"(q1) : "l"(Qn));
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y0) : "f"(-q0));
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y1) : "f"(-q1));
-    // relu(z) - (a/2) * erfc: beyond the clamp erfc < 2e-8, so a stands in for |z|
-    const uint64_t H = fma_f32x2(A, f32x2(-0.5f, -0.5f), f32x2(0.f, 0.f));
-    const uint64_t G = fma_f32x2(H, f32x2(y0, y1), f32x2(fmaxf(z0, 0.0f), fmaxf(z1, 0.0f)));
-    float g0, g1;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(g0), "=f"(g1) : "l"(G));
-    __nv_bfloat162 v = __floats2bfloat162_rn(g0, g1);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-
-__device__ __forceinline__ void cp_async_wait_pending(int n) {
-    if (n <= 0) ptx::cp_async_wait_group<0>();
-    else if (n == 1) ptx::cp_async_wait_group<1>();
-    else ptx::cp_async_wait_group<2>();
-}
-
-// Bounded wait by every lane of a warp; the result is the same in all lanes.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    const bool ok = ptx::mbar_wait(ptx::smem_u32(bar), parity, abort_flag);
-    return __all_sync(0xffffffffu, ok);
-}
-// One arrival for the whole warp, after every lane has reached this point.
-__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
-    __syncwarp();
-    if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(bar));
-}
 
 // ---- lean forms for the single-thread roles -------------------------------------------------
 // A warp that walks a chain of dependent scalar instructions with shared-memory round trips in
@@ -177,21 +115,6 @@ static __device__ __noinline__ bool turn_wait_slow(volatile uint32_t* issued, ui
     }
     return true;
 }
-
-// One lane of a fully converged warp.  The single-thread instructions (TMA, UMMA, commit) are
-// issued from inside `if (elect_one())` while the whole warp walks the schedule: operands
-// computed by all lanes stay warp-uniform, which about halves the cost of issuing them
-// compared with a lane-0 branch around the whole loop.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "elect.sync _|p, 0xffffffff;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(pred));
-    return pred != 0;
-}
-
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -504,37 +427,52 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         auto drain_y = [&](uint32_t t_idx, int32_t grow) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
-#pragma unroll 1
-            for (int pass = 0; pass < D / 128; ++pass) {
-                const int col0 = half * (D / 2) + pass * 64;
-#pragma unroll 1
-                for (int sub = 0; sub < 2; ++sub) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(lane_base + col0 + sub * 32, r);
-                    ptx::tmem_ld_wait();
+            // 64 columns per pass.  The TMEM loads of the next pass are in flight while this pass's
+            // rows go out, and the row numbers of the store steps are fetched once.
+            constexpr int NP = D / 128;
+            const int ch = lane & 7;
+            int32_t grs[8];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t dst = stg + lane * 128 + (((4 * sub + i) ^ (lane & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
-                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1]))),
-                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]))),
-                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]))),
-                                     "r"(pack_bf16x2(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])))
-                                     : "memory");
-                    }
+            for (int step = 0; step < 8; ++step) grs[step] = __shfl_sync(0xffffffffu, grow, step * 4 + (lane >> 3));
+            __nv_bfloat16* ycol = Y + half * (D / 2) + ch * 8;
+            uint32_t ra[32], rb[32];
+            ptx::tmem_ld_32x32(lane_base + half * (D / 2), ra);
+            ptx::tmem_ld_32x32(lane_base + half * (D / 2) + 32, rb);
+            ptx::tmem_ld_wait();
+#pragma unroll 1
+            for (int pass = 0; pass < NP; ++pass) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + ((i ^ (lane & 7)) << 4)),
+                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i]), __uint_as_float(ra[8 * i + 1]))),
+                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i + 2]), __uint_as_float(ra[8 * i + 3]))),
+                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i + 4]), __uint_as_float(ra[8 * i + 5]))),
+                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i + 6]), __uint_as_float(ra[8 * i + 7])))
+                                 : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((4 + i) ^ (lane & 7)) << 4)),
+                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i]), __uint_as_float(rb[8 * i + 1]))),
+                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 2]), __uint_as_float(rb[8 * i + 3]))),
+                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 4]), __uint_as_float(rb[8 * i + 5]))),
+                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 6]), __uint_as_float(rb[8 * i + 7])))
+                                 : "memory");
+                }
+                if (pass + 1 < NP) {
+                    const int col1 = half * (D / 2) + (pass + 1) * 64;
+                    ptx::tmem_ld_32x32(lane_base + col1, ra);
+                    ptx::tmem_ld_32x32(lane_base + col1 + 32, rb);
                 }
                 __syncwarp();
 #pragma unroll
                 for (int step = 0; step < 8; ++step) {
-                    const int rr = step * 4 + (lane >> 3), ch = lane & 7;
+                    const int rr = step * 4 + (lane >> 3);
                     uint4 v;
                     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                                  : "r"(stg + rr * 128 + ((ch ^ (rr & 7)) << 4)));
-                    const int32_t gr = __shfl_sync(0xffffffffu, grow, rr);
-                    if (gr >= 0) *reinterpret_cast<uint4*>(Y + (size_t)gr * D + col0 + ch * 8) = v;
+                    if (grs[step] >= 0) *reinterpret_cast<uint4*>(ycol + (size_t)grs[step] * D + pass * 64) = v;
                 }
                 __syncwarp();
+                if (pass + 1 < NP) ptx::tmem_ld_wait();
             }
             ptx::tc_fence_before_sync();
             warp_arrive(&misc->y_empty);
@@ -551,6 +489,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 for (int j = 0; j < C::NBATCH && ok; ++j) {
                     // 32 rows x 64 columns of the hidden accumulator -> registers
                     const int blk = half * C::NBATCH + j;        // hidden block = 64 channels
+                    // Y of the previous tile is complete about now (its last GEMM2 was queued right
+                    // after this tile's first GEMM1): store it before this warp's last batch of the
+                    // chunk is loaded, while no accumulator values are held in registers
+                    if (j == C::NBATCH - 1 && c == 0 && ti > 0) {
+                        drain_y((uint32_t)(ti - 1), prev_row);
+                        if (!ok) break;
+                    }
                     uint32_t h0[32], h1[32];
                     const uint32_t tcol = lane_base + C::H_COL0 + blk * 64;
                     ptx::tmem_ld_32x32(tcol, h0);
@@ -560,12 +505,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                         // the accumulator is in registers: GEMM1 of the next chunk may start
                         ptx::tc_fence_before_sync();
                         warp_arrive(&misc->h_tmem_empty);
-                        // the previous tile's Y is complete about now (its last GEMM2 was queued
-                        // right after this chunk's GEMM1): store it before the arithmetic
-                        if (c == 0 && ti > 0) {
-                            drain_y(ti - 1, prev_row);
-                            if (!ok) break;
-                        }
                     }
                     uint32_t pk[32];
 #pragma unroll
@@ -604,36 +543,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem, kTmemCols);
     }
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
-// bf16 row-major [rows, cols] -> map with a box of `box_rows` rows x 64 columns, 128-byte swizzle.
-bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (fn == nullptr) return false;
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int D>

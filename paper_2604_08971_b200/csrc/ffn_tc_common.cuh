@@ -1,0 +1,116 @@
+// Pieces shared by the tcgen05 FFN kernels: the GELU epilogue arithmetic, warp-level barrier
+// helpers, single-lane election and the TMA tensor-map encoder.
+#pragma once
+#include <cuda.h>
+#include <math.h>
+
+#include "common.cuh"
+#include "ptx/sm100.cuh"
+
+namespace {
+
+// gelu(z) = z/2 (1 + erf(z / sqrt 2)), with erf(z / sqrt 2) evaluated as tanh(z (c1 + c2 z^2)) on the
+// hardware tanh (one special-function operation per element).  c1 = 0.7985835, c2 = 0.03538746:
+// own fit that minimises the largest error relative to gelu(|z|) -- 1.5e-4 of gelu(|z|) for every
+// z (checked against scipy.special.erf on 160 k points); the tanh unit adds at most 2^-11 of its
+// result, i.e. 2.4e-4 |z|.  Both are more than ten times below the rounding of the bf16 value
+// that is stored (2^-9 of it).  Both coefficients are positive, so z (c1 + c2 z^2) is monotone
+// and saturates the tanh for large |z| without a clamp.
+// Evaluated on two values at once with the packed fp32 instructions of sm_100 (two lanes of a
+// 64-bit register per instruction), result rounded to a bf16 pair: 4.5 issue slots per element,
+// which matters because the GELU epilogue is what the tensor pipe ends up waiting for.
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t gelu_erf_fast_bf16x2(float z0, float z1) {
+    const uint64_t Z = f32x2(z0, z1), zero = f32x2(0.f, 0.f);
+    const uint64_t Z2 = fma_f32x2(Z, Z, zero);
+    const uint64_t P = fma_f32x2(Z2, f32x2(0.03538746f, 0.03538746f), f32x2(0.7985835f, 0.7985835f));
+    const uint64_t U = fma_f32x2(P, Z, zero);
+    float u0, u1, t0, t1;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(u0), "=f"(u1) : "l"(U));
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t0) : "f"(u0));
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(u1));
+    const uint64_t H = fma_f32x2(Z, f32x2(0.5f, 0.5f), zero);
+    const uint64_t G = fma_f32x2(H, f32x2(t0, t1), H);
+    float g0, g1;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(g0), "=f"(g1) : "l"(G));
+    __nv_bfloat162 v = __floats2bfloat162_rn(g0, g1);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ void cp_async_wait_pending(int n) {
+    if (n <= 0) ptx::cp_async_wait_group<0>();
+    else if (n == 1) ptx::cp_async_wait_group<1>();
+    else ptx::cp_async_wait_group<2>();
+}
+
+// Bounded wait by every lane of a warp; the result is the same in all lanes.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    const bool ok = ptx::mbar_wait(ptx::smem_u32(bar), parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
+}
+// One arrival for the whole warp, after every lane has reached this point.
+__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(bar));
+}
+
+// One lane of a fully converged warp.  The single-thread instructions (TMA, UMMA, commit) are
+// issued from inside `if (elect_one())` while the whole warp walks the schedule: operands
+// computed by all lanes stay warp-uniform, which about halves the cost of issuing them
+// compared with a lane-0 branch around the whole loop.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 row-major [rows, cols] -> map with a box of `box_rows` rows x 64 columns, 128-byte swizzle.
+bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
