@@ -342,6 +342,59 @@ __device__ inline void warp_select_topk_radix(const uint32_t* keys, int n, int k
     __syncwarp();
 }
 
+// Top-k of n <= 32 * KPL order keys by ONE warp with the keys in registers (lane l holds keys
+// l, l + 32, ...): the k-th largest key is built bit by bit from the top (a candidate bit stays
+// set if at least k keys are >= the candidate: 32 steps of KPL compares and one warp add), then
+// the entries above it and the first ties are compacted in ascending index order.  No shared-
+// memory histograms, no atomics and no block barriers.
+template <int KPL>
+__device__ __forceinline__ void warp_select_topk_bits(const uint32_t* keys, int n, int k, int32_t* out,
+                                                      const uint16_t* remap) {
+    const int lane = threadIdx.x & 31;
+    uint32_t r[KPL];
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+        const int i = j * 32 + lane;
+        r[j] = i < n ? keys[i] : 0u;     // padding: below every candidate (candidates are >= 1)
+    }
+    uint32_t t = 0;
+#pragma unroll 1
+    for (int b = 31; b >= 0; --b) {
+        const uint32_t cand = t | (1u << b);
+        int cnt = 0;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) cnt += (r[j] >= cand) ? 1 : 0;
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (cnt >= k) t = cand;
+    }
+    // t is the k-th largest key (0 only if fewer than k keys are non-zero: then every entry ties)
+    int gt = 0;
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) gt += (r[j] > t) ? 1 : 0;
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    const int need_eq = k - gt;
+    int base = 0, eq_seen = 0;
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+        if (j * 32 >= n) break;          // warp-uniform
+        const int i = j * 32 + lane;
+        const bool is_eq = i < n && r[j] == t, is_gt = i < n && r[j] > t;
+        const unsigned em = __ballot_sync(0xffffffffu, is_eq);
+        const bool keep = is_gt || (is_eq && eq_seen + __popc(em & ((1u << lane) - 1u)) < need_eq);
+        const unsigned km = __ballot_sync(0xffffffffu, keep);
+        if (keep) out[base + __popc(km & ((1u << lane) - 1u))] = (int32_t)remap[i];
+        base += __popc(km);
+        eq_seen += __popc(em);
+    }
+    __syncwarp();
+}
+// Warp hh selects for head hh (keys [rk][stride], n <= 256 per head).
+__device__ __forceinline__ void warps_select_topk_heads(const uint32_t* keys, int stride, int n, int k, int rk,
+                                                        int32_t (*out)[kMaxActive], const uint16_t* remap) {
+    const int warp = threadIdx.x >> 5;
+    if (warp < rk) warp_select_topk_bits<8>(keys + (size_t)warp * stride, n, k, out[warp], remap);
+}
+
 // The same selection for the rk <= kMaxRK heads of a group at once, by the whole block: all
 // threads count digits for every head (the long part), warp hh then picks head hh's digit, and
 // at the end compacts head hh's selection.  keys: [rk][stride] order keys, n per head;
@@ -946,7 +999,10 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         }
         __syncthreads();
         // ---- the U present queries with the largest score are active
-        block_select_topk_heads(s_keys, Tlen, Tv, U, rk, s_act, s_valid, s_hist);
+        // short lists: one warp per head with the keys in registers; longer ones: digit counting
+        // by the whole block (measured: the warp form wins up to 256 keys, loses from 1024 on)
+        if (Tv <= 256) warps_select_topk_heads(s_keys, Tlen, Tv, U, rk, s_act, s_valid);
+        else block_select_topk_heads(s_keys, Tlen, Tv, U, rk, s_act, s_valid, s_hist);
         __syncthreads();
         if (active_out != nullptr)
             for (int i = threadIdx.x; i < rk * U_max; i += blockDim.x) {

@@ -20,8 +20,9 @@
 // never waits for the GELU epilogue with nothing else queued.
 //
 // Warp roles (512 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
-// warps 1 and 15 = UMMA issuers (alternate stages), warps 3-6 = X row gather, warps 7-14 =
-// epilogue (two warps per TMEM lane quarter).  Producer and issuer warps stay converged and elect one lane per instruction.  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
+// warp 1 = UMMA issuer, warp 15 = its watcher (does the barrier waits), warps 3-6 = X row
+// gather, warps 7-14 = epilogue (two warps per TMEM lane quarter).  Producer and issuer warps stay
+// converged and elect one lane per instruction.  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
 // and unwinds.
 #include <cuda.h>
 #include <math.h>
@@ -67,7 +68,7 @@ struct Misc {
     uint64_t y_full, y_empty;
     uint32_t tmem_base;
     int abort_flag;
-    uint32_t issued;   // weight stages whose UMMAs have been issued (turn counter of the two issuers)
+    uint32_t issued;   // weight stages whose operands the watcher has seen complete (polled by the issuer)
 };
 static_assert(sizeof(Misc) <= 2048, "misc block too large");
 
@@ -108,7 +109,7 @@ static __device__ __noinline__ bool wait_each_slow(uint32_t b0, uint32_t p0, uin
     if (ok && b3 != 0u) ok = ptx::mbar_wait(b3, p3, abort_flag);
     return ok;
 }
-// Slow path of the issuers' turn: poll until `n` stages have been issued, bounded.
+// Slow path of the issuer's poll: until the watcher has published `n` stages, bounded.
 static __device__ __noinline__ bool turn_wait_slow(volatile uint32_t* issued, uint32_t n, volatile int* abort_flag) {
     for (uint32_t spins = 0; *issued < n; ++spins) {
         if (spins > (1u << 22) || *abort_flag) { *abort_flag = 1; return false; }
@@ -244,46 +245,57 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             if (++c == NC) { c = 0; ++ti; }
         }
     } else if (warp == 1 || warp == kIssuerB) {
-        // ------------------------------------------------------------------ UMMA issuers
-        // Two warps take the weight stages in turn (even / odd ring position).  Each waits for
-        // its own stage's operands, then for its turn (all earlier stages issued: the tensor
-        // pipe executes in issue order, and the ring's phase parities need in-order use), and
-        // one elected lane issues the stage's UMMAs, passes the turn on and commits.  A commit
-        // tracks the UMMAs of the thread that issues it; since the pipe is in order, a commit
-        // after the last stage of a GEMM also covers the other issuer's earlier stages.  While
-        // one issuer is blocked issuing into the short UMMA queue, the other does its waiting
-        // and bookkeeping, so the queue does not run dry between stages.
-        const uint32_t me = (warp == 1) ? 0u : 1u;
+        // ------------------------------------------------------- UMMA issuer and its watcher
+        // Both warps walk the same schedule of weight stages.  The watcher (warp kIssuerB) does
+        // the waiting: for every stage it probes the barriers the stage needs (weights landed,
+        // operand blocks written, accumulator released) and then publishes the stage number.
+        // The issuer (warp 1) only polls that number, and one elected lane issues the stage's
+        // UMMAs and commits.  ALL UMMAs therefore come from one thread: the tensor pipe runs the
+        // instructions of one thread in issue order, but nothing orders the instructions of two
+        // threads, and accumulators fed alternately by two issuing warps were summed in an order
+        // that changed from run to run (results differed in the last bit).  The split keeps part
+        // of what two warps were good for: the barrier round trips of the next stage overlap the
+        // issue of the current one.
+        const bool is_issuer = (warp == 1);
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
         constexpr uint32_t kBlkLo = kBlockBytes >> 4, kStageLo = kStageBytes >> 4;
         const uint32_t tm_h = tmem + C::H_COL0;
         const uint32_t xs_lo = desc_lo(xs), hs_lo = desc_lo(hs), w_lo = desc_lo(wsm);
         volatile uint32_t* issued = &misc->issued;
-        // One stage: probe every barrier it needs at once, take the turn, issue, pass the turn
-        // on, commit.  wb*: barriers to wait on besides the weights (0 = none), cb*: barriers to
+        // One stage.  wb*: barriers to wait on besides the weights (0 = none), cb*: barriers to
         // commit to besides w_empty (0 = none); a_lo1 != 0: the stage holds two K blocks.
         auto stage = [&](uint32_t n, uint32_t d_tm, uint32_t a_lo0, uint32_t a_lo1, uint32_t idesc, bool overwrite,
                          uint32_t wb0, uint32_t wp0, uint32_t wb1, uint32_t wp1, uint32_t wb2, uint32_t wp2,
-                         bool tmem_guard, uint32_t cb0, uint32_t cb1, uint32_t cb2) -> bool {
+                         bool /*writes TMEM others read: fenced in every case*/, uint32_t cb0, uint32_t cb1,
+                         uint32_t cb2) -> bool {
             const uint32_t sl = n % kStages, ph = (n / kStages) & 1u;
-            const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
-            bool p = ptx::mbar_try_wait(wf, ph);
-            if (wb0 != 0u) p &= ptx::mbar_try_wait(wb0, wp0);
-            if (wb1 != 0u) p &= ptx::mbar_try_wait(wb1, wp1);
-            if (wb2 != 0u) p &= ptx::mbar_try_wait(wb2, wp2);
-            if (!__all_sync(0xffffffffu, p) &&
-                !__all_sync(0xffffffffu, wait_each_slow(wf, ph, wb0, wp0, wb1, wp1, wb2, wp2, abort_flag)))
+            if (!is_issuer) {
+                // watcher: every barrier of the stage, probed at once, then the stage is published
+                const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
+                bool p = ptx::mbar_try_wait(wf, ph);
+                if (wb0 != 0u) p &= ptx::mbar_try_wait(wb0, wp0);
+                if (wb1 != 0u) p &= ptx::mbar_try_wait(wb1, wp1);
+                if (wb2 != 0u) p &= ptx::mbar_try_wait(wb2, wp2);
+                if (!__all_sync(0xffffffffu, p) &&
+                    !__all_sync(0xffffffffu, wait_each_slow(wf, ph, wb0, wp0, wb1, wp1, wb2, wp2, abort_flag)))
+                    return false;
+                if (elect_one()) {
+                    __threadfence_block();
+                    *issued = n + 1;
+                }
+                __syncwarp();
+                return true;
+            }
+            if (!__all_sync(0xffffffffu, *issued > n) &&
+                !__all_sync(0xffffffffu, turn_wait_slow(issued, n + 1, abort_flag)))
                 return false;
-            if (tmem_guard) ptx::tc_fence_after_sync();   // orders the UMMAs after the epilogue's TMEM reads
-            if (!__all_sync(0xffffffffu, *issued >= n) &&
-                !__all_sync(0xffffffffu, turn_wait_slow(issued, n, abort_flag)))
-                return false;
+            __threadfence_block();
+            ptx::tc_fence_after_sync();   // orders the UMMAs after the epilogue's TMEM reads and operand writes
             if (elect_one()) {
                 const uint32_t b_lo = w_lo + sl * kStageLo;
                 mma_kblock_lo(d_tm, a_lo0, b_lo, idesc, overwrite ? 0u : 1u);
                 if (a_lo1 != 0u) mma_kblock_lo(d_tm, a_lo1, b_lo + kBlkLo, idesc, 1u);
-                *issued = n + 1;
                 if (cb0 != 0u) ptx::umma_commit(cb0);
                 if (cb1 != 0u) ptx::umma_commit(cb1);
                 ptx::umma_commit(MISC_BAR(mb, w_empty) + 8u * sl);
@@ -303,7 +315,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 const uint32_t hp = (q & 1u) ^ 1u;
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
-                    if (!ok || ((n + i) & 1u) != me) continue;
+                    if (!ok) continue;
                     const uint32_t he = (i == 0) ? MISC_BAR(mb, h_tmem_empty) : 0u;
                     const uint32_t hf = (i == SPG - 1) ? MISC_BAR(mb, h_full) : 0u;
                     if constexpr (D == 384) {
@@ -331,7 +343,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 const uint32_t yf = last ? MISC_BAR(mb, y_full) : 0u;
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
-                    if (!ok || ((n + i) & 1u) != me) continue;
+                    if (!ok) continue;
                     if constexpr (D == 256) {
                         ok = stage(n + i, tmem, hs_lo + i * kBlkLo, 0u, idesc256, first && i == 0,
                                    MISC_BAR(mb, hs_full) + 8u * i, gp, 0u, 0u, i == 0 ? ye : 0u, yp, first && i == 0,
@@ -427,20 +439,22 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         auto drain_y = [&](uint32_t t_idx, int32_t grow) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
-            // 64 columns per pass.  The TMEM loads of the next pass are in flight while this pass's
-            // rows go out, and the row numbers of the store steps are fetched once.
+            // 64 columns per pass: two TMEM loads and one wait, bf16 rows through the staging
+            // piece, then whole 128-byte row segments to global memory.  The registers a TMEM
+            // load writes are not named again before its wait.
             constexpr int NP = D / 128;
             const int ch = lane & 7;
             int32_t grs[8];
 #pragma unroll
             for (int step = 0; step < 8; ++step) grs[step] = __shfl_sync(0xffffffffu, grow, step * 4 + (lane >> 3));
             __nv_bfloat16* ycol = Y + half * (D / 2) + ch * 8;
-            uint32_t ra[32], rb[32];
-            ptx::tmem_ld_32x32(lane_base + half * (D / 2), ra);
-            ptx::tmem_ld_32x32(lane_base + half * (D / 2) + 32, rb);
-            ptx::tmem_ld_wait();
 #pragma unroll 1
             for (int pass = 0; pass < NP; ++pass) {
+                uint32_t ra[32], rb[32];
+                const int col0 = half * (D / 2) + pass * 64;
+                ptx::tmem_ld_32x32(lane_base + col0, ra);
+                ptx::tmem_ld_32x32(lane_base + col0 + 32, rb);
+                ptx::tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + ((i ^ (lane & 7)) << 4)),
@@ -456,11 +470,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                                  "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 6]), __uint_as_float(rb[8 * i + 7])))
                                  : "memory");
                 }
-                if (pass + 1 < NP) {
-                    const int col1 = half * (D / 2) + (pass + 1) * 64;
-                    ptx::tmem_ld_32x32(lane_base + col1, ra);
-                    ptx::tmem_ld_32x32(lane_base + col1 + 32, rb);
-                }
                 __syncwarp();
 #pragma unroll
                 for (int step = 0; step < 8; ++step) {
@@ -472,7 +481,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (grs[step] >= 0) *reinterpret_cast<uint4*>(ycol + (size_t)grs[step] * D + pass * 64) = v;
                 }
                 __syncwarp();
-                if (pass + 1 < NP) ptx::tmem_ld_wait();
             }
             ptx::tc_fence_before_sync();
             warp_arrive(&misc->y_empty);

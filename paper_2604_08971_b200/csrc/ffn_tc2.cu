@@ -11,8 +11,8 @@
 // issue, commits by single threads) is spread over twice the arithmetic, and the weight
 // traffic from L2 into shared memory is halved.
 //
-// Who talks to whom.  All UMMAs are issued by the even CTA of the pair (the leader, two issuer
-// warps as in the single-CTA kernel).  Barriers the issuer waits on (weights landed, X block
+// Who talks to whom.  All UMMAs are issued by one thread of the even CTA of the pair (the
+// leader; a second warp does the waiting for it, as in the single-CTA kernel).  Barriers the issuer waits on (weights landed, X block
 // landed, hidden block written, accumulators drained) live in the leader's shared memory and
 // count arrivals from BOTH CTAs: the peer arrives remotely, its TMA copies credit their bytes
 // to the leader's barrier.  Barriers the issuer signals (ring slot free, X slot free, hidden
@@ -20,7 +20,7 @@
 // multicast commit.  No multicast copies anywhere: every CTA loads its own operands.
 //
 // Warp roles per CTA (512 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
-// warps 1 and 15 = UMMA issuers (leader only; idle in the peer), warps 3-6 = X row gather,
+// warp 1 = UMMA issuer, warp 15 = its watcher (leader only; idle in the peer), warps 3-6 = X row gather,
 // warps 7-14 = epilogue.  Every wait is bounded; on expiry the CTA raises
 // SENTRY_STATUS_BIT_TIMEOUT and unwinds, and the pair leaves together.
 #include <cuda.h>
@@ -281,10 +281,12 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
             if (++c == NC) { c = 0; ++ti; }
         }
     } else if ((warp == 1 || warp == kIssuerB) && rank == 0) {
-        // ------------------------------------------------------------------ UMMA issuers
-        // Two warps of the leader take the ring slots in turn (even / odd ring position), as in
-        // the single-CTA kernel; every UMMA runs on both CTAs, every commit goes to both.
-        const uint32_t me = (warp == 1) ? 0u : 1u;
+        // ------------------------------------------------------- UMMA issuer and its watcher
+        // As in the single-CTA kernel: warp kIssuerB of the leader waits for every slot's
+        // barriers and publishes the slot number, one elected lane of warp 1 issues every UMMA
+        // (one issuing thread: a fixed summation order); every UMMA runs on both CTAs, every
+        // commit goes to both.
+        const bool is_issuer = (warp == 1);
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(256, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(256, 128);
         constexpr uint32_t kBlkLo = kBlockBytes >> 4, kSlotLo = kSlotBytes >> 4;
@@ -293,22 +295,32 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
         volatile uint32_t* issued = &misc->issued;
         auto run = [&](uint32_t n, const SlotWork& w) -> bool {
             const uint32_t sl = n % kStages, ph = (n / kStages) & 1u;
-            const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
-            bool p = ptx::mbar_try_wait_cluster(wf, ph);
-#pragma unroll
-            for (int j = 0; j <= kMaxKb; ++j)
-                if (w.wb[j] != 0u) p &= ptx::mbar_try_wait_cluster(w.wb[j], w.wp[j]);
-            if (!__all_sync(0xffffffffu, p)) {
-                bool ok = wait_cluster_slow(wf, ph, abort_flag);
+            if (!is_issuer) {
+                // watcher: every barrier of the slot, probed at once, then the slot is published
+                const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
+                bool p = ptx::mbar_try_wait_cluster(wf, ph);
 #pragma unroll
                 for (int j = 0; j <= kMaxKb; ++j)
-                    if (ok && w.wb[j] != 0u) ok = wait_cluster_slow(w.wb[j], w.wp[j], abort_flag);
-                if (!__all_sync(0xffffffffu, ok)) return false;
+                    if (w.wb[j] != 0u) p &= ptx::mbar_try_wait_cluster(w.wb[j], w.wp[j]);
+                if (!__all_sync(0xffffffffu, p)) {
+                    bool ok = wait_cluster_slow(wf, ph, abort_flag);
+#pragma unroll
+                    for (int j = 0; j <= kMaxKb; ++j)
+                        if (ok && w.wb[j] != 0u) ok = wait_cluster_slow(w.wb[j], w.wp[j], abort_flag);
+                    if (!__all_sync(0xffffffffu, ok)) return false;
+                }
+                if (elect_one()) {
+                    __threadfence_block();
+                    *issued = n + 1;
+                }
+                __syncwarp();
+                return true;
             }
-            ptx::tc_fence_after_sync();   // orders the UMMAs after the other warps' TMEM reads and operand writes
-            if (!__all_sync(0xffffffffu, *issued >= n) &&
-                !__all_sync(0xffffffffu, turn_wait_slow2(issued, n, abort_flag)))
+            if (!__all_sync(0xffffffffu, *issued > n) &&
+                !__all_sync(0xffffffffu, turn_wait_slow2(issued, n + 1, abort_flag)))
                 return false;
+            __threadfence_block();
+            ptx::tc_fence_after_sync();   // orders the UMMAs after the other warps' TMEM reads and operand writes
             if (elect_one()) {
                 const uint32_t b_lo = w_lo + sl * kSlotLo;
 #pragma unroll
@@ -316,7 +328,6 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
                     if (j < w.nkb)
                         mma_kblock_pair(w.d_tm, w.a_lo[j], b_lo + (uint32_t)j * w.b_blk_lo, w.idesc,
                                         (j == 0 && w.overwrite) ? 0u : 1u);
-                *issued = n + 1;
 #pragma unroll
                 for (int j = 0; j <= kMaxKb; ++j)
                     if (w.cb[j] != 0u) ptx::umma_commit_pair(w.cb[j], (uint16_t)3);
@@ -336,7 +347,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
                 const uint32_t hp = (q & 1u) ^ 1u;
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
-                    if (!ok || ((n + i) & 1u) != me) continue;
+                    if (!ok) continue;
                     SlotWork w = {};
                     w.d_tm = tm_h;
                     w.idesc = (C::CH == 256) ? idesc256 : idesc128;
@@ -365,7 +376,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
                 const uint32_t yp = (pti & 1u) ^ 1u;
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
-                    if (!ok || ((n + i) & 1u) != me) continue;
+                    if (!ok) continue;
                     SlotWork w = {};
                     w.nkb = SS::g2_nkb();
                     w.b_blk_lo = (uint32_t)(SS::g2_rows(i) * 128) >> 4;
@@ -456,20 +467,22 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
         auto drain_y = [&](uint32_t t_idx, int32_t grow) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
-            // 64 columns per pass.  The TMEM loads of the next pass are in flight while this pass's
-            // rows go out, and the row numbers of the store steps are fetched once.
+            // 64 columns per pass: two TMEM loads and one wait, bf16 rows through the staging
+            // piece, then whole 128-byte row segments to global memory.  The registers a TMEM
+            // load writes are not named again before its wait.
             constexpr int NP = D / 128;
             const int ch = lane & 7;
             int32_t grs[8];
 #pragma unroll
             for (int step = 0; step < 8; ++step) grs[step] = __shfl_sync(0xffffffffu, grow, step * 4 + (lane >> 3));
             __nv_bfloat16* ycol = Y + half * (D / 2) + ch * 8;
-            uint32_t ra[32], rb[32];
-            ptx::tmem_ld_32x32(lane_base + half * (D / 2), ra);
-            ptx::tmem_ld_32x32(lane_base + half * (D / 2) + 32, rb);
-            ptx::tmem_ld_wait();
 #pragma unroll 1
             for (int pass = 0; pass < NP; ++pass) {
+                uint32_t ra[32], rb[32];
+                const int col0 = half * (D / 2) + pass * 64;
+                ptx::tmem_ld_32x32(lane_base + col0, ra);
+                ptx::tmem_ld_32x32(lane_base + col0 + 32, rb);
+                ptx::tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + ((i ^ (lane & 7)) << 4)),
@@ -485,11 +498,6 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
                                  "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 6]), __uint_as_float(rb[8 * i + 7])))
                                  : "memory");
                 }
-                if (pass + 1 < NP) {
-                    const int col1 = half * (D / 2) + (pass + 1) * 64;
-                    ptx::tmem_ld_32x32(lane_base + col1, ra);
-                    ptx::tmem_ld_32x32(lane_base + col1 + 32, rb);
-                }
                 __syncwarp();
 #pragma unroll
                 for (int step = 0; step < 8; ++step) {
@@ -501,7 +509,6 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
                     if (grs[step] >= 0) *reinterpret_cast<uint4*>(ycol + (size_t)grs[step] * D + pass * 64) = v;
                 }
                 __syncwarp();
-                if (pass + 1 < NP) ptx::tmem_ld_wait();
             }
             ptx::tc_fence_before_sync();
             warp_arrive_leader(&misc->y_empty);
