@@ -20,7 +20,7 @@
 // never waits for the GELU epilogue with nothing else queued.
 //
 // Warp roles (512 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
-// warp 1 = UMMA issuer, warp 15 = its watcher (does the barrier waits), warps 3-6 = X row
+// warp 1 = UMMA issuer (warp 15 is idle), warps 3-6 = X row
 // gather, warps 7-14 = epilogue (two warps per TMEM lane quarter).  Producer and issuer warps stay
 // converged and elect one lane per instruction.  Every wait is bounded; on expiry the CTA raises SENTRY_STATUS_BIT_TIMEOUT
 // and unwinds.
@@ -41,7 +41,6 @@ constexpr int kStages = 3;
 constexpr int kThreads = 512;
 constexpr int kLoaderWarp0 = 3, kLoaderWarps = 4, kLoaderThreads = kLoaderWarps * 32;
 constexpr int kEpiWarp0 = 7, kEpiWarps = 8;
-constexpr int kIssuerB = 15;   // second UMMA issuer warp (the first is warp 1)
 constexpr int kTmemCols = 512;
 
 template <int D>
@@ -68,7 +67,6 @@ struct Misc {
     uint64_t y_full, y_empty;
     uint32_t tmem_base;
     int abort_flag;
-    uint32_t issued;   // weight stages whose operands the watcher has seen complete (polled by the issuer)
 };
 static_assert(sizeof(Misc) <= 2048, "misc block too large");
 
@@ -109,13 +107,6 @@ static __device__ __noinline__ bool wait_each_slow(uint32_t b0, uint32_t p0, uin
     if (ok && b3 != 0u) ok = ptx::mbar_wait(b3, p3, abort_flag);
     return ok;
 }
-// Slow path of the issuer's poll: until the watcher has published `n` stages, bounded.
-static __device__ __noinline__ bool turn_wait_slow(volatile uint32_t* issued, uint32_t n, volatile int* abort_flag) {
-    for (uint32_t spins = 0; *issued < n; ++spins) {
-        if (spins > (1u << 22) || *abort_flag) { *abort_flag = 1; return false; }
-    }
-    return true;
-}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -154,7 +145,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         ptx::mbar_init(ptx::smem_u32(&misc->y_full), 1);
         ptx::mbar_init(ptx::smem_u32(&misc->y_empty), kEpiWarps);
         misc->abort_flag = 0;
-        misc->issued = 0;
         ptx::fence_barrier_init();
     }
     if (warp == 0) {
@@ -244,25 +234,21 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             }
             if (++c == NC) { c = 0; ++ti; }
         }
-    } else if (warp == 1 || warp == kIssuerB) {
-        // ------------------------------------------------------- UMMA issuer and its watcher
-        // Both warps walk the same schedule of weight stages.  The watcher (warp kIssuerB) does
-        // the waiting: for every stage it probes the barriers the stage needs (weights landed,
-        // operand blocks written, accumulator released) and then publishes the stage number.
-        // The issuer (warp 1) only polls that number, and one elected lane issues the stage's
-        // UMMAs and commits.  ALL UMMAs therefore come from one thread: the tensor pipe runs the
-        // instructions of one thread in issue order, but nothing orders the instructions of two
-        // threads, and accumulators fed alternately by two issuing warps were summed in an order
-        // that changed from run to run (results differed in the last bit).  The split keeps part
-        // of what two warps were good for: the barrier round trips of the next stage overlap the
-        // issue of the current one.
-        const bool is_issuer = (warp == 1);
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------- UMMA issuer
+        // One warp walks the schedule of weight stages; for every stage it probes the barriers
+        // the stage needs (weights landed, operand blocks written, accumulator released), and
+        // one elected lane issues the stage's UMMAs and commits.  ALL UMMAs come from one
+        // thread: the tensor pipe runs the instructions of one thread in issue order, but
+        // nothing orders the instructions of two threads, and accumulators fed alternately by
+        // two issuing warps were summed in an order that changed from run to run (results
+        // differed in the last bit).  A second warp that did the waiting and handed the stage
+        // number over through shared memory measured slower than the issuer waiting itself.
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
         constexpr uint32_t kBlkLo = kBlockBytes >> 4, kStageLo = kStageBytes >> 4;
         const uint32_t tm_h = tmem + C::H_COL0;
         const uint32_t xs_lo = desc_lo(xs), hs_lo = desc_lo(hs), w_lo = desc_lo(wsm);
-        volatile uint32_t* issued = &misc->issued;
         // One stage.  wb*: barriers to wait on besides the weights (0 = none), cb*: barriers to
         // commit to besides w_empty (0 = none); a_lo1 != 0: the stage holds two K blocks.
         auto stage = [&](uint32_t n, uint32_t d_tm, uint32_t a_lo0, uint32_t a_lo1, uint32_t idesc, bool overwrite,
@@ -270,8 +256,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                          bool /*writes TMEM others read: fenced in every case*/, uint32_t cb0, uint32_t cb1,
                          uint32_t cb2) -> bool {
             const uint32_t sl = n % kStages, ph = (n / kStages) & 1u;
-            if (!is_issuer) {
-                // watcher: every barrier of the stage, probed at once, then the stage is published
+            {
                 const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
                 bool p = ptx::mbar_try_wait(wf, ph);
                 if (wb0 != 0u) p &= ptx::mbar_try_wait(wb0, wp0);
@@ -280,17 +265,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 if (!__all_sync(0xffffffffu, p) &&
                     !__all_sync(0xffffffffu, wait_each_slow(wf, ph, wb0, wp0, wb1, wp1, wb2, wp2, abort_flag)))
                     return false;
-                if (elect_one()) {
-                    __threadfence_block();
-                    *issued = n + 1;
-                }
-                __syncwarp();
-                return true;
             }
-            if (!__all_sync(0xffffffffu, *issued > n) &&
-                !__all_sync(0xffffffffu, turn_wait_slow(issued, n + 1, abort_flag)))
-                return false;
-            __threadfence_block();
             ptx::tc_fence_after_sync();   // orders the UMMAs after the epilogue's TMEM reads and operand writes
             if (elect_one()) {
                 const uint32_t b_lo = w_lo + sl * kStageLo;

@@ -12,7 +12,7 @@
 // traffic from L2 into shared memory is halved.
 //
 // Who talks to whom.  All UMMAs are issued by one thread of the even CTA of the pair (the
-// leader; a second warp does the waiting for it, as in the single-CTA kernel).  Barriers the issuer waits on (weights landed, X block
+// leader).  Barriers the issuer waits on (weights landed, X block
 // landed, hidden block written, accumulators drained) live in the leader's shared memory and
 // count arrivals from BOTH CTAs: the peer arrives remotely, its TMA copies credit their bytes
 // to the leader's barrier.  Barriers the issuer signals (ring slot free, X slot free, hidden
@@ -20,7 +20,7 @@
 // multicast commit.  No multicast copies anywhere: every CTA loads its own operands.
 //
 // Warp roles per CTA (512 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
-// warp 1 = UMMA issuer, warp 15 = its watcher (leader only; idle in the peer), warps 3-6 = X row gather,
+// warp 1 = UMMA issuer (leader only; idle in the peer; warp 15 is idle), warps 3-6 = X row gather,
 // warps 7-14 = epilogue.  Every wait is bounded; on expiry the CTA raises
 // SENTRY_STATUS_BIT_TIMEOUT and unwinds, and the pair leaves together.
 #include <cuda.h>
@@ -41,7 +41,6 @@ constexpr int kStages = 3;
 constexpr int kThreads = 512;
 constexpr int kLoaderWarp0 = 3, kLoaderWarps = 4, kLoaderThreads = kLoaderWarps * 32;
 constexpr int kEpiWarp0 = 7, kEpiWarps = 8;
-constexpr int kIssuerB = 15;
 constexpr int kTmemCols = 512;
 constexpr int kMaxKb = 4;                // K blocks (64 wide) per ring slot at most
 
@@ -84,7 +83,6 @@ struct Misc {
     uint64_t y_full, y_empty;
     uint32_t tmem_base;
     int abort_flag;
-    uint32_t issued;
 };
 static_assert(sizeof(Misc) <= 2048, "misc block too large");
 
@@ -125,12 +123,6 @@ static __device__ __noinline__ bool wait_cluster_slow(uint32_t bar, uint32_t par
             }
         }
     }
-}
-static __device__ __noinline__ bool turn_wait_slow2(volatile uint32_t* issued, uint32_t n, volatile int* abort_flag) {
-    for (uint32_t spins = 0; *issued < n; ++spins) {
-        if (spins > (1u << 22) || *abort_flag) { *abort_flag = 1; return false; }
-    }
-    return true;
 }
 // One arrival for the whole warp on the barrier at this offset in the leader CTA.
 __device__ __forceinline__ void warp_arrive_leader(uint64_t* bar) {
@@ -191,7 +183,6 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
         ptx::mbar_init(ptx::smem_u32(&misc->y_full), 1);
         ptx::mbar_init(ptx::smem_u32(&misc->y_empty), 2 * kEpiWarps);
         misc->abort_flag = 0;
-        misc->issued = 0;
         ptx::fence_barrier_init();
     }
     if (warp == 0) {
@@ -280,23 +271,19 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
             }
             if (++c == NC) { c = 0; ++ti; }
         }
-    } else if ((warp == 1 || warp == kIssuerB) && rank == 0) {
-        // ------------------------------------------------------- UMMA issuer and its watcher
-        // As in the single-CTA kernel: warp kIssuerB of the leader waits for every slot's
-        // barriers and publishes the slot number, one elected lane of warp 1 issues every UMMA
-        // (one issuing thread: a fixed summation order); every UMMA runs on both CTAs, every
-        // commit goes to both.
-        const bool is_issuer = (warp == 1);
+    } else if (warp == 1 && rank == 0) {
+        // ------------------------------------------------------------------- UMMA issuer
+        // As in the single-CTA kernel: one warp of the leader walks the schedule, waits for every
+        // slot's barriers, and one elected lane issues every UMMA (one issuing thread: a fixed
+        // summation order); every UMMA runs on both CTAs, every commit goes to both.
         constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(256, 256);
         constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(256, 128);
         constexpr uint32_t kBlkLo = kBlockBytes >> 4, kSlotLo = kSlotBytes >> 4;
         const uint32_t tm_h = tmem + C::H_COL0;
         const uint32_t xs_lo = desc_lo(xs), hs_lo = desc_lo(hs), w_lo = desc_lo(wsm);
-        volatile uint32_t* issued = &misc->issued;
         auto run = [&](uint32_t n, const SlotWork& w) -> bool {
             const uint32_t sl = n % kStages, ph = (n / kStages) & 1u;
-            if (!is_issuer) {
-                // watcher: every barrier of the slot, probed at once, then the slot is published
+            {
                 const uint32_t wf = MISC_BAR(mb, w_full) + 8u * sl;
                 bool p = ptx::mbar_try_wait_cluster(wf, ph);
 #pragma unroll
@@ -309,17 +296,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_const
                         if (ok && w.wb[j] != 0u) ok = wait_cluster_slow(w.wb[j], w.wp[j], abort_flag);
                     if (!__all_sync(0xffffffffu, ok)) return false;
                 }
-                if (elect_one()) {
-                    __threadfence_block();
-                    *issued = n + 1;
-                }
-                __syncwarp();
-                return true;
             }
-            if (!__all_sync(0xffffffffu, *issued > n) &&
-                !__all_sync(0xffffffffu, turn_wait_slow2(issued, n + 1, abort_flag)))
-                return false;
-            __threadfence_block();
             ptx::tc_fence_after_sync();   // orders the UMMAs after the other warps' TMEM reads and operand writes
             if (elect_one()) {
                 const uint32_t b_lo = w_lo + sl * kSlotLo;
