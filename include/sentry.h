@@ -209,6 +209,13 @@ typedef struct sentry_ffn_desc {
  * The kept columns of W1 and rows of W2 are gathered into the workspace on
  * every call (the "materialised" pruned weights), then a fused GEMM pair runs
  * over the present rows.  Supported: D % 8 == 0, D <= 1024.
+ * bf16 with D in {128, 256, 384} runs on the tcgen05 tensor cores, one CTA
+ * per SM; the environment variable SENTRY_FFN_KERNEL=pair (read once per
+ * process, at the first call) selects the variant that runs every tensor
+ * instruction on a pair of CTAs instead.  The GELU of the bf16 path evaluates
+ * erf through the hardware tanh: within 4e-4 of gelu(|z|), below the rounding
+ * of the bf16 hidden value it is stored as; fp32 uses erff.  Results are
+ * bit-identical from call to call for identical inputs.
  */
 SENTRY_API int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X,
                    const void* W1, const void* W2, const int32_t* kept_channels,
