@@ -209,10 +209,9 @@ typedef struct sentry_ffn_desc {
  * The kept columns of W1 and rows of W2 are gathered into the workspace on
  * every call (the "materialised" pruned weights), then a fused GEMM pair runs
  * over the present rows.  Supported: D % 8 == 0, D <= 1024.
- * bf16 with D in {128, 256, 384} runs on the tcgen05 tensor cores, one CTA
- * per SM; the environment variable SENTRY_FFN_KERNEL=pair (read once per
- * process, at the first call) selects the variant that runs every tensor
- * instruction on a pair of CTAs instead.  The GELU of the bf16 path evaluates
+ * bf16 with D in {128, 256, 384} runs on the tcgen05 tensor cores, one
+ * persistent CTA per SM; every other shape and fp32 run on the plain ALUs with
+ * fp32 accumulation.  The GELU of the bf16 path evaluates
  * erf through the hardware tanh: within 4e-4 of gelu(|z|), below the rounding
  * of the bf16 hidden value it is stored as; fp32 uses erff.  Results are
  * bit-identical from call to call for identical inputs.
@@ -221,6 +220,16 @@ SENTRY_API int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, cons
                    const void* W1, const void* W2, const int32_t* kept_channels,
                    const int32_t* list_of_sample, const int32_t* token_modality_ids,
                    const uint32_t* masks, void* Y, void* stream);
+
+/* Self-test of the bounded device waits.  Every wait inside the kernels (on a
+ * TMA copy, a tensor-core commit, another warp) gives up after about a second,
+ * raises SENTRY_STATUS_BIT_TIMEOUT, lets copies in flight land, frees its
+ * tensor memory and returns.  This call enqueues one small CTA that waits on a
+ * barrier nothing ever signals, with a limit of `limit_cycles` SM clock cycles
+ * (1 .. 1e8), and then leaves through that same path: afterwards
+ * sentry_get_last_status reports SENTRY_STATUS_BIT_TIMEOUT and the context is
+ * usable as before.  Nothing hangs or faults. */
+SENTRY_API int sentry_selftest_wait_expiry(sentry_ctx* ctx, long long limit_cycles, void* stream);
 
 /* Number of kernels the last call on this context enqueued (for launch
  * accounting in benchmarks). */

@@ -26,7 +26,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_num_active_queries", "sentry_workspace_bytes", "sentry_set_workspace",
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
-           "sentry_kernel_name", "sentry_gate_select_static"]
+           "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
                                       vp, ci, vp, vp, vp, vp]
     lib.sentry_ffn_fwd.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_last_launch_count.argtypes = [vp]
+    lib.sentry_selftest_wait_expiry.argtypes = [vp, ctypes.c_longlong, vp]
     lib.sentry_profile_enable.argtypes = [vp, ci]
     lib.sentry_profile_slots.argtypes = []
     lib.sentry_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
@@ -181,6 +182,12 @@ class Sentry:
         if rc < 0:
             raise SentryError(rc, "sentry_get_last_status")
         return rc
+
+    def selftest_wait_expiry(self, limit_cycles: int = 100000):
+        """Enqueue the wait-expiry self-test (one CTA whose wait runs out after limit_cycles)."""
+        rc = self.lib.sentry_selftest_wait_expiry(self.h, int(limit_cycles), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_selftest_wait_expiry")
 
     def last_launch_count(self) -> int:
         return int(self.lib.sentry_last_launch_count(self.h))

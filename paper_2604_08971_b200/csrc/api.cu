@@ -1,5 +1,7 @@
 // C ABI of libsentry: argument validation, workspace carving and dispatch.
 // Everything numerical happens in the kernels of the other translation units.
+#include <stdlib.h>
+
 #include <new>
 
 #include "common.cuh"
@@ -54,7 +56,7 @@ int sentry_create(sentry_ctx** out, int device) {
     *out = nullptr;
     int n = 0;
     if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return SENTRY_ERR_CUDA;
-    SENTRY_CUDA_TRY(cudaSetDevice(device));
+    SENTRY_ON_DEVICE(device);
     sentry_ctx* c = new (std::nothrow) sentry_ctx();
     if (c == nullptr) return SENTRY_ERR_CUDA;
     c->device = device;
@@ -77,7 +79,7 @@ int sentry_create(sentry_ctx** out, int device) {
 
 int sentry_destroy(sentry_ctx* ctx) {
     if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
-    cudaSetDevice(ctx->device);
+    DeviceGuard guard(ctx->device);
     cudaFree(ctx->d_status);
     for (ProfRec& r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
     for (cudaEvent_t e : ctx->pool) cudaEventDestroy(e);
@@ -102,7 +104,7 @@ const char* sentry_kernel_name(int slot) {
 int sentry_profile_read(sentry_ctx* ctx, float* ms, int* launches, int n) {
     if (ctx == nullptr || ms == nullptr || launches == nullptr || n < KS_COUNT)
         return SENTRY_ERR_INVALID_ARG;
-    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    SENTRY_ON_DEVICE(ctx->device);
     SENTRY_CUDA_TRY(cudaDeviceSynchronize());
     for (int i = 0; i < n; ++i) { ms[i] = 0.f; launches[i] = 0; }
     for (ProfRec& r : ctx->prof) {
@@ -120,7 +122,7 @@ int sentry_profile_read(sentry_ctx* ctx, float* ms, int* launches, int n) {
 
 int sentry_get_last_status(sentry_ctx* ctx, void* stream) {
     if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
-    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    SENTRY_ON_DEVICE(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
     SENTRY_CUDA_TRY(cudaStreamSynchronize(st));
     unsigned int h = 0;
@@ -167,6 +169,13 @@ int sentry_set_workspace(sentry_ctx* ctx, void* dev_ptr, size_t bytes) {
     return SENTRY_OK;
 }
 
+int sentry_selftest_wait_expiry(sentry_ctx* ctx, long long limit_cycles, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > 100000000LL) return SENTRY_ERR_BAD_SHAPE;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_wait_expiry_selftest(ctx, limit_cycles, (cudaStream_t)stream);
+}
+
 int sentry_last_launch_count(const sentry_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 
 int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
@@ -187,7 +196,7 @@ int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
     int32_t* rows = a.take<int32_t>((size_t)S * k);
     uint32_t* groups = a.take<uint32_t>((size_t)S);
     if (!a.ok) return SENTRY_ERR_WORKSPACE;
-    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    SENTRY_ON_DEVICE(ctx->device);
     return launch_gate_select(ctx, scores, S, n_units, masks, n_masks, k, kept, kv_groups,
                               heads_per_group, rows, groups, (cudaStream_t)stream);
 }
@@ -232,10 +241,12 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
     a.selection_given = active_in != nullptr;
     a.active = a.selection_given ? const_cast<int32_t*>(active_in)
                                  : (active_out != nullptr ? active_out : ws_active);
-    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    SENTRY_ON_DEVICE(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
     a.active_out_user = active_out;
-    rc = attend_bf16_supported(*desc) ? launch_attend_bf16(ctx, a, st) : launch_attend_generic(ctx, a, st);
+    static const bool tc_path = getenv("SENTRY_ATTEND_TC") != nullptr;   // bring-up switch
+    if (attend_tc_supported(*desc) && tc_path) rc = launch_attend_tc(ctx, a, st);
+    else rc = attend_bf16_supported(*desc) ? launch_attend_bf16(ctx, a, st) : launch_attend_generic(ctx, a, st);
     if (rc != SENTRY_OK) return rc;
     if (a.selection_given && active_out != nullptr && active_out != active_in) {
         SENTRY_CUDA_TRY(cudaMemcpyAsync(active_out, active_in,
@@ -269,7 +280,7 @@ int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, 
     a.masks = masks;
     a.Y = Y;
     a.status = ctx->d_status;
-    SENTRY_CUDA_TRY(cudaSetDevice(ctx->device));
+    SENTRY_ON_DEVICE(ctx->device);
     return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, (cudaStream_t)stream);
 }
 

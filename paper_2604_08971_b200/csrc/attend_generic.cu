@@ -50,12 +50,12 @@ attend_score_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                     unsigned int* status) {
     extern __shared__ uint16_t s_valid[];
     __shared__ int red[66];
-    const int bh = blockIdx.y, b = bh / k_h;
+    const int bh = blockIdx.x, b = bh / k_h;
     const uint32_t mask = masks[b];
     const int Tv = block_build_valid(ids, Tlen, mask, s_valid, red);
     if (Tv == 0) return;
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (blockIdx.x * blockDim.x >= Tv) return;
+    const int p = blockIdx.y * blockDim.x + threadIdx.x;
+    if (blockIdx.y * blockDim.x >= Tv) return;
     const int h = kept_heads[bh];
     if (h < 0 || h >= Hq) {
         if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
@@ -232,7 +232,7 @@ int launch_typed(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
             if (valid_bytes > 48 * 1024)
                 SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)valid_bytes));
-            dim3 grid((d.T + kScoreThreads - 1) / kScoreThreads, BH);
+            dim3 grid(BH, (d.T + kScoreThreads - 1) / kScoreThreads);   // (sample, head) on x: no 65535 limit
             LaunchScope ls(ctx, KS_ATT_SCORE, st);
             kern<<<grid, kScoreThreads, valid_bytes, st>>>(
                 (const T*)a.Q, (const T*)a.K, a.kept_heads, a.ids, a.masks, a.sample_table,

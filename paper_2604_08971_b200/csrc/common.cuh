@@ -57,6 +57,27 @@ struct LaunchScope {
         if (_e != cudaSuccess) return SENTRY_ERR_CUDA; \
     } while (0)
 
+// Makes `device` current for the lifetime of the object and puts the caller's device back
+// afterwards, so that no entry point changes the calling thread's current device.
+struct DeviceGuard {
+    int prev;
+    bool ok, switched;
+    explicit DeviceGuard(int device) : prev(-1), ok(false), switched(false) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        if (prev != device) {
+            if (cudaSetDevice(device) != cudaSuccess) return;
+            switched = true;
+        }
+        ok = true;
+    }
+    ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+    DeviceGuard(const DeviceGuard&) = delete;
+    DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
+#define SENTRY_ON_DEVICE(device)      \
+    DeviceGuard _dev_guard(device);   \
+    if (!_dev_guard.ok) return SENTRY_ERR_CUDA
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Bump allocator over the caller-provided workspace.
@@ -299,6 +320,8 @@ struct AttendArgs {
     unsigned int* status;
 };
 int launch_attend_generic(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
+bool attend_tc_supported(const sentry_attend_desc& d);
+int launch_attend_tc(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_bf16_supported(const sentry_attend_desc& d);
 int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 
@@ -313,4 +336,5 @@ struct FfnArgs {
     unsigned int* status;
 };
 size_t ffn_workspace_bytes(const sentry_ffn_desc& d);
+int launch_wait_expiry_selftest(sentry_ctx* ctx, long long limit_cycles, cudaStream_t st);
 int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cudaStream_t st);

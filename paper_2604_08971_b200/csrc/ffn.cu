@@ -3,8 +3,6 @@
 // and the plain-ALU fp32-accumulate kernel; the tensor-core kernel for bf16
 // lives in ffn_tc.cu and shares the plan.
 #include <math.h>
-#include <stdlib.h>
-#include <string.h>
 
 #include "common.cuh"
 #include "ffn_plan.cuh"
@@ -13,9 +11,6 @@ int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* 
                   int kc_pad, int max_tiles, cudaStream_t st);  // ffn_tc.cu
 bool ffn_tc_supported(const sentry_ffn_desc& d);
 int ffn_tc_kc_pad(int D, int k_c);
-int launch_ffn_tc_pair(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,
-                       int kc_pad, int max_tiles, cudaStream_t st);  // ffn_tc2.cu
-int ffn_tc_pair_tile_rows();
 
 namespace {
 
@@ -318,16 +313,6 @@ FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes) {
     return w;
 }
 
-// The tensor-core FFN runs one CTA per SM unless SENTRY_FFN_KERNEL=pair asks for the CTA-pair kernel.
-bool use_pair_kernel() {
-    static int pair = -1;
-    if (pair < 0) {
-        const char* e = getenv("SENTRY_FFN_KERNEL");
-        pair = (e != nullptr && strcmp(e, "pair") == 0) ? 1 : 0;
-    }
-    return pair == 1;
-}
-
 int kc_pad_for(const sentry_ffn_desc& d) {
     if (d.dtype == SENTRY_BF16 && ffn_tc_supported(d)) return ffn_tc_kc_pad(d.D, d.k_c);
     return (d.k_c + 7) / 8 * 8;
@@ -345,8 +330,7 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cud
     const int kc_pad = kc_pad_for(d);
     FfnWs w = carve(d, kc_pad, ws, ws_bytes);
     if (!w.ok) return SENTRY_ERR_WORKSPACE;
-    const bool pair = tc && use_pair_kernel();
-    const int tile_rows = tc ? (pair ? ffn_tc_pair_tile_rows() : kTcTileRows) : kGenericTileRows;
+    const int tile_rows = tc ? kTcTileRows : kGenericTileRows;
 
     {
         const size_t per = (size_t)kc_pad * d.D;
@@ -373,8 +357,7 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cud
     const long long rows = (long long)d.B * d.T;
     const int max_tiles = (int)((rows + tile_rows - 1) / tile_rows) + d.n_lists;
     if (tc) {
-        int rc = pair ? launch_ffn_tc_pair(ctx, a, w.plan, w.w1p, w.w2p, kc_pad, max_tiles, st)
-                      : launch_ffn_tc(ctx, a, w.plan, w.w1p, w.w2p, kc_pad, max_tiles, st);
+        int rc = launch_ffn_tc(ctx, a, w.plan, w.w1p, w.w2p, kc_pad, max_tiles, st);
         if (rc != SENTRY_OK) return rc;
     } else {
         const size_t smem = ((size_t)kGenericTileRows * d.D + kGenericTileRows * kGenericThreads) * 4;

@@ -29,7 +29,7 @@
 
 #include "common.cuh"
 #include "ffn_plan.cuh"
-#include "ffn_tc_common.cuh"
+#include "tc_common.cuh"
 #include "ptx/sm100.cuh"
 
 namespace {
@@ -106,6 +106,24 @@ static __device__ __noinline__ bool wait_each_slow(uint32_t b0, uint32_t p0, uin
     if (ok && b2 != 0u) ok = ptx::mbar_wait(b2, p2, abort_flag);
     if (ok && b3 != 0u) ok = ptx::mbar_wait(b3, p3, abort_flag);
     return ok;
+}
+
+// End of a CTA: if any wait ran out, raise the status bit and give copies and UMMAs that may
+// still be in flight time to land before shared memory and TMEM go away; then free the TMEM.
+__device__ __forceinline__ void cta_teardown(volatile int* abort_flag, unsigned int* status, uint32_t tmem,
+                                             uint32_t tmem_cols) {
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_TIMEOUT);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+        __syncthreads();
+    }
+    if ((threadIdx.x >> 5) == 0) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, tmem_cols);
+    }
 }
 
 template <int D>
@@ -512,20 +530,35 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         if (ok && ti > 0) drain_y(ti - 1, my_row);
     }
 
-    // ---------------------------------------------------------------------------- teardown
+    cta_teardown(abort_flag, status, tmem, kTmemCols);
+}
+
+// One CTA that waits, through the same bounded wait as the kernels above, on a barrier nobody
+// ever arrives on, and then unwinds through the same teardown (status bit, grace period, TMEM
+// release).  It exists so that a test can watch a wait run out without hanging anything.
+__global__ void __launch_bounds__(128, 1) wait_expiry_selftest_kernel(long long limit_cycles, unsigned int* status) {
+    __shared__ uint64_t never;
+    __shared__ uint32_t tmem_base;
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&never), 1);
+        abort_word = 0;
+        ptx::fence_barrier_init();
+    }
+    if ((threadIdx.x >> 5) == 0) {
+        ptx::tmem_alloc(ptx::smem_u32(&tmem_base), 32);
+        ptx::tmem_relinquish();
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (*abort_flag) {
-        if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_TIMEOUT);
-        // give copies and UMMAs still in flight time to land before shared memory and TMEM go away
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
-        __syncthreads();
-    }
-    if (warp == 0) {
-        ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem, kTmemCols);
-    }
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = tmem_base;
+    // warp 1 waits with the limit under test; the other warps wait with the default limit and
+    // must be released by the abort flag that warp 1 raises
+    const long long limit = (threadIdx.x >> 5) == 1 ? limit_cycles : ptx::kWaitLimitCycles;
+    (void)ptx::mbar_wait(ptx::smem_u32(&never), 0u, abort_flag, limit);
+    cta_teardown(abort_flag, status, tmem, 32);
 }
 
 template <int D>
@@ -557,6 +590,12 @@ bool ffn_tc_supported(const sentry_ffn_desc& d) {
 int ffn_tc_kc_pad(int D, int k_c) {
     const int ch = (D == 384) ? 128 : 256;
     return (k_c + ch - 1) / ch * ch;
+}
+
+int launch_wait_expiry_selftest(sentry_ctx* ctx, long long limit_cycles, cudaStream_t st) {
+    wait_expiry_selftest_kernel<<<1, 128, 0, st>>>(limit_cycles, ctx->d_status);
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
 }
 
 int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,

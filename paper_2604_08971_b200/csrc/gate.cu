@@ -212,7 +212,7 @@ extern "C" int sentry_gate_select_static(int device, const float* scores, int S,
         return SENTRY_ERR_WORKSPACE;
     if (n_masks == 0) return SENTRY_OK;
 
-    SENTRY_CUDA_TRY(cudaSetDevice(device));
+    SENTRY_ON_DEVICE(device);
     StaticDevice sd;
     int rc = static_scratch_of(device, &sd);
     if (rc != SENTRY_OK) return rc;

@@ -49,27 +49,29 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait.  Gives up after ~kWaitLimitCycles or as soon as another thread of the CTA has
-// given up (abort flag in shared memory); returns false in both cases.  The caller must then
-// leave its loop: nothing in the kernels waits without a limit.
+// Bounded wait.  Gives up after ~limit cycles (default: about a second) or as soon as another
+// thread of the CTA has given up (abort flag in shared memory); returns false in both cases.
+// The caller must then leave its loop: nothing in the kernels waits without a limit.
 constexpr long long kWaitLimitCycles = 2000000000LL;  // about a second
 // The polling loop is kept out of line: one copy per kernel file instead of one per wait.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                   long long limit = kWaitLimitCycles) {
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag);
+    return mbar_wait_slow(bar, parity, abort_flag, limit);
 }
 
 // ------------------------------------------------------------------------------- proxies
@@ -153,77 +155,19 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr)
         : "memory");
 }
+// 32 lanes x 16 consecutive fp32 columns.
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// ------------------------------------------------------------------- CTA pairs (clusters of 2)
-// Two CTAs of a cluster on neighbouring SMs can run one UMMA together (cta_group::2): each
-// holds its own 128 rows of A and of the accumulator and one half of B's rows; the instruction
-// is issued by one thread of the even CTA (the leader) and reads both CTAs' shared memory at
-// the same offsets.
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// All threads of both CTAs: arrive and wait (release / acquire at cluster scope).
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Arrive on the mbarrier at the same shared-memory offset in CTA `cta` of the cluster.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t local_bar, uint32_t cta) {
-    asm volatile(
-        "{\n\t.reg .b32 ra;\n\t"
-        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
-        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
-        ::"r"(local_bar), "r"(cta)
-        : "memory");
-}
-// Probe of a phase with acquire semantics at cluster scope (the arrivals may come from the peer CTA).
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// 2-D tiled load into THIS CTA's shared memory whose byte count is credited to the mbarrier at
-// the same offset in the leader CTA of the pair (`bar_in_leader`: a shared::cluster address).
-// No multicast: every CTA fetches its own tile.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t smem_dst, const void* tmap, int x, int y,
-                                                 uint32_t bar_in_leader) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3}], [%4];"
-        :
-        : "r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar_in_leader)
-        : "memory");
-}
-// TMEM of both CTAs of a pair: one warp of EACH CTA executes these.
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result),
-                 "r"(ncols)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
-                 : "memory");
-}
-// Arrive, once every UMMA this thread issued before has completed, on the mbarrier at this
-// offset in every CTA of the pair named by `cta_mask` (bit r = CTA rank r).
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"(cta_mask)
-        : "memory");
 }
 
 // Instruction descriptor of a dense bf16 x bf16 -> fp32 UMMA, both operands K-major.
@@ -249,6 +193,28 @@ __device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t smem_addr) {
     d |= (uint64_t)1u << 46;
     d |= (uint64_t)2u << 61;
     return d;
+}
+
+// General forms for operand tiles whose rows are 32, 64 or 128 bytes wide (swizzle mode of that
+// width; layout code 6 / 4 / 2), 8-row groups `sbo_bytes` apart (8 x row bytes when the rows are
+// contiguous).  K-major operand: a row is one M/N index, its bytes run along K.  MN-major operand
+// (major bit set in the instruction descriptor): a row is one K index, its bytes run along M/N,
+// and sbo_bytes is the distance between groups of 8 K indices.
+__host__ __device__ constexpr uint32_t umma_layout_code(int row_bytes) {
+    return row_bytes == 128 ? 2u : (row_bytes == 64 ? 4u : 6u);
+}
+__device__ __forceinline__ uint64_t umma_smem_desc_rows(uint32_t smem_addr, int row_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1u << 16;
+    d |= (uint64_t)((8u * (uint32_t)row_bytes) >> 4) << 32;
+    d |= (uint64_t)1u << 46;
+    d |= (uint64_t)umma_layout_code(row_bytes) << 61;
+    return d;
+}
+// bf16 x bf16 -> fp32 with either operand K-major (false) or MN-major (true).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_major(int M, int N, bool a_mn_major, bool b_mn_major) {
+    return umma_idesc_bf16(M, N) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u);
 }
 
 }  // namespace ptx

@@ -1,5 +1,5 @@
-// Pieces shared by the tcgen05 FFN kernels: the GELU epilogue arithmetic, warp-level barrier
-// helpers, single-lane election and the TMA tensor-map encoder.
+// Pieces shared by the tcgen05 kernels (FFN pair, SentryAttend core): the GELU epilogue
+// arithmetic, warp-level barrier helpers, single-lane election and the TMA tensor-map encoder.
 #pragma once
 #include <cuda.h>
 #include <math.h>
@@ -100,17 +100,31 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// bf16 row-major [rows, cols] -> map with a box of `box_rows` rows x 64 columns, 128-byte swizzle.
-bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// bf16 row-major [rows, cols] -> 2-D map with a box of box_rows x box_cols elements whose rows
+// are box_cols * 2 = 32, 64 or 128 bytes wide, swizzled with the mode of that width.
+bool make_map_2d(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                 uint32_t box_cols) {
     EncodeTiledFn fn = get_encode_fn();
     if (fn == nullptr) return false;
+    CUtensorMapSwizzle sw;
+    switch (box_cols * 2) {
+        case 32: sw = CU_TENSOR_MAP_SWIZZLE_32B; break;
+        case 64: sw = CU_TENSOR_MAP_SWIZZLE_64B; break;
+        case 128: sw = CU_TENSOR_MAP_SWIZZLE_128B; break;
+        default: return false;
+    }
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// bf16 row-major [rows, cols] -> map with a box of `box_rows` rows x 64 columns, 128-byte swizzle.
+bool make_weight_map(CUtensorMap* tm, void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    return make_map_2d(tm, ptr, rows, cols, box_rows, 64);
 }
 
 }  // namespace

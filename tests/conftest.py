@@ -24,3 +24,18 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """Table of every CUDA-vs-oracle comparison of the session: the bounded figure that was
+    asserted and the plain max-abs/RMS figure beside it."""
+    try:
+        from tests import parity
+    except Exception:
+        return
+    if not parity.REPORT:
+        return
+    tr = terminalreporter
+    tr.write_sep("-", "parity figures (max-abs error / output RMS; bounded = asserted, raw = plain)")
+    for case, stage, bounded, raw, note in parity.REPORT:
+        tr.write_line("%-30s %-7s bounded %.3e  raw %.3e  %s" % (case, stage, bounded, raw, note))

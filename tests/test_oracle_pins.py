@@ -278,7 +278,7 @@ def test_dropping_a_modality_equals_deleting_its_tokens():
                           table_offsets=offs), O_drop)
 
 
-def test_output_length_preserved_and_flop_scaling():
+def test_output_length_preserved_and_active_row_count():
     # every present position gets a row (Section 4.4: output length preserved)
     B, Hq, Hk, T, d = 1, 2, 1, 128, 4
     Q, K, V = _rand_attn(B, Hq, Hk, T, d, 23)

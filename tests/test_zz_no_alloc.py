@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2604_08971_b200 as sentry
 
 pytestmark = pytest.mark.gpu
@@ -46,6 +47,9 @@ def test_static_entry_point_matches_context_entry_point_twice_in_a_row():
             torch.cuda.synchronize()
             assert torch.cuda.memory_allocated() == before
             assert torch.equal(kept, want_kept)
+            # and the same lists as the float64 oracle's full ordering (ties -> lower index)
+            np.testing.assert_array_equal(
+                kept.cpu().numpy(), oracle.gate_select(scores.cpu().numpy(), masks.cpu().numpy(), k))
             if hpg > 0:
                 assert torch.equal(groups, want_groups)
             assert int(status.item()) == 0
