@@ -189,6 +189,24 @@ SENTRY_API int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc
                       int n_subsets, void* O, int32_t* active_out,
                       const int32_t* active_in, void* stream);
 
+/* Which kernels run Eq. 6 for bf16 tensors whose K/V of one KV group fit in
+ * shared memory (T up to ~1.4 k at d = 32).  Two hand-written forms exist:
+ *   SENTRY_ATTEND_WARP_MMA  K/V staged by 16-byte async copies, Q K^T and P V
+ *                           on the register-level warp MMA, online softmax
+ *   SENTRY_ATTEND_TCGEN05   K/V staged by TMA tensor copies, Q K^T and P V on
+ *                           tcgen05 with the accumulators and the softmax
+ *                           weights in tensor memory, two-pass softmax
+ * Both split every softmax weight into a bf16 head and a bf16 remainder, so the
+ * results agree to well below the bf16 rounding of the stored output.
+ * SENTRY_ATTEND_AUTO (default) takes the one that measured faster for the
+ * shape.  Other shapes: bf16 with longer T runs a score kernel and a streamed
+ * warp-MMA kernel; fp32, Hq/Hk > 4, U > 48 or T > 8192 run on the plain ALUs. */
+#define SENTRY_OPT_ATTEND_KERNEL 1
+#define SENTRY_ATTEND_AUTO 0
+#define SENTRY_ATTEND_WARP_MMA 1
+#define SENTRY_ATTEND_TCGEN05 2
+SENTRY_API int sentry_set_option(sentry_ctx* ctx, int option, int value);
+
 /* ---------------------------------------------------------------------------
  * Channel-compacted FFN forward (Sec. 4.6): for every present row x,
  *   y = gelu(x . W1[:, N]) . W2[N, :],  gelu(z) = z/2 (1 + erf(z/sqrt 2)),

@@ -21,12 +21,14 @@ LIB_PATH = os.path.join(_HERE, "libsentry.so")
 
 SENTRY_F32, SENTRY_BF16 = 0, 1
 STATUS_BIT_TIMEOUT, STATUS_BIT_EMPTY_MASK, STATUS_BIT_BAD_INDEX = 1, 2, 4
+OPT_ATTEND_KERNEL = 1
+ATTEND_AUTO, ATTEND_WARP_MMA, ATTEND_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_status_string",
            "sentry_num_active_queries", "sentry_workspace_bytes", "sentry_set_workspace",
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
-           "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry"]
+           "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -75,6 +77,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_fwd.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_last_launch_count.argtypes = [vp]
     lib.sentry_selftest_wait_expiry.argtypes = [vp, ctypes.c_longlong, vp]
+    lib.sentry_set_option.argtypes = [vp, ci, ci]
     lib.sentry_profile_enable.argtypes = [vp, ci]
     lib.sentry_profile_slots.argtypes = []
     lib.sentry_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
@@ -188,6 +191,12 @@ class Sentry:
         rc = self.lib.sentry_selftest_wait_expiry(self.h, int(limit_cycles), _stream())
         if rc != 0:
             raise SentryError(rc, "sentry_selftest_wait_expiry")
+
+    def set_attend_kernel(self, which: int):
+        """SENTRY_OPT_ATTEND_KERNEL: ATTEND_AUTO, ATTEND_WARP_MMA or ATTEND_TCGEN05."""
+        rc = self.lib.sentry_set_option(self.h, OPT_ATTEND_KERNEL, int(which))
+        if rc != 0:
+            raise SentryError(rc, "sentry_set_option")
 
     def last_launch_count(self) -> int:
         return int(self.lib.sentry_last_launch_count(self.h))

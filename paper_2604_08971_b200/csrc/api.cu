@@ -1,7 +1,5 @@
 // C ABI of libsentry: argument validation, workspace carving and dispatch.
 // Everything numerical happens in the kernels of the other translation units.
-#include <stdlib.h>
-
 #include <new>
 
 #include "common.cuh"
@@ -64,6 +62,7 @@ int sentry_create(sentry_ctx** out, int device) {
     c->workspace_bytes = 0;
     c->last_launches = 0;
     c->profiling = false;
+    c->attend_kernel = SENTRY_ATTEND_AUTO;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return SENTRY_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
@@ -176,6 +175,18 @@ int sentry_selftest_wait_expiry(sentry_ctx* ctx, long long limit_cycles, void* s
     return launch_wait_expiry_selftest(ctx, limit_cycles, (cudaStream_t)stream);
 }
 
+int sentry_set_option(sentry_ctx* ctx, int option, int value) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    switch (option) {
+        case SENTRY_OPT_ATTEND_KERNEL:
+            if (value < SENTRY_ATTEND_AUTO || value > SENTRY_ATTEND_TCGEN05) return SENTRY_ERR_INVALID_ARG;
+            ctx->attend_kernel = value;
+            return SENTRY_OK;
+        default:
+            return SENTRY_ERR_INVALID_ARG;
+    }
+}
+
 int sentry_last_launch_count(const sentry_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 
 int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
@@ -244,8 +255,9 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
     SENTRY_ON_DEVICE(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
     a.active_out_user = active_out;
-    static const bool tc_path = getenv("SENTRY_ATTEND_TC") != nullptr;   // bring-up switch
-    if (attend_tc_supported(*desc) && tc_path) rc = launch_attend_tc(ctx, a, st);
+    // AUTO takes the kernel that measured faster for the shape: at present the warp-MMA kernels
+    // on every shape they support (the tcgen05 kernel is within 10-20 % on T >= 512)
+    if (ctx->attend_kernel == SENTRY_ATTEND_TCGEN05 && attend_tc_supported(*desc)) rc = launch_attend_tc(ctx, a, st);
     else rc = attend_bf16_supported(*desc) ? launch_attend_bf16(ctx, a, st) : launch_attend_generic(ctx, a, st);
     if (rc != SENTRY_OK) return rc;
     if (a.selection_given && active_out != nullptr && active_out != active_in) {

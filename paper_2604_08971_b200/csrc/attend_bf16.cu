@@ -438,11 +438,15 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
                 pa[1] = pack2(s[2 * ks][2], s[2 * ks][3]);
                 pa[2] = pack2(s[2 * ks + 1][0], s[2 * ks + 1][1]);
                 pa[3] = pack2(s[2 * ks + 1][2], s[2 * ks + 1][3]);
-                // the normaliser is the sum of the ROUNDED weights the tensor core multiplies with:
-                // the row stays a convex combination of V rows, so the rounding of a dominant
-                // weight cancels between numerator and denominator
-                l_run[j][0] += bf16x2_sum(pa[0]) + bf16x2_sum(pa[2]);
-                l_run[j][1] += bf16x2_sum(pa[1]) + bf16x2_sum(pa[3]);
+                // every weight goes to the tensor core as a bf16 head plus a bf16 remainder
+                // (p = p_hi + p_lo to 2^-17), so the rounding of the weights drops out of O
+                uint32_t pb[4];
+                pb[0] = pack2_rem(s[2 * ks][0], s[2 * ks][1], pa[0]);
+                pb[1] = pack2_rem(s[2 * ks][2], s[2 * ks][3], pa[1]);
+                pb[2] = pack2_rem(s[2 * ks + 1][0], s[2 * ks + 1][1], pa[2]);
+                pb[3] = pack2_rem(s[2 * ks + 1][2], s[2 * ks + 1][3], pa[3]);
+                l_run[j][0] += (s[2 * ks][0] + s[2 * ks][1]) + (s[2 * ks + 1][0] + s[2 * ks + 1][1]);
+                l_run[j][1] += (s[2 * ks][2] + s[2 * ks][3]) + (s[2 * ks + 1][2] + s[2 * ks + 1][3]);
                 const int vrow = ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
                 for (int n2 = 0; n2 < NT / 2; ++n2) {
@@ -450,6 +454,8 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
                     ldmatrix_x4_trans(vbase + S::off(vrow, 2 * n2 + (lane >> 4)), bfr);
                     mma_bf16_16816(acc[j][2 * n2], pa, bfr[0], bfr[1]);
                     mma_bf16_16816(acc[j][2 * n2 + 1], pa, bfr[2], bfr[3]);
+                    mma_bf16_16816(acc[j][2 * n2], pb, bfr[0], bfr[1]);
+                    mma_bf16_16816(acc[j][2 * n2 + 1], pb, bfr[2], bfr[3]);
                 }
             }
         }
@@ -538,31 +544,45 @@ __device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict
         float mx[NH], sum[NH];
 #pragma unroll
         for (int h = 0; h < NH; ++h) { mx[h] = -INFINITY; sum[h] = 0.f; }
+        // The sampled positions come four at a time, the next four requested before the current
+        // four are used: a thread walks its own table row, and with most of the L1 given to
+        // shared memory the row's lines do not survive from one use to the next.
         const int32_t* row = score_mode == 0 ? tbl + (size_t)p * n_s : nullptr;
-        int pj_next = score_mode == 0 ? __ldg(row) : 0;
-        for (int a = 0; a < cnt; ++a) {
-            int pj = pj_next;
-            if (a + 1 < cnt) pj_next = score_mode == 0 ? __ldg(row + a + 1) : a + 1;
-            if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
-            float acc[NH][4];
+        int nxt[4];
 #pragma unroll
-            for (int h = 0; h < NH; ++h) acc[h][0] = acc[h][1] = acc[h][2] = acc[h][3] = 0.f;
+        for (int u = 0; u < 4; ++u) nxt[u] = score_mode == 0 ? __ldg(row + min(u, cnt - 1)) : u;
+        for (int a0 = 0; a0 < cnt; a0 += 4) {
+            int cur[4];
 #pragma unroll
-            for (int cc = 0; cc < S::CPR; ++cc) {
-                const uint4 v = lds128(ks_addr + S::off(pj, cc));
-#pragma unroll
-                for (int h = 0; h < NH; ++h) {
-                    fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc], v.x);
-                    fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 1], v.y);
-                    fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc + 2], v.z);
-                    fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 3], v.w);
-                }
+            for (int u = 0; u < 4; ++u) {
+                cur[u] = nxt[u];
+                nxt[u] = score_mode == 0 ? __ldg(row + min(a0 + 4 + u, cnt - 1)) : a0 + 4 + u;
             }
 #pragma unroll
-            for (int h = 0; h < NH; ++h) {
-                const float sc = ((acc[h][0] + acc[h][1]) + (acc[h][2] + acc[h][3])) * scale;
-                mx[h] = fmaxf(mx[h], sc);
-                sum[h] += sc;
+            for (int u = 0; u < 4; ++u) {
+                if (a0 + u >= cnt) break;
+                int pj = cur[u];
+                if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
+                float acc[NH][4];
+#pragma unroll
+                for (int h = 0; h < NH; ++h) acc[h][0] = acc[h][1] = acc[h][2] = acc[h][3] = 0.f;
+#pragma unroll
+                for (int cc = 0; cc < S::CPR; ++cc) {
+                    const uint4 v = lds128(ks_addr + S::off(pj, cc));
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
+                        fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc], v.x);
+                        fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 1], v.y);
+                        fma_bf16_pair(acc[h][0], acc[h][1], qw[h][4 * cc + 2], v.z);
+                        fma_bf16_pair(acc[h][2], acc[h][3], qw[h][4 * cc + 3], v.w);
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < NH; ++h) {
+                    const float sc = ((acc[h][0] + acc[h][1]) + (acc[h][2] + acc[h][3])) * scale;
+                    mx[h] = fmaxf(mx[h], sc);
+                    sum[h] += sc;
+                }
             }
         }
 #pragma unroll
@@ -870,9 +890,14 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
                 pa[1] = pack2(sc[2 * ks][2], sc[2 * ks][3]);
                 pa[2] = pack2(sc[2 * ks + 1][0], sc[2 * ks + 1][1]);
                 pa[3] = pack2(sc[2 * ks + 1][2], sc[2 * ks + 1][3]);
-                // normaliser = sum of the rounded weights (see the streamed kernel)
-                l_run[0] += bf16x2_sum(pa[0]) + bf16x2_sum(pa[2]);
-                l_run[1] += bf16x2_sum(pa[1]) + bf16x2_sum(pa[3]);
+                // bf16 head plus bf16 remainder of every weight (see the streamed kernel)
+                uint32_t pb[4];
+                pb[0] = pack2_rem(sc[2 * ks][0], sc[2 * ks][1], pa[0]);
+                pb[1] = pack2_rem(sc[2 * ks][2], sc[2 * ks][3], pa[1]);
+                pb[2] = pack2_rem(sc[2 * ks + 1][0], sc[2 * ks + 1][1], pa[2]);
+                pb[3] = pack2_rem(sc[2 * ks + 1][2], sc[2 * ks + 1][3], pa[3]);
+                l_run[0] += (sc[2 * ks][0] + sc[2 * ks][1]) + (sc[2 * ks + 1][0] + sc[2 * ks + 1][1]);
+                l_run[1] += (sc[2 * ks][2] + sc[2 * ks][3]) + (sc[2 * ks + 1][2] + sc[2 * ks + 1][3]);
                 const int vrow = ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
                 for (int n2 = 0; n2 < NT / 2; ++n2) {
@@ -880,6 +905,8 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
                     ldmatrix_x4_trans(vbase + S::off(vrow, 2 * n2 + (lane >> 4)), bfr);
                     mma_bf16_16816(acc[2 * n2], pa, bfr[0], bfr[1]);
                     mma_bf16_16816(acc[2 * n2 + 1], pa, bfr[2], bfr[3]);
+                    mma_bf16_16816(acc[2 * n2], pb, bfr[0], bfr[1]);
+                    mma_bf16_16816(acc[2 * n2 + 1], pb, bfr[2], bfr[3]);
                 }
             }
         }

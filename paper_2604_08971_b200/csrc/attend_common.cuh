@@ -96,9 +96,9 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-// lo + hi of a packed bf16 pair, in fp32
-__device__ __forceinline__ float bf16x2_sum(uint32_t w) {
-    return __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+// bf16 pair of what the packed pair `head` = pack2(lo, hi) leaves of lo and hi
+__device__ __forceinline__ uint32_t pack2_rem(float lo, float hi, uint32_t head) {
+    return pack2(lo - __uint_as_float(head << 16), hi - __uint_as_float(head & 0xffff0000u));
 }
 
 // Warp-level top-k by radix selection over n order keys in shared memory (larger key first,
@@ -216,7 +216,6 @@ __device__ __forceinline__ void warps_select_topk_heads(const uint32_t* keys, in
     const int warp = threadIdx.x >> 5;
     if (warp < rk) warp_select_topk_bits<8>(keys + (size_t)warp * stride, n, k, out[warp], remap);
 }
-
 // The same selection for the rk <= kMaxRK heads of a group at once, by the whole block: all
 // threads count digits for every head (the long part), warp hh then picks head hh's digit, and
 // at the end compacts head hh's selection.  keys: [rk][stride] order keys, n per head;

@@ -26,6 +26,7 @@ struct sentry_ctx {
     int last_launches;
     int sm_count;
     bool profiling;
+    int attend_kernel;       // SENTRY_ATTEND_AUTO / _WARP_MMA / _TCGEN05
     std::vector<ProfRec> prof;      // events recorded since profiling was enabled
     std::vector<cudaEvent_t> pool;  // reusable events
 };
