@@ -189,6 +189,29 @@ SENTRY_API int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc
                       int n_subsets, void* O, int32_t* active_out,
                       const int32_t* active_in, void* stream);
 
+/* The same with the pruned weights materialised ONCE, as Sec. 4.6 describes
+ * ("materialize a pruned model" per modality mask and budget), instead of on
+ * every call:
+ *   sentry_ffn_packed_bytes   size of the buffer for W1' and W2' of all lists
+ *                             (0 for an invalid descriptor; only D, F, k_c,
+ *                             n_lists and dtype matter)
+ *   sentry_ffn_prepack        gathers W1[:, N] and W2[N, :] of every list into
+ *                             `packed` (caller-owned device buffer of at least
+ *                             that size, 256-byte aligned; the layout is the
+ *                             library's own)
+ *   sentry_ffn_fwd_packed     sentry_ffn_fwd with `packed` in place of W1, W2 and
+ *                             kept_channels; the descriptor must have the same
+ *                             D, F, k_c, n_lists and dtype as at prepack time.
+ * The buffer stays valid until the weights or the kept lists change. */
+SENTRY_API size_t sentry_ffn_packed_bytes(const sentry_ffn_desc* desc);
+SENTRY_API int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* W1,
+                       const void* W2, const int32_t* kept_channels, void* packed,
+                       size_t packed_bytes, void* stream);
+SENTRY_API int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X,
+                          const void* packed, const int32_t* list_of_sample,
+                          const int32_t* token_modality_ids, const uint32_t* masks, void* Y,
+                          void* stream);
+
 /* Which kernels run Eq. 6 for bf16 tensors whose K/V of one KV group fit in
  * shared memory (T up to ~1.4 k at d = 32).  Two hand-written forms exist:
  *   SENTRY_ATTEND_WARP_MMA  K/V staged by 16-byte async copies, Q K^T and P V

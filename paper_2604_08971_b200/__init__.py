@@ -28,7 +28,8 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_num_active_queries", "sentry_workspace_bytes", "sentry_set_workspace",
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
-           "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option"]
+           "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
+           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -78,6 +79,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_last_launch_count.argtypes = [vp]
     lib.sentry_selftest_wait_expiry.argtypes = [vp, ctypes.c_longlong, vp]
     lib.sentry_set_option.argtypes = [vp, ci, ci]
+    lib.sentry_ffn_packed_bytes.argtypes = [ctypes.POINTER(FfnDesc)]
+    lib.sentry_ffn_packed_bytes.restype = ctypes.c_size_t
+    lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_profile_enable.argtypes = [vp, ci]
     lib.sentry_profile_slots.argtypes = []
     lib.sentry_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
@@ -85,7 +90,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_kernel_name.argtypes = [ci]
     lib.sentry_kernel_name.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("sentry_status_string", "sentry_workspace_bytes", "sentry_kernel_name"):
+        if name not in ("sentry_status_string", "sentry_workspace_bytes", "sentry_kernel_name",
+                        "sentry_ffn_packed_bytes"):
             getattr(lib, name).restype = ci
     if path is None:
         _lib = lib
@@ -279,4 +285,36 @@ class Sentry:
                                      _ptr(token_modality_ids), _ptr(masks), _ptr(Y), _stream())
         if rc != 0:
             raise SentryError(rc, "sentry_ffn_fwd")
+        return Y
+
+    def ffn_prepack(self, W1, W2, kept_channels, packed=None):
+        """sentry_ffn_prepack: materialise W1[:, N], W2[N, :] of every kept list once.  Returns the
+        packed buffer (a uint8 tensor) for ffn_fwd_packed."""
+        if kept_channels.dim() == 1:
+            kept_channels = kept_channels[None, :]
+        D, F = W1.shape
+        n_lists, k_c = kept_channels.shape
+        desc = FfnDesc(1, 1, D, F, k_c, n_lists, _dtype_code(W1))
+        nbytes = int(self.lib.sentry_ffn_packed_bytes(ctypes.byref(desc)))
+        if packed is None:
+            packed = torch.empty((nbytes,), dtype=torch.uint8, device=W1.device)
+        rc = self.lib.sentry_ffn_prepack(self.h, ctypes.byref(desc), _ptr(W1), _ptr(W2), _ptr(kept_channels),
+                                         _ptr(packed), packed.numel(), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_ffn_prepack")
+        return packed
+
+    def ffn_fwd_packed(self, X, packed, F: int, k_c: int, n_lists: int, list_of_sample=None,
+                       token_modality_ids=None, masks=None, Y=None):
+        """sentry_ffn_fwd_packed.  Returns Y [B,T,D]."""
+        B, T, D = X.shape
+        desc = FfnDesc(B, T, D, int(F), int(k_c), int(n_lists), _dtype_code(X))
+        if Y is None:
+            Y = torch.empty_like(X)
+        self.ensure_workspace(self.workspace_bytes(ffn=desc))
+        rc = self.lib.sentry_ffn_fwd_packed(self.h, ctypes.byref(desc), _ptr(X), _ptr(packed),
+                                            _ptr(list_of_sample), _ptr(token_modality_ids), _ptr(masks),
+                                            _ptr(Y), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_ffn_fwd_packed")
         return Y

@@ -293,7 +293,53 @@ int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, 
     a.Y = Y;
     a.status = ctx->d_status;
     SENTRY_ON_DEVICE(ctx->device);
-    return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, (cudaStream_t)stream);
+    return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, nullptr, (cudaStream_t)stream);
+}
+
+size_t sentry_ffn_packed_bytes(const sentry_ffn_desc* desc) {
+    return check_ffn_desc(desc) == SENTRY_OK ? ffn_packed_bytes(*desc) : 0;
+}
+
+int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* W1, const void* W2,
+                       const int32_t* kept_channels, void* packed, size_t packed_bytes, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_ffn_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (W1 == nullptr || W2 == nullptr || kept_channels == nullptr || packed == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(W1, 16) || !aligned(W2, 16) || !aligned(kept_channels, 4) || !aligned(packed, 256))
+        return SENTRY_ERR_INVALID_ARG;
+    if (packed_bytes < ffn_packed_bytes(*desc)) return SENTRY_ERR_WORKSPACE;
+    ctx->last_launches = 0;
+    FfnArgs a = {};
+    a.d = *desc;
+    a.W1 = W1; a.W2 = W2;
+    a.kept = kept_channels;
+    a.status = ctx->d_status;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_ffn_prepack(ctx, a, packed, (cudaStream_t)stream);
+}
+
+int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, const void* packed,
+                          const int32_t* list_of_sample, const int32_t* token_modality_ids,
+                          const uint32_t* masks, void* Y, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_ffn_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (X == nullptr || packed == nullptr || Y == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if ((token_modality_ids == nullptr) != (masks == nullptr)) return SENTRY_ERR_INVALID_ARG;
+    if (desc->n_lists > 1 && list_of_sample == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(packed, 256)) return SENTRY_ERR_INVALID_ARG;
+    ctx->last_launches = 0;
+    FfnArgs a = {};
+    a.d = *desc;
+    a.X = X;
+    a.list_of_sample = list_of_sample;
+    a.ids = token_modality_ids;
+    a.masks = masks;
+    a.Y = Y;
+    a.status = ctx->d_status;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, packed, (cudaStream_t)stream);
 }
 
 }  // extern "C"

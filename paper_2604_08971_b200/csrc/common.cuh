@@ -337,5 +337,7 @@ struct FfnArgs {
     unsigned int* status;
 };
 size_t ffn_workspace_bytes(const sentry_ffn_desc& d);
+size_t ffn_packed_bytes(const sentry_ffn_desc& d);
+int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStream_t st);
 int launch_wait_expiry_selftest(sentry_ctx* ctx, long long limit_cycles, cudaStream_t st);
-int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cudaStream_t st);
+int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, const void* packed, cudaStream_t st);

@@ -298,16 +298,25 @@ struct FfnWs {
     size_t used;
 };
 
-FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes) {
+// One of W1', W2' (all lists), rounded so that the second starts 256-byte aligned.
+size_t packed_half_bytes(const sentry_ffn_desc& d, int kc_pad) {
+    const size_t esz = d.dtype == SENTRY_F32 ? 4 : 2;
+    return align_up((size_t)d.n_lists * kc_pad * d.D * esz, 256);
+}
+
+// Row plan (and, unless the caller brings materialised weights, W1' and W2') from the workspace.
+FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes, bool with_weights) {
     WsAlloc a(ws, bytes);
     FfnWs w;
-    const size_t esz = d.dtype == SENTRY_F32 ? 4 : 2;
     w.plan.sample_row0 = a.take<int32_t>(d.B);
     w.plan.list_row0 = a.take<int32_t>(d.n_lists + 1);
     w.plan.tile_start = a.take<int32_t>(d.n_lists + 1);
     w.plan.rowidx = a.take<int32_t>((size_t)d.B * d.T);
-    w.w1p = a.take<uint8_t>((size_t)d.n_lists * kc_pad * d.D * esz);
-    w.w2p = a.take<uint8_t>((size_t)d.n_lists * kc_pad * d.D * esz);
+    w.w1p = w.w2p = nullptr;
+    if (with_weights) {
+        w.w1p = a.take<uint8_t>(packed_half_bytes(d, kc_pad));
+        w.w2p = a.take<uint8_t>(packed_half_bytes(d, kc_pad));
+    }
     w.ok = a.ok;
     w.used = a.off;
     return w;
@@ -321,15 +330,49 @@ int kc_pad_for(const sentry_ffn_desc& d) {
 }  // namespace
 
 size_t ffn_workspace_bytes(const sentry_ffn_desc& d) {
-    return carve(d, kc_pad_for(d), nullptr, 0).used + 256;
+    return carve(d, kc_pad_for(d), nullptr, 0, true).used + 256;
 }
 
-int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cudaStream_t st) {
+size_t ffn_packed_bytes(const sentry_ffn_desc& d) { return 2 * packed_half_bytes(d, kc_pad_for(d)); }
+
+// The weight gather alone: W1' = W1[:, N], W2' = W2[N, :] for every list into `packed`.
+int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStream_t st) {
     const sentry_ffn_desc& d = a.d;
     const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
     const int kc_pad = kc_pad_for(d);
-    FfnWs w = carve(d, kc_pad, ws, ws_bytes);
+    const size_t per = (size_t)kc_pad * d.D;
+    const size_t pack_blocks = tc ? 2 * (size_t)d.n_lists * (kc_pad / 32) * (d.D / 64)
+                                  : 2 * (size_t)d.n_lists * ((per + 255) / 256);
+    uint8_t* w1p = (uint8_t*)packed;
+    uint8_t* w2p = w1p + packed_half_bytes(d, kc_pad);
+    FfnPlan none = {};
+    LaunchScope ls(ctx, KS_FFN_PREPARE, st);
+    // no row-table and no zero-fill blocks (B = 0, no ids): every block gathers weights
+    if (d.dtype == SENTRY_F32)
+        ffn_prepare_kernel<float><<<(unsigned)pack_blocks, 256, 0, st>>>(
+            nullptr, nullptr, nullptr, 0, d.T, 1, kGenericTileRows, none, nullptr, (const float*)a.W1,
+            (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, (float*)w1p, (float*)w2p, a.status);
+    else
+        ffn_prepare_kernel<__nv_bfloat16><<<(unsigned)pack_blocks, 256, 0, st>>>(
+            nullptr, nullptr, nullptr, 0, d.T, 1, tc ? kTcTileRows : kGenericTileRows, none, nullptr,
+            (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad,
+            tc ? 1 : 0, (__nv_bfloat16*)w1p, (__nv_bfloat16*)w2p, a.status);
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}
+
+// packed == nullptr: gather the weights into the workspace first (every call); otherwise use the
+// caller's materialised W1', W2' (launch_ffn_prepack) and only build the row plan.
+int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, const void* packed, cudaStream_t st) {
+    const sentry_ffn_desc& d = a.d;
+    const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
+    const int kc_pad = kc_pad_for(d);
+    FfnWs w = carve(d, kc_pad, ws, ws_bytes, packed == nullptr);
     if (!w.ok) return SENTRY_ERR_WORKSPACE;
+    if (packed != nullptr) {
+        w.w1p = const_cast<void*>(packed);
+        w.w2p = (uint8_t*)w.w1p + packed_half_bytes(d, kc_pad);
+    }
     const int tile_rows = tc ? kTcTileRows : kGenericTileRows;
 
     {
@@ -338,8 +381,9 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, cud
         int zsplit = (4 * ctx->sm_count + d.B - 1) / d.B;
         if (zsplit < 1) zsplit = 1;
         if (zsplit > 32) zsplit = 32;
-        const size_t pack_blocks = tc ? 2 * (size_t)d.n_lists * (kc_pad / 32) * (d.D / 64)
-                                      : 2 * (size_t)d.n_lists * ((per + 255) / 256);
+        const size_t pack_blocks = packed != nullptr ? 0
+                                   : (tc ? 2 * (size_t)d.n_lists * (kc_pad / 32) * (d.D / 64)
+                                         : 2 * (size_t)d.n_lists * ((per + 255) / 256));
         const size_t grid = (size_t)d.B + (a.ids != nullptr ? (size_t)d.B * zsplit : 0) + pack_blocks;
         LaunchScope ls(ctx, KS_FFN_PREPARE, st);
         if (d.dtype == SENTRY_F32)

@@ -286,3 +286,28 @@ def test_bounded_wait_expires_and_context_survives(sn):
     assert err <= TOL["bf16"]
     with pytest.raises(sentry.SentryError):
         sn.selftest_wait_expiry(0)
+
+
+def test_ffn_with_weights_materialised_once(sn):
+    """sentry_ffn_prepack + sentry_ffn_fwd_packed: the pruned weights are gathered once (Section 4.6)
+    and reused; results bit-identical to sentry_ffn_fwd and within tolerance of the oracle."""
+    for w in (synth.config1(), synth.config2().with_(B=40), synth.config4().with_(B=24), synth.config5(16, 256)):
+        inp = synth.generate(w, n_s_of)
+        _, kept_c = parity.gate_lists(sn, inp)
+        X, W1, W2 = inp.X.cuda(), inp.W1.cuda(), inp.W2.cuda()
+        los, ids, masks = dev(inp.list_of_sample), dev(inp.ids), masks_dev(inp.masks)
+        packed = sn.ffn_prepack(W1, W2, kept_c)
+        Y_ref = sn.ffn_fwd(X, W1, W2, kept_c, los, ids, masks).clone()
+        for _ in range(2):   # the packed buffer is reused
+            Y = sn.ffn_fwd_packed(X, packed, w.F, w.k_c, kept_c.shape[0], los, ids, masks)
+            assert torch.equal(Y.view(torch.int16 if w.dtype == "bf16" else torch.int32),
+                               Y_ref.view(torch.int16 if w.dtype == "bf16" else torch.int32))
+        want = oracle.ffn(inp.X, inp.W1, inp.W2, kept_c.cpu().numpy(), inp.list_of_sample, inp.ids, inp.masks)
+        got = Y.float().cpu().numpy()
+        err = parity.rel_err(got, want, w.dtype, np.ones(got.shape[:2], dtype=bool))
+        parity.record(w.name, "ffn_pk", err, parity.raw_rel_err(got, want), "weights materialised once")
+        assert err <= TOL[w.dtype]
+        assert sn.last_status() == 0
+    with pytest.raises(sentry.SentryError) as e:   # buffer too small: refused on the host
+        sn.ffn_prepack(W1, W2, kept_c, packed=torch.empty((256,), dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -4
