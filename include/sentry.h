@@ -113,6 +113,35 @@ SENTRY_API int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, i
                        uint32_t* kv_groups, int heads_per_group, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * SentryGate on the device (Sec. 4.2, Eq. 1) and the cross-layer threshold of
+ * Sec. 4.6 ("evaluate the gate outputs for all layers, then apply a global
+ * threshold determined by a desired pruning ratio").
+ *
+ * Units of all layers are concatenated: layer l owns the unit indices
+ * [layer_offsets[l], layer_offsets[l+1]), layer_offsets[n_layers] = n_units.
+ *   z_i(s) = zeta[i] + gamma[l(i)] * f_i(m_s),   g_i(s) = 1 / (1 + exp(-z_i(s)))
+ *   f_i(m) = w2[i,:] . relu(W1[i,:,:] m + b1[i,:]) + b2[i]
+ * with m_s in {0,1}^M the bits of the mask value s (bit j = modality j present).
+ * The paper says "a two-layer MLP with a nonlinearity"; ReLU is this library's
+ * reading.  All parameters fp32, device:
+ *   zeta [n_units], gamma [n_layers], W1 [n_units, hidden, M], b1, w2 [n_units, hidden], b2 [n_units]
+ *   logits out [2^M, n_units] (row index = mask value): the score table for
+ *          sentry_gate_select -- ranking z equals ranking g and does not saturate
+ *   gates  out [2^M, n_units] or NULL: g itself
+ * The global threshold is then sentry_gate_select(logits, S = 2^M, n_units,
+ * masks, k = units kept over ALL layers); sentry_gate_layer_counts turns the
+ * kept lists [n_masks, k] (ascending) into counts [n_masks, n_layers] per layer
+ * (the kept units of layer l are the next counts[l] entries of the list).
+ */
+SENTRY_API int sentry_gate_eval(sentry_ctx* ctx, int M, int hidden, int n_layers,
+                     const int32_t* layer_offsets, int n_units, const float* zeta,
+                     const float* gamma, const float* W1, const float* b1, const float* w2,
+                     const float* b2, float* logits, float* gates, void* stream);
+SENTRY_API int sentry_gate_layer_counts(sentry_ctx* ctx, const int32_t* kept, int n_masks, int k,
+                             const int32_t* layer_offsets, int n_layers, int32_t* counts,
+                             void* stream);
+
+/* ---------------------------------------------------------------------------
  * Gate selection for callers that cannot allocate device memory.
  *
  * (No counterpart in the paper: this is a deployment convenience, not part of

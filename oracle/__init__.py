@@ -161,3 +161,18 @@ def ffn(X, W1, W2, kept_channels, list_of_sample=None, ids=None, masks=None) -> 
     _load().oracle_ffn(_p(X), _p(W1), _p(W2), B, T, D, F, _p(kc), kc.shape[1],
                        _p(los), _p(ii), _p(mk), _p(Y))
     return Y
+
+
+def gate_eval(layer_offsets, zeta, gamma, W1, b1, w2, b2):
+    """SentryGate (Eq. 1) for every mask value: returns (z, g), both [2^M, n_units] float64.
+    W1 [n_units, hidden, M]; b1, w2 [n_units, hidden]; zeta, b2 [n_units]; gamma [n_layers]."""
+    lo = _i32(layer_offsets)
+    zeta, gamma, W1, b1, w2, b2 = (_f64(x) for x in (zeta, gamma, W1, b1, w2, b2))
+    n_units, hidden, M = W1.shape
+    n_layers = gamma.shape[0]
+    assert lo.shape == (n_layers + 1,) and lo[0] == 0 and lo[-1] == n_units
+    z = np.empty((1 << M, n_units), dtype=np.float64)
+    g = np.empty_like(z)
+    _load().oracle_gate_eval(int(M), int(hidden), int(n_layers), _p(lo), int(n_units), _p(zeta), _p(gamma),
+                             _p(W1), _p(b1), _p(w2), _p(b2), _p(z), _p(g))
+    return z, g

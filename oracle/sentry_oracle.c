@@ -20,6 +20,8 @@
  *                          GQA duplication, rows of softmax sum to 1,
  *                          dropping == deleting, brute-force sparsity score
  *   oracle_ffn             library matmul + erf, masked full FFN
+ *   oracle_gate_eval       library matmul form of the perceptron, closed forms
+ *                          (zero first layer, gamma = 0, one hidden unit by hand)
  * The paper's GFLOP figures and accuracies need undisclosed architectures and
  * data: parity unpinned for those (they are not computed here).
  */
@@ -300,4 +302,35 @@ void oracle_ffn(const double* X, const double* W1, const double* W2,
         }
         free(h);
     }
+}
+
+/* ---- SentryGate score function (Section 4.2, Eq. 1):
+ *   g_i(m) = sigmoid( zeta_i + gamma_l * f_i(m) ),  f_i = a two-layer perceptron on the mask m.
+ * The paper names neither the hidden width nor the nonlinearity; ReLU is the reading taken:
+ *   f_i(m) = sum_j w2[i][j] * max(0, b1[i][j] + sum_q W1[i][j][q] * m_q) + b2[i].
+ * Units of all layers are concatenated; layer l owns [layer_offsets[l], layer_offsets[l+1]).
+ * Writes z (the argument of the sigmoid) and g for every mask value s (m_q = bit q of s). */
+void oracle_gate_eval(int M, int hidden, int n_layers, const int32_t* layer_offsets, int n_units,
+                      const double* zeta, const double* gamma, const double* W1, const double* b1,
+                      const double* w2, const double* b2, double* z_out, double* g_out) {
+    const int S = 1 << M;
+    for (int s = 0; s < S; ++s) {
+        for (int l = 0; l < n_layers; ++l) {
+            for (int i = layer_offsets[l]; i < layer_offsets[l + 1]; ++i) {
+                double f = b2[i];
+                for (int j = 0; j < hidden; ++j) {
+                    double a = b1[(size_t)i * hidden + j];
+                    for (int q = 0; q < M; ++q) {
+                        const double m_q = (double)((s >> q) & 1);
+                        a += W1[((size_t)i * hidden + j) * M + q] * m_q;
+                    }
+                    f += w2[(size_t)i * hidden + j] * (a > 0.0 ? a : 0.0);
+                }
+                const double z = zeta[i] + gamma[l] * f;
+                z_out[(size_t)s * n_units + i] = z;
+                g_out[(size_t)s * n_units + i] = 1.0 / (1.0 + exp(-z));
+            }
+        }
+    }
+    (void)n_units;
 }

@@ -29,7 +29,8 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
-           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed"]
+           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
+           "sentry_gate_eval", "sentry_gate_layer_counts"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -79,6 +80,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_last_launch_count.argtypes = [vp]
     lib.sentry_selftest_wait_expiry.argtypes = [vp, ctypes.c_longlong, vp]
     lib.sentry_set_option.argtypes = [vp, ci, ci]
+    lib.sentry_gate_eval.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sentry_gate_layer_counts.argtypes = [vp, vp, ci, ci, vp, ci, vp, vp]
     lib.sentry_ffn_packed_bytes.argtypes = [ctypes.POINTER(FfnDesc)]
     lib.sentry_ffn_packed_bytes.restype = ctypes.c_size_t
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -318,3 +321,28 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_ffn_fwd_packed")
         return Y
+
+    def gate_eval(self, layer_offsets, zeta, gamma, W1, b1, w2, b2, return_gates: bool = False):
+        """sentry_gate_eval: logits (and gates) [2^M, n_units] of SentryGate's per-unit MLP (Eq. 1)."""
+        n_units, hidden, M = W1.shape
+        n_layers = gamma.shape[0]
+        S = 1 << M
+        logits = torch.empty((S, n_units), dtype=torch.float32, device=W1.device)
+        gates = torch.empty_like(logits) if return_gates else None
+        rc = self.lib.sentry_gate_eval(self.h, M, hidden, n_layers, _ptr(layer_offsets), n_units, _ptr(zeta),
+                                       _ptr(gamma), _ptr(W1), _ptr(b1), _ptr(w2), _ptr(b2), _ptr(logits),
+                                       _ptr(gates), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_gate_eval")
+        return (logits, gates) if return_gates else logits
+
+    def gate_layer_counts(self, kept, layer_offsets):
+        """sentry_gate_layer_counts: kept [n_masks, k] ascending -> counts [n_masks, n_layers]."""
+        n_masks, k = kept.shape
+        n_layers = layer_offsets.shape[0] - 1
+        counts = torch.empty((n_masks, n_layers), dtype=torch.int32, device=kept.device)
+        rc = self.lib.sentry_gate_layer_counts(self.h, _ptr(kept), n_masks, k, _ptr(layer_offsets), n_layers,
+                                               _ptr(counts), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_gate_layer_counts")
+        return counts

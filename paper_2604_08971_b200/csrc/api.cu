@@ -96,7 +96,7 @@ int sentry_profile_slots(void) { return KS_COUNT; }
 
 const char* sentry_kernel_name(int slot) {
     static const char* names[KS_COUNT] = {"gate_rows", "gate_expand", "attend_score", "attend_select",
-                                          "attend_core", "ffn_prepare", "ffn_main"};
+                                          "attend_core", "ffn_prepare", "ffn_main", "gate_eval"};
     return (slot >= 0 && slot < KS_COUNT) ? names[slot] : "?";
 }
 
@@ -210,6 +210,30 @@ int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
     SENTRY_ON_DEVICE(ctx->device);
     return launch_gate_select(ctx, scores, S, n_units, masks, n_masks, k, kept, kv_groups,
                               heads_per_group, rows, groups, (cudaStream_t)stream);
+}
+
+int sentry_gate_eval(sentry_ctx* ctx, int M, int hidden, int n_layers, const int32_t* layer_offsets,
+                     int n_units, const float* zeta, const float* gamma, const float* W1, const float* b1,
+                     const float* w2, const float* b2, float* logits, float* gates, void* stream) {
+    if (ctx == nullptr || layer_offsets == nullptr || zeta == nullptr || gamma == nullptr || W1 == nullptr ||
+        b1 == nullptr || w2 == nullptr || b2 == nullptr || logits == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (M < 1 || M > 16 || hidden < 1 || hidden > 4096 || n_layers < 1 || n_units < 1) return SENTRY_ERR_BAD_SHAPE;
+    if (n_units > kMaxUnits) return SENTRY_ERR_UNSUPPORTED;
+    ctx->last_launches = 0;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_gate_eval(ctx, zeta, gamma, layer_offsets, n_layers, W1, b1, w2, b2, M, hidden, n_units, logits,
+                            gates, (cudaStream_t)stream);
+}
+
+int sentry_gate_layer_counts(sentry_ctx* ctx, const int32_t* kept, int n_masks, int k,
+                             const int32_t* layer_offsets, int n_layers, int32_t* counts, void* stream) {
+    if (ctx == nullptr || kept == nullptr || layer_offsets == nullptr || counts == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (n_masks < 0 || k < 1 || n_layers < 1) return SENTRY_ERR_BAD_SHAPE;
+    ctx->last_launches = 0;
+    if (n_masks == 0) return SENTRY_OK;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_layer_counts(ctx, kept, n_masks, k, layer_offsets, n_layers, counts, (cudaStream_t)stream);
 }
 
 int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const void* Q,

@@ -13,7 +13,7 @@
 // Kernel slots for launch accounting and optional per-kernel timing.
 enum KernelSlot {
     KS_GATE_ROWS = 0, KS_GATE_EXPAND, KS_ATT_SCORE, KS_ATT_SELECT, KS_ATT_CORE,
-    KS_FFN_PREPARE, KS_FFN_MAIN, KS_COUNT
+    KS_FFN_PREPARE, KS_FFN_MAIN, KS_GATE_EVAL, KS_COUNT
 };
 
 struct ProfRec { cudaEvent_t start, stop; int slot; };
@@ -302,6 +302,12 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                        const uint32_t* masks, int n_masks, int k, int32_t* kept,
                        uint32_t* kv_groups, int heads_per_group, int32_t* ws_rows,
                        uint32_t* ws_groups, cudaStream_t st);
+
+int launch_gate_eval(sentry_ctx* ctx, const float* zeta, const float* gamma, const int32_t* layer_offsets,
+                     int n_layers, const float* W1, const float* b1, const float* w2, const float* b2, int M,
+                     int hidden, int N, float* logits, float* gates, cudaStream_t st);
+int launch_layer_counts(sentry_ctx* ctx, const int32_t* kept, int n_masks, int k, const int32_t* layer_offsets,
+                        int n_layers, int32_t* counts, cudaStream_t st);
 
 struct AttendArgs {
     sentry_attend_desc d;

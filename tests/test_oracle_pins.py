@@ -364,3 +364,63 @@ def test_generators_are_seeded_and_shaped_like_the_configs():
         tbl = i5.sample_table[off:off + tv * n_s].reshape(tv, n_s)
         assert tbl.min() >= 0 and tbl.max() < tv
         assert np.all(np.diff(tbl, axis=1) > 0)      # distinct, ascending
+
+
+# ----------------------------------------------------------------- SentryGate MLP
+def _gate_params(g, n_layers, units, hidden, M):
+    lo = np.concatenate([[0], np.cumsum(units)]).astype(np.int32)
+    N = int(lo[-1])
+    return (lo, g.standard_normal(N), g.standard_normal(n_layers), g.standard_normal((N, hidden, M)),
+            g.standard_normal((N, hidden)), g.standard_normal((N, hidden)), g.standard_normal(N))
+
+
+def test_gate_eval_equals_library_matmul_form():
+    # Eq. 1 with the perceptron written as library matrix products over all masks at once
+    g = np.random.default_rng(31)
+    M, hidden, units = 3, 5, [4, 7, 2]
+    lo, zeta, gamma, W1, b1, w2, b2 = _gate_params(g, 3, units, hidden, M)
+    z, gt = oracle.gate_eval(lo, zeta, gamma, W1, b1, w2, b2)
+    masks = np.array([[(s >> q) & 1 for q in range(M)] for s in range(1 << M)], dtype=np.float64)   # [S, M]
+    hid = np.maximum(np.einsum("ijq,sq->sij", W1, masks) + b1[None], 0.0)                          # [S, N, hidden]
+    f = np.einsum("sij,ij->si", hid, w2) + b2[None]
+    gam = np.repeat(gamma, units)
+    want_z = zeta[None] + gam[None] * f
+    np.testing.assert_allclose(z, want_z, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(gt, 1.0 / (1.0 + np.exp(-want_z)), rtol=1e-12, atol=1e-12)
+
+
+def test_gate_eval_closed_forms():
+    g = np.random.default_rng(32)
+    M, hidden, units = 2, 3, [3, 3]
+    lo, zeta, gamma, W1, b1, w2, b2 = _gate_params(g, 2, units, hidden, M)
+    # gamma = 0: the gate is sigmoid(zeta) whatever the mask (Eq. 1)
+    z, gt = oracle.gate_eval(lo, zeta, np.zeros(2), W1, b1, w2, b2)
+    np.testing.assert_allclose(gt, np.tile(1.0 / (1.0 + np.exp(-zeta)), (4, 1)), rtol=1e-13)
+    # zero first-layer weights: f is the constant w2 . relu(b1) + b2
+    z, _ = oracle.gate_eval(lo, zeta, gamma, np.zeros_like(W1), b1, w2, b2)
+    const = (w2 * np.maximum(b1, 0)).sum(1) + b2
+    np.testing.assert_allclose(z, np.tile(zeta + np.repeat(gamma, units) * const, (4, 1)), rtol=1e-13)
+    # one unit, one hidden unit, by hand: W1 = [2, -3], b1 = 0.5, w2 = 4, b2 = -1, zeta = 0.25, gamma = 0.5
+    z, gt = oracle.gate_eval([0, 1], [0.25], [0.5], [[[2.0, -3.0]]], [[0.5]], [[4.0]], [-1.0])
+    # masks 0..3: a = 0.5, 2.5, -2.5, -0.5 -> relu 0.5, 2.5, 0, 0 -> f = 1, 9, -1, -1 -> z = .75, 4.75, -.25, -.25
+    np.testing.assert_allclose(z[:, 0], [0.75, 4.75, -0.25, -0.25], rtol=1e-15)
+    assert abs(gt[0, 0] - 1.0 / (1.0 + math.exp(-0.75))) < 1e-15
+    # an absent modality's first-layer column has no effect: masks that differ only there agree
+    z, _ = oracle.gate_eval(lo, zeta, gamma, W1 * np.array([1.0, 0.0]), b1, w2, b2)
+    np.testing.assert_array_equal(z[0], z[2])
+    np.testing.assert_array_equal(z[1], z[3])
+
+
+def test_global_threshold_is_topk_over_all_layers():
+    # Section 4.6: one threshold over the gate outputs of all layers = top-k of the concatenated row
+    g = np.random.default_rng(33)
+    lo, zeta, gamma, W1, b1, w2, b2 = _gate_params(g, 3, [6, 10, 5], 4, 3)
+    z, gt = oracle.gate_eval(lo, zeta, gamma, W1, b1, w2, b2)
+    masks = np.arange(1, 8, dtype=np.uint32)
+    k = 9
+    kept = oracle.gate_select(z.astype(np.float32), masks, k)
+    for r, s in enumerate(masks):
+        order = np.argsort(-z[s].astype(np.float32), kind="stable")[:k]
+        np.testing.assert_array_equal(kept[r], np.sort(order))
+        thr = np.sort(gt[s])[-k]                 # the threshold on g itself keeps the same units
+        assert set(np.nonzero(gt[s] >= thr)[0]) == set(kept[r].tolist())
