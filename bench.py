@@ -37,7 +37,7 @@ L2_BYTES = 126 * 1024 * 1024
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
 # keyed by (kernel slot, workload); None once the kernel has changed since its capture.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {("attend_core", "cfg4_full_layer"): 40.67e6, ("ffn_main", "cfg4_full_layer"): 36.70e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -474,7 +474,7 @@ def run_ours(args, w: synth.Workload):
 
     # ---- the same step with the pruned FFN weights materialised once (Section 4.6)
     once = None
-    if world == 1:
+    if world == 1 and not args.no_once:
         wb1 = Workbench(sentry, w, dev, local_rank, rank, not args.no_overlap, not args.no_graph,
                         ATTEND_KERNELS[args.attend_kernel], materialise_once=True)
         b1 = wb1.time_blocks(args.steps, max(3, args.replays // 2 + 1), args.warmup)
@@ -535,16 +535,18 @@ def run_ours(args, w: synth.Workload):
         torch.cuda.synchronize()
 
     n_e2e = max(3, min(args.steps, 20))
-    for _ in range(3):
-        e2e_step()
-    barrier_sync()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(n_e2e):
-        e2e_step()
-    ev1.record()
-    barrier_sync()
-    e2e_tokens, e2e_ms = aggregate(float(wm["tokens"]) * n_e2e, ev0.elapsed_time(ev1), dev)
+    e2e_tokens, e2e_ms = None, None
+    if not args.no_e2e:
+        for _ in range(3):
+            e2e_step()
+        barrier_sync()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        ev1.record()
+        barrier_sync()
+        e2e_tokens, e2e_ms = aggregate(float(wm["tokens"]) * n_e2e, ev0.elapsed_time(ev1), dev)
     status = wb.status()
     launches = wb.launches
     graphs_on = wb.graphs is not None
@@ -628,7 +630,7 @@ def run_ours(args, w: synth.Workload):
         "block_ms": blocks, "replays": args.replays,
         "useful_tflops": (wm["att_flops"] + wm["ffn_flops"]) * world * args.steps / (ms * 1e-3) / 1e12,
         "materialised_once": once,
-        "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+        "e2e": None if e2e_ms is None else {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": n_e2e,
                 "pipeline": "%d sample chunks; upload, kernels and download on three streams" % n_chunks},
         "gpu_launches": launches * args.steps,
@@ -653,6 +655,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the table of the other named workloads and sweep cells")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (for profiler launch lists)")
+    ap.add_argument("--no-once", action="store_true", help="skip the materialised-once leg (for profiler launch lists)")
     ap.add_argument("--replays", type=int, default=5, help="timed blocks of --steps steps; the median is reported")
     ap.add_argument("--attend-kernel", default="auto", choices=sorted(ATTEND_KERNELS),
                     help="SENTRY_OPT_ATTEND_KERNEL for the attention call")
