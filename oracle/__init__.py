@@ -176,3 +176,29 @@ def gate_eval(layer_offsets, zeta, gamma, W1, b1, w2, b2):
     _load().oracle_gate_eval(int(M), int(hidden), int(n_layers), _p(lo), int(n_units), _p(zeta), _p(gamma),
                              _p(W1), _p(b1), _p(w2), _p(b2), _p(z), _p(g))
     return z, g
+
+
+def project_qkv(X, WQ, WK, WV, kept_heads, ids, masks, Hq: int, Hk: int, d: int):
+    """Pruned Q/K/V projections (Section 4.6): only the column blocks of the kept heads / referenced
+    KV groups, only present tokens; everything else zero.  Returns Q [B,Hq,T,d], K, V [B,Hk,T,d]."""
+    X, WQ, WK, WV = (_f64(x) for x in (X, WQ, WK, WV))
+    kh, ii, mk = _i32(kept_heads), _i32(ids), _u32(masks)
+    B, T, D = X.shape
+    assert WQ.shape == (D, Hq * d) and WK.shape == (D, Hk * d) and WV.shape == (D, Hk * d)
+    Q = np.empty((B, Hq, T, d)); K = np.empty((B, Hk, T, d)); V = np.empty((B, Hk, T, d))
+    _load().oracle_project_qkv(_p(X), _p(WQ), _p(WK), _p(WV), B, T, D, Hq, Hk, d, _p(kh), kh.shape[1],
+                               _p(ii), _p(mk), _p(Q), _p(K), _p(V))
+    return Q, K, V
+
+
+def project_out(A, WO, kept_heads, ids, masks, Hq: int):
+    """Pruned output projection: A [B,k_h,T,d] (kept-list order) times the kept row blocks of W_O
+    [Hq d, D]; rows of absent tokens zero.  Returns [B,T,D]."""
+    A, WO = _f64(A), _f64(WO)
+    kh, ii, mk = _i32(kept_heads), _i32(ids), _u32(masks)
+    B, k_h, T, d = A.shape
+    D = WO.shape[1]
+    assert WO.shape == (Hq * d, D) and kh.shape == (B, k_h)
+    out = np.empty((B, T, D))
+    _load().oracle_project_out(_p(A), _p(WO), B, T, D, Hq, d, _p(kh), k_h, _p(ii), _p(mk), _p(out))
+    return out

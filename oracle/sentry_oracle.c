@@ -20,6 +20,8 @@
  *                          GQA duplication, rows of softmax sum to 1,
  *                          dropping == deleting, brute-force sparsity score
  *   oracle_ffn             library matmul + erf, masked full FFN
+ *   oracle_project_qkv/out library matmul on sliced and on masked full weight matrices;
+ *                          unpruned chain == textbook multi-head attention layer
  *   oracle_gate_eval       library matmul form of the perceptron, closed forms
  *                          (zero first layer, gamma = 0, one hidden unit by hand)
  * The paper's GFLOP figures and accuracies need undisclosed architectures and
@@ -333,4 +335,67 @@ void oracle_gate_eval(int M, int hidden, int n_layers, const int32_t* layer_offs
         }
     }
     (void)n_units;
+}
+
+/* ---- Head pruning with GQA consistency (Section 4.6): the projections of a pruned layer.
+ * "Given the query projection W_Q in R^{d_model x H_q d_h}, we keep only the column blocks
+ * associated with H_keep ... K_keep = floor(H_keep / (H_q/H_k)) and apply analogous block
+ * filtering to W_K and W_V."  For every sample b and present token t:
+ *   Q[b,h,t,:] = x_t . W_Q[:, h d : (h+1) d]        for h in H_keep(b)
+ *   K[b,g,t,:] = x_t . W_K[:, g d : (g+1) d],  V likewise,  for g in K_keep(b)
+ * Everything else (pruned heads, unreferenced groups, absent tokens) is left at zero here.
+ * X [B,T,D]; W_Q [D, Hq d]; W_K, W_V [D, Hk d]; outputs Q [B,Hq,T,d], K, V [B,Hk,T,d]. */
+void oracle_project_qkv(const double* X, const double* WQ, const double* WK, const double* WV, int B, int T, int D,
+                        int Hq, int Hk, int d, const int32_t* kept_heads, int k_h, const int32_t* ids,
+                        const uint32_t* masks, double* Q, double* K, double* V) {
+    const int r = Hq / Hk;
+    memset(Q, 0, sizeof(double) * (size_t)B * Hq * T * d);
+    memset(K, 0, sizeof(double) * (size_t)B * Hk * T * d);
+    memset(V, 0, sizeof(double) * (size_t)B * Hk * T * d);
+#pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int t = 0; t < T; ++t) {
+            if (!((masks[b] >> ids[t]) & 1u)) continue;
+            const double* x = X + ((size_t)b * T + t) * D;
+            for (int j = 0; j < k_h; ++j) {
+                const int h = kept_heads[(size_t)b * k_h + j];
+                const int g = h / r;
+                for (int c = 0; c < d; ++c) {
+                    double q = 0.0, kk = 0.0, vv = 0.0;
+                    for (int e = 0; e < D; ++e) {
+                        q += x[e] * WQ[(size_t)e * Hq * d + h * d + c];
+                        kk += x[e] * WK[(size_t)e * Hk * d + g * d + c];
+                        vv += x[e] * WV[(size_t)e * Hk * d + g * d + c];
+                    }
+                    Q[(((size_t)b * Hq + h) * T + t) * d + c] = q;
+                    K[(((size_t)b * Hk + g) * T + t) * d + c] = kk;   /* same value from every head of the group */
+                    V[(((size_t)b * Hk + g) * T + t) * d + c] = vv;
+                }
+            }
+        }
+    }
+}
+
+/* Output projection of the pruned layer: the row blocks of W_O that belong to the kept heads.
+ * (The paper never writes W_O; this is the transpose of the rule it states for W_Q: a pruned head
+ * contributes nothing, so its rows of W_O drop out.)
+ *   out[b,t,:] = sum_j A[b,j,t,:] . W_O[h_j d : (h_j+1) d, :]   for present t, else 0
+ * A [B,k_h,T,d] (heads in kept-list order); W_O [Hq d, D]; out [B,T,D]. */
+void oracle_project_out(const double* A, const double* WO, int B, int T, int D, int Hq, int d,
+                        const int32_t* kept_heads, int k_h, const int32_t* ids, const uint32_t* masks, double* out) {
+    memset(out, 0, sizeof(double) * (size_t)B * T * D);
+    (void)Hq;
+#pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int t = 0; t < T; ++t) {
+            if (!((masks[b] >> ids[t]) & 1u)) continue;
+            double* o = out + ((size_t)b * T + t) * D;
+            for (int j = 0; j < k_h; ++j) {
+                const int h = kept_heads[(size_t)b * k_h + j];
+                const double* a = A + (((size_t)b * k_h + j) * T + t) * d;
+                for (int c = 0; c < d; ++c)
+                    for (int e = 0; e < D; ++e) o[e] += a[c] * WO[(size_t)(h * d + c) * D + e];
+            }
+        }
+    }
 }

@@ -424,3 +424,65 @@ def test_global_threshold_is_topk_over_all_layers():
         np.testing.assert_array_equal(kept[r], np.sort(order))
         thr = np.sort(gt[s])[-k]                 # the threshold on g itself keeps the same units
         assert set(np.nonzero(gt[s] >= thr)[0]) == set(kept[r].tolist())
+
+
+# ------------------------------------------------------------ pruned projections
+def test_pruned_projections_equal_sliced_and_masked_full_projections():
+    """Section 4.6: keeping the column blocks of W_Q (and of W_K, W_V for the referenced groups) is the
+    full projection with the other blocks masked out; the output projection with the kept row blocks
+    of W_O is the full one applied to head outputs that are zero on pruned heads."""
+    g = np.random.default_rng(41)
+    B, T, D, Hq, Hk, d, k_h = 3, 9, 20, 6, 2, 4, 3
+    r = Hq // Hk
+    X = g.standard_normal((B, T, D))
+    WQ, WK, WV = g.standard_normal((D, Hq * d)), g.standard_normal((D, Hk * d)), g.standard_normal((D, Hk * d))
+    WO = g.standard_normal((Hq * d, D))
+    kept = np.array([[0, 1, 2], [1, 4, 5], [3, 4, 5]], dtype=np.int32)     # sample 0 and 2 use one group only
+    ids = np.array([0, 0, 0, 1, 1, 1, 2, 2, 2], dtype=np.int32)
+    masks = np.array([7, 5, 2], dtype=np.uint32)
+    Q, K, V = oracle.project_qkv(X, WQ, WK, WV, kept, ids, masks, Hq, Hk, d)
+    fullQ = (X @ WQ).reshape(B, T, Hq, d).transpose(0, 2, 1, 3)            # library matmul
+    fullK = (X @ WK).reshape(B, T, Hk, d).transpose(0, 2, 1, 3)
+    fullV = (X @ WV).reshape(B, T, Hk, d).transpose(0, 2, 1, 3)
+    for b in range(B):
+        present = ((int(masks[b]) >> ids) & 1).astype(bool)
+        hm = np.isin(np.arange(Hq), kept[b])
+        gm = np.isin(np.arange(Hk), kept[b] // r)
+        np.testing.assert_allclose(Q[b], fullQ[b] * hm[:, None, None] * present[None, :, None], atol=1e-12)
+        np.testing.assert_allclose(K[b], fullK[b] * gm[:, None, None] * present[None, :, None], atol=1e-12)
+        np.testing.assert_allclose(V[b], fullV[b] * gm[:, None, None] * present[None, :, None], atol=1e-12)
+        # sliced weight matrices: W_Q[:, blocks(H_keep)]
+        cols = np.concatenate([np.arange(h * d, (h + 1) * d) for h in kept[b]])
+        np.testing.assert_allclose(Q[b][kept[b]][:, present].transpose(1, 0, 2).reshape(-1, k_h * d),
+                                   X[b][present] @ WQ[:, cols], atol=1e-12)
+    assert np.all(K[0, 1] == 0) and np.all(K[2, 0] == 0)                    # unreferenced group removed
+    A = g.standard_normal((B, k_h, T, d))
+    out = oracle.project_out(A, WO, kept, ids, masks, Hq)
+    for b in range(B):
+        present = ((int(masks[b]) >> ids) & 1).astype(bool)
+        full_heads = np.zeros((T, Hq, d))
+        full_heads[:, kept[b]] = A[b].transpose(1, 0, 2)                    # pruned heads contribute zero
+        want = full_heads.reshape(T, Hq * d) @ WO
+        np.testing.assert_allclose(out[b], want * present[:, None], atol=1e-12)
+        rows = np.concatenate([np.arange(h * d, (h + 1) * d) for h in kept[b]])
+        np.testing.assert_allclose(out[b][present], A[b].transpose(1, 0, 2).reshape(T, -1)[present] @ WO[rows], atol=1e-12)
+
+
+def test_projected_layer_chains_into_attention_like_dense_layer_when_nothing_is_pruned():
+    # nothing pruned, group size 1, U = T_v: projections + SentryAttend + output projection equal a textbook
+    # multi-head self-attention layer computed with library routines
+    g = np.random.default_rng(42)
+    B, T, D, H, d = 2, 6, 12, 3, 4
+    X = g.standard_normal((B, T, D))
+    WQ, WK, WV = (g.standard_normal((D, H * d)) for _ in range(3))
+    WO = g.standard_normal((H * d, D))
+    kept = np.tile(np.arange(H, dtype=np.int32), (B, 1))
+    ids = np.zeros((T,), dtype=np.int32)
+    masks = np.ones((B,), dtype=np.uint32)
+    Q, K, V = oracle.project_qkv(X, WQ, WK, WV, kept, ids, masks, H, H, d)
+    A = oracle.attend(Q, K, V, kept, ids, masks, c=100, score_mode=1)       # U = T_v: every row is an Eq. 6 row
+    out = oracle.project_out(A, WO, kept, ids, masks, H)
+    qt, kt, vt = (torch.as_tensor((X @ W).reshape(B, T, H, d).transpose(0, 2, 1, 3)) for W in (WQ, WK, WV))
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt).numpy()
+    want = ref.transpose(0, 2, 1, 3).reshape(B, T, H * d) @ WO
+    np.testing.assert_allclose(out, want, rtol=1e-10, atol=1e-10)
