@@ -241,6 +241,41 @@ SENTRY_API int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* des
                           const int32_t* token_modality_ids, const uint32_t* masks, void* Y,
                           void* stream);
 
+/* ---------------------------------------------------------------------------
+ * Projections of the pruned layer (Sec. 4.6, "Head pruning with GQA
+ * consistency": of W_Q in R^{d_model x Hq d} only the column blocks of H_keep
+ * are kept, of W_K and W_V the blocks of K_keep = floor(H_keep / (Hq/Hk)); a KV
+ * group no kept head references is removed).  The paper never writes the
+ * output projection; its row blocks follow the same rule.
+ *
+ *   X [B,T,D]; WQ [D, Hq*d]; WK, WV [D, Hk*d]; WO [Hq*d, D]   (row-major)
+ *   kept_heads [B,k_h] i32 ascending; token_modality_ids [T]; masks [B]
+ * sentry_project_qkv writes, for every present token t of sample b,
+ *   Q[b,h,t,:] for the kept heads h and K[b,g,t,:], V[b,g,t,:] for the referenced
+ *   groups g, into Q [B,Hq,T,d] and K, V [B,Hk,T,d] -- the layouts
+ *   sentry_attend_fwd reads.  Nothing else is touched: slots of pruned heads,
+ *   unreferenced groups and absent tokens keep what they held (sentry_attend_fwd
+ *   never reads them).
+ * sentry_project_out takes A [B,k_h,T,d] (sentry_attend_fwd's output, heads in
+ *   kept-list order) and writes out [B,T,D] = sum_j A[b,j,t,:] . WO[h_j d:(h_j+1) d, :]
+ *   for present tokens, zero rows for absent ones.
+ * No bias, residual or normalisation.  fp32 accumulation, one rounding at the
+ * store.  Limits: Hk <= 32, k_h <= 64, D <= 8192.
+ */
+typedef struct sentry_proj_desc {
+    int B, T, D;       /* batch, tokens per sample, d_model */
+    int Hq, Hk, d;     /* query heads, KV heads, head dim */
+    int k_h;           /* kept heads per sample */
+    int dtype;         /* sentry_dtype of every tensor */
+} sentry_proj_desc;
+SENTRY_API int sentry_project_qkv(sentry_ctx* ctx, const sentry_proj_desc* desc, const void* X,
+                       const void* WQ, const void* WK, const void* WV, const int32_t* kept_heads,
+                       const int32_t* token_modality_ids, const uint32_t* masks, void* Q, void* K,
+                       void* V, void* stream);
+SENTRY_API int sentry_project_out(sentry_ctx* ctx, const sentry_proj_desc* desc, const void* A,
+                       const void* WO, const int32_t* kept_heads, const int32_t* token_modality_ids,
+                       const uint32_t* masks, void* out, void* stream);
+
 /* Which kernels run Eq. 6 for bf16 tensors whose K/V of one KV group fit in
  * shared memory (T up to ~1.4 k at d = 32).  Two hand-written forms exist:
  *   SENTRY_ATTEND_WARP_MMA  K/V staged by 16-byte async copies, Q K^T and P V

@@ -30,7 +30,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
            "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
-           "sentry_gate_eval", "sentry_gate_layer_counts"]
+           "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -40,6 +40,10 @@ class AttendDesc(ctypes.Structure):
 
 class FfnDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("B", "T", "D", "F", "k_c", "n_lists", "dtype")]
+
+
+class ProjDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("B", "T", "D", "Hq", "Hk", "d", "k_h", "dtype")]
 
 
 class SentryError(RuntimeError):
@@ -82,6 +86,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_set_option.argtypes = [vp, ci, ci]
     lib.sentry_gate_eval.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_gate_layer_counts.argtypes = [vp, vp, ci, ci, vp, ci, vp, vp]
+    lib.sentry_project_qkv.argtypes = [vp, ctypes.POINTER(ProjDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sentry_project_out.argtypes = [vp, ctypes.POINTER(ProjDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_ffn_packed_bytes.argtypes = [ctypes.POINTER(FfnDesc)]
     lib.sentry_ffn_packed_bytes.restype = ctypes.c_size_t
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -346,3 +352,34 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_gate_layer_counts")
         return counts
+
+    def project_qkv(self, X, WQ, WK, WV, kept_heads, token_modality_ids, masks, Hq: int, Hk: int, d: int,
+                    Q=None, K=None, V=None):
+        """sentry_project_qkv.  Returns Q [B,Hq,T,d], K, V [B,Hk,T,d]; fresh outputs start at zero."""
+        B, T, D = X.shape
+        desc = ProjDesc(B, T, D, int(Hq), int(Hk), int(d), kept_heads.shape[1], _dtype_code(X))
+        if Q is None:
+            Q = torch.zeros((B, Hq, T, d), dtype=X.dtype, device=X.device)
+        if K is None:
+            K = torch.zeros((B, Hk, T, d), dtype=X.dtype, device=X.device)
+        if V is None:
+            V = torch.zeros((B, Hk, T, d), dtype=X.dtype, device=X.device)
+        rc = self.lib.sentry_project_qkv(self.h, ctypes.byref(desc), _ptr(X), _ptr(WQ), _ptr(WK), _ptr(WV),
+                                         _ptr(kept_heads), _ptr(token_modality_ids), _ptr(masks), _ptr(Q), _ptr(K),
+                                         _ptr(V), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_project_qkv")
+        return Q, K, V
+
+    def project_out(self, A, WO, kept_heads, token_modality_ids, masks, Hq: int, out=None):
+        """sentry_project_out.  A [B,k_h,T,d] -> out [B,T,D]."""
+        B, k_h, T, d = A.shape
+        D = WO.shape[1]
+        desc = ProjDesc(B, T, D, int(Hq), 1, d, k_h, _dtype_code(A))
+        if out is None:
+            out = torch.empty((B, T, D), dtype=A.dtype, device=A.device)
+        rc = self.lib.sentry_project_out(self.h, ctypes.byref(desc), _ptr(A), _ptr(WO), _ptr(kept_heads),
+                                         _ptr(token_modality_ids), _ptr(masks), _ptr(out), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_project_out")
+        return out

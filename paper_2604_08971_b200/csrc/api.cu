@@ -96,7 +96,7 @@ int sentry_profile_slots(void) { return KS_COUNT; }
 
 const char* sentry_kernel_name(int slot) {
     static const char* names[KS_COUNT] = {"gate_rows", "gate_expand", "attend_score", "attend_select",
-                                          "attend_core", "ffn_prepare", "ffn_main", "gate_eval"};
+                                          "attend_core", "ffn_prepare", "ffn_main", "gate_eval", "project_qkv", "project_out"};
     return (slot >= 0 && slot < KS_COUNT) ? names[slot] : "?";
 }
 
@@ -318,6 +318,63 @@ int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, 
     a.status = ctx->d_status;
     SENTRY_ON_DEVICE(ctx->device);
     return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, nullptr, (cudaStream_t)stream);
+}
+
+static int check_proj_desc(const sentry_proj_desc* d) {
+    if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->B < 1 || d->T < 1 || d->D < 1 || d->Hq < 1 || d->Hk < 1 || d->d < 1 || d->k_h < 1) return SENTRY_ERR_BAD_SHAPE;
+    if (d->Hq % d->Hk != 0 || d->k_h > d->Hq) return SENTRY_ERR_BAD_SHAPE;
+    if (d->Hk > 32 || d->k_h > 64 || d->D > 8192 || d->k_h * d->d > 8192) return SENTRY_ERR_UNSUPPORTED;
+    if ((long long)d->B * d->T > 0x7fffffffLL) return SENTRY_ERR_UNSUPPORTED;
+    return SENTRY_OK;
+}
+
+int sentry_project_qkv(sentry_ctx* ctx, const sentry_proj_desc* desc, const void* X, const void* WQ,
+                       const void* WK, const void* WV, const int32_t* kept_heads,
+                       const int32_t* token_modality_ids, const uint32_t* masks, void* Q, void* K, void* V,
+                       void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_proj_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (X == nullptr || WQ == nullptr || WK == nullptr || WV == nullptr || kept_heads == nullptr ||
+        token_modality_ids == nullptr || masks == nullptr || Q == nullptr || K == nullptr || V == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(WQ, 16) || !aligned(WK, 16) || !aligned(WV, 16) || !aligned(Q, 16) ||
+        !aligned(K, 16) || !aligned(V, 16))
+        return SENTRY_ERR_INVALID_ARG;
+    ctx->last_launches = 0;
+    ProjArgs a = {};
+    a.d = *desc;
+    a.X = X; a.WQ = WQ; a.WK = WK; a.WV = WV;
+    a.kept_heads = kept_heads; a.ids = token_modality_ids; a.masks = masks;
+    a.Q = Q; a.K = K; a.V = V;
+    a.status = ctx->d_status;
+    SENTRY_ON_DEVICE(ctx->device);
+    return project_qkv_tc_supported(*desc) ? launch_project_qkv_tc(ctx, a, (cudaStream_t)stream)
+                                           : launch_project_qkv_generic(ctx, a, (cudaStream_t)stream);
+}
+
+int sentry_project_out(sentry_ctx* ctx, const sentry_proj_desc* desc, const void* A, const void* WO,
+                       const int32_t* kept_heads, const int32_t* token_modality_ids, const uint32_t* masks,
+                       void* out, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_proj_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (A == nullptr || WO == nullptr || kept_heads == nullptr || token_modality_ids == nullptr || masks == nullptr ||
+        out == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(A, 16) || !aligned(WO, 16) || !aligned(out, 16)) return SENTRY_ERR_INVALID_ARG;
+    ctx->last_launches = 0;
+    ProjArgs a = {};
+    a.d = *desc;
+    a.A = A; a.WO = WO;
+    a.kept_heads = kept_heads; a.ids = token_modality_ids; a.masks = masks;
+    a.out = out;
+    a.status = ctx->d_status;
+    SENTRY_ON_DEVICE(ctx->device);
+    return project_out_tc_supported(*desc) ? launch_project_out_tc(ctx, a, (cudaStream_t)stream)
+                                           : launch_project_out_generic(ctx, a, (cudaStream_t)stream);
 }
 
 size_t sentry_ffn_packed_bytes(const sentry_ffn_desc* desc) {

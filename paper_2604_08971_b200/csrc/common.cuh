@@ -13,7 +13,7 @@
 // Kernel slots for launch accounting and optional per-kernel timing.
 enum KernelSlot {
     KS_GATE_ROWS = 0, KS_GATE_EXPAND, KS_ATT_SCORE, KS_ATT_SELECT, KS_ATT_CORE,
-    KS_FFN_PREPARE, KS_FFN_MAIN, KS_GATE_EVAL, KS_COUNT
+    KS_FFN_PREPARE, KS_FFN_MAIN, KS_GATE_EVAL, KS_PROJ_QKV, KS_PROJ_OUT, KS_COUNT
 };
 
 struct ProfRec { cudaEvent_t start, stop; int slot; };
@@ -331,6 +331,23 @@ bool attend_tc_supported(const sentry_attend_desc& d);
 int launch_attend_tc(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_bf16_supported(const sentry_attend_desc& d);
 int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
+
+struct ProjArgs {
+    sentry_proj_desc d;
+    const void *X, *WQ, *WK, *WV;     // QKV projection
+    const void *A, *WO;               // output projection
+    const int32_t* kept_heads;
+    const int32_t* ids;
+    const uint32_t* masks;
+    void *Q, *K, *V, *out;
+    unsigned int* status;
+};
+int launch_project_qkv_generic(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
+int launch_project_out_generic(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
+bool project_qkv_tc_supported(const sentry_proj_desc& d);
+bool project_out_tc_supported(const sentry_proj_desc& d);
+int launch_project_qkv_tc(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
+int launch_project_out_tc(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
 
 struct FfnArgs {
     sentry_ffn_desc d;
