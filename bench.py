@@ -389,6 +389,64 @@ class Workbench:
         sn.profile_enable(False)
         return prof
 
+    def time_chained_layer(self, steps: int, replays: int):
+        """The full pruned encoder layer chained on one stream: gate selection for heads -> pruned Q/K/V
+        projections of X -> SentryAttend -> pruned output projection -> gate selection for channels ->
+        channel-compacted FFN on the projected rows (no residual or normalisation: the paper names none).
+        Returns (median ms per step, launches per step)."""
+        w, sn, dev = self.w, self.sn, self.dev
+        if w.D % 8 != 0:
+            return None
+        dt = synth.torch_dtype(w)
+        g = torch.Generator(device=dev).manual_seed(w.seed + 77)
+        mk = lambda *shape: (torch.randn(shape, generator=g, device=dev) * (4 * w.w_std)).to(dt)
+        WQ, WK, WV, WO = mk(w.D, w.Hq * w.d), mk(w.D, w.Hk * w.d), mk(w.D, w.Hk * w.d), mk(w.Hq * w.d, w.D)
+        s0 = self.sets[0]
+        Q, K, V = torch.zeros_like(s0.Q), torch.zeros_like(s0.K), torch.zeros_like(s0.V)
+        H = torch.empty_like(s0.X)
+        n = [0]
+
+        def chain(count=False):
+            c = 0
+            sn.gate_select(self.sh, self.masks, w.k_h, kept=s0.kept_h); c += sn.last_launch_count()
+            sn.project_qkv(s0.X, WQ, WK, WV, s0.kept_h, self.ids, self.masks, w.Hq, w.Hk, w.d, Q=Q, K=K, V=V)
+            c += sn.last_launch_count()
+            sn.attend_fwd(Q, K, V, s0.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s0.O)
+            c += sn.last_launch_count()
+            sn.project_out(s0.O, WO, s0.kept_h, self.ids, self.masks, w.Hq, out=H); c += sn.last_launch_count()
+            sn.gate_select(self.sc, self.subsets, w.k_c, kept=s0.kept_c); c += sn.last_launch_count()
+            sn.ffn_fwd(H, self.W1, self.W2, s0.kept_c, self.los, self.ids, self.masks, Y=s0.Y)
+            c += sn.last_launch_count()
+            if count:
+                n[0] = c
+
+        chain(count=True)
+        torch.cuda.synchronize()
+        graph = None
+        if self.graphs is not None:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    chain()
+            torch.cuda.current_stream().wait_stream(side)
+        run = graph.replay if graph is not None else chain
+        for _ in range(3):
+            run()
+        out = []
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(replays):
+            torch.cuda.synchronize()
+            ev0.record()
+            for _ in range(steps):
+                run()
+            ev1.record()
+            torch.cuda.synchronize()
+            out.append(ev0.elapsed_time(ev1) / steps)
+        assert sn.last_status() == 0
+        return float(np.median(out)), n[0]
+
     def work(self):
         kept_h_host = self.sets[0].kept_h.cpu().numpy()
         return work_model(self.w, self.inp.masks, kept_h_host, self.n_s_of)
@@ -471,6 +529,22 @@ def run_ours(args, w: synth.Workload):
     # ---- per-kernel pass (same steps, events around every kernel, no graph)
     n_prof = min(args.steps, 50)
     prof = wb.per_kernel(n_prof)
+
+    # ---- the whole layer chained X -> Q,K,V -> attention -> output projection -> FFN
+    chained = None
+    if world == 1 and not args.no_once:
+        res = wb.time_chained_layer(max(5, args.steps // 4), 3)
+        if res is not None:
+            c_ms, c_launches = res
+            r_ = w.Hq // w.Hk
+            proj_flops = sum(2.0 * w.D * w.d * synth.present_count(w, int(m)) *
+                             (2 * w.k_h + 2 * len(set(int(h) // r_ for h in kh)))
+                             for m, kh in zip(inp.masks, base.kept_h.cpu().numpy()))
+            chained = {"ms_per_step": c_ms, "tokens_per_s": wm["tokens"] / (c_ms * 1e-3), "gpu_launches_per_step": c_launches,
+                       "useful_tflops": (wm["att_flops"] + wm["ffn_flops"] + proj_flops) / (c_ms * 1e-3) / 1e12,
+                       "projection_flops": proj_flops,
+                       "what": "one stream: gate(heads), sentry_project_qkv, sentry_attend_fwd, sentry_project_out, "
+                               "gate(channels), sentry_ffn_fwd on the projected rows"}
 
     # ---- the same step with the pruned FFN weights materialised once (Section 4.6)
     once = None
@@ -629,7 +703,7 @@ def run_ours(args, w: synth.Workload):
                              "and timed with CUDA events" % (args.replays, args.steps)},
         "block_ms": blocks, "replays": args.replays,
         "useful_tflops": (wm["att_flops"] + wm["ffn_flops"]) * world * args.steps / (ms * 1e-3) / 1e12,
-        "materialised_once": once,
+        "materialised_once": once, "chained_layer": chained,
         "e2e": None if e2e_ms is None else {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": n_e2e,
                 "pipeline": "%d sample chunks; upload, kernels and download on three streams" % n_chunks},
