@@ -202,3 +202,17 @@ def project_out(A, WO, kept_heads, ids, masks, Hq: int):
     out = np.empty((B, T, D))
     _load().oracle_project_out(_p(A), _p(WO), B, T, D, Hq, d, _p(kh), k_h, _p(ii), _p(mk), _p(out))
     return out
+
+
+def moe_ffn(X, W1, W2, kept_channels, expert_ids, expert_weights) -> np.ndarray:
+    """Sparse-MoE block with expert-internal channel pruning (Section 4.6); routing given.
+    X [N,D]; W1 [E,D,F]; W2 [E,F,D]; kept_channels [E,k_c]; expert_ids, expert_weights [N,top_k]."""
+    X, W1, W2, wt = _f64(X), _f64(W1), _f64(W2), _f64(expert_weights)
+    kc, ex = _i32(kept_channels), _i32(expert_ids)
+    N, D = X.shape
+    E, _, F = W1.shape
+    assert W1.shape == (E, D, F) and W2.shape == (E, F, D) and kc.shape[0] == E and ex.shape == wt.shape
+    assert ex.min() >= 0 and ex.max() < E
+    Y = np.empty((N, D), dtype=np.float64)
+    _load().oracle_moe_ffn(_p(X), _p(W1), _p(W2), N, D, F, E, _p(kc), kc.shape[1], _p(ex), _p(wt), ex.shape[1], _p(Y))
+    return Y

@@ -22,6 +22,8 @@
  *   oracle_ffn             library matmul + erf, masked full FFN
  *   oracle_project_qkv/out library matmul on sliced and on masked full weight matrices;
  *                          unpruned chain == textbook multi-head attention layer
+ *   oracle_moe_ffn         library matmul per expert on sliced and on masked weights; one expert,
+ *                          top-1 == oracle_ffn; linear in the routing weights
  *   oracle_gate_eval       library matmul form of the perceptron, closed forms
  *                          (zero first layer, gamma = 0, one hidden unit by hand)
  * The paper's GFLOP figures and accuracies need undisclosed architectures and
@@ -398,4 +400,42 @@ void oracle_project_out(const double* A, const double* WO, int B, int T, int D, 
             }
         }
     }
+}
+
+/* ---- Sparse-MoE FFN pruning (Section 4.6): "the total number of experts and Top-k routing policy
+ * remain fixed.  Each expert contains its own internal FFN; ... W_{1,e}' = W_{1,e}[:, N_keep,e],
+ * W_{2,e}' = W_{2,e}[N_keep,e, :]".  The routing result (which experts a token goes to, with which
+ * weights) is an INPUT: pruning does not touch it.  For every token t
+ *   y_t = sum_j weight[t][j] * ( gelu(x_t . W1_e[:, N_e]) . W2_e[N_e, :] ),   e = expert[t][j],
+ * gelu as in oracle_ffn (exact erf; the paper names no activation).
+ * X [N,D]; W1 [E,D,F]; W2 [E,F,D]; kept [E,k_c]; expert [N,top_k]; weight [N,top_k]; Y [N,D]. */
+void oracle_moe_ffn(const double* X, const double* W1, const double* W2, int N, int D, int F, int E,
+                    const int32_t* kept, int k_c, const int32_t* expert, const double* weight, int top_k,
+                    double* Y) {
+#pragma omp parallel
+    {
+        double* h = (double*)malloc(sizeof(double) * (size_t)k_c);
+#pragma omp for schedule(dynamic, 16)
+        for (int t = 0; t < N; ++t) {
+            const double* x = X + (size_t)t * D;
+            double* y = Y + (size_t)t * D;
+            for (int e2 = 0; e2 < D; ++e2) y[e2] = 0.0;
+            for (int j = 0; j < top_k; ++j) {
+                const int e = expert[(size_t)t * top_k + j];
+                const double g = weight[(size_t)t * top_k + j];
+                const double* w1 = W1 + (size_t)e * D * F;
+                const double* w2 = W2 + (size_t)e * F * D;
+                const int32_t* Ne = kept + (size_t)e * k_c;
+                for (int n = 0; n < k_c; ++n) {
+                    double z = 0.0;
+                    for (int e2 = 0; e2 < D; ++e2) z += x[e2] * w1[(size_t)e2 * F + Ne[n]];
+                    h[n] = 0.5 * z * (1.0 + erf(z / sqrt(2.0)));
+                }
+                for (int n = 0; n < k_c; ++n)
+                    for (int e2 = 0; e2 < D; ++e2) y[e2] += g * h[n] * w2[(size_t)Ne[n] * D + e2];
+            }
+        }
+        free(h);
+    }
+    (void)E;
 }

@@ -486,3 +486,40 @@ def test_projected_layer_chains_into_attention_like_dense_layer_when_nothing_is_
     ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt).numpy()
     want = ref.transpose(0, 2, 1, 3).reshape(B, T, H * d) @ WO
     np.testing.assert_allclose(out, want, rtol=1e-10, atol=1e-10)
+
+
+# ------------------------------------------------------------------ Sparse-MoE FFN
+def test_moe_ffn_equals_library_form_and_reduces_to_plain_ffn():
+    g = np.random.default_rng(51)
+    N, D, F, E, k, k_c = 17, 12, 40, 4, 2, 15
+    X = g.standard_normal((N, D))
+    W1, W2 = g.standard_normal((E, D, F)) * 0.3, g.standard_normal((E, F, D)) * 0.3
+    kept = np.stack([np.sort(g.choice(F, k_c, replace=False)) for _ in range(E)]).astype(np.int32)
+    ex = np.stack([g.choice(E, k, replace=False) for _ in range(N)]).astype(np.int32)
+    wt = g.random((N, k))
+    got = oracle.moe_ffn(X, W1, W2, kept, ex, wt)
+    # library form: per expert, sliced weight matrices (W1_e[:, N_e], W2_e[N_e, :]) and numpy matmul
+    want = np.zeros((N, D))
+    for e in range(E):
+        y_e = _gelu(X @ W1[e][:, kept[e]]) @ W2[e][kept[e], :]
+        for j in range(k):
+            sel = ex[:, j] == e
+            want[sel] += wt[sel, j][:, None] * y_e[sel]
+    np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-12)
+    # masked full expert FFN: a pruned channel contributes exactly zero
+    want2 = np.zeros((N, D))
+    for e in range(E):
+        m = np.zeros(F); m[kept[e]] = 1.0
+        y_e = (_gelu(X @ W1[e]) * m) @ W2[e]
+        for j in range(k):
+            sel = ex[:, j] == e
+            want2[sel] += wt[sel, j][:, None] * y_e[sel]
+    np.testing.assert_allclose(got, want2, rtol=1e-11, atol=1e-12)
+    # one expert, top-1, weight 1: the plain channel-compacted FFN of Section 4.6
+    one = oracle.moe_ffn(X, W1[:1], W2[:1], kept[:1], np.zeros((N, 1), dtype=np.int32), np.ones((N, 1)))
+    np.testing.assert_allclose(one, oracle.ffn(X[None], W1[0], W2[0], kept[:1])[0], rtol=1e-12, atol=1e-13)
+    # routing weights enter linearly; a zero weight removes the expert
+    wt0 = wt.copy(); wt0[:, 1] = 0.0
+    a = oracle.moe_ffn(X, W1, W2, kept, ex, wt0)
+    b = oracle.moe_ffn(X, W1, W2, kept, ex[:, :1], wt[:, :1])
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
