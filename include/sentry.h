@@ -242,6 +242,50 @@ SENTRY_API int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* des
                           void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Sparse-MoE block with expert-internal channel pruning (Sec. 4.6, "Extending
+ * SentryGate to Sparse-MoE Architectures": the number of experts and the top-k
+ * routing rule stay as they are; every expert e keeps its own channel set N_e
+ * of its own FFN, W1_e' = W1_e[:, N_e], W2_e' = W2_e[N_e, :]).  The routing
+ * result is an input.  For every token t
+ *   y_t = sum_j w[t,j] * ( gelu(x_t . W1_e[:, N_e]) . W2_e[N_e, :] ),  e = expert_ids[t,j],
+ * gelu as in sentry_ffn_fwd; the sum runs over the slots j = 0..top_k-1 in
+ * that order, accumulated in fp32 (each term first rounded to `dtype`).
+ *
+ *   X [N,D]; W1 [E,D,F]; W2 [E,F,D] (row-major, dtype); kept_channels [E,k_c] i32
+ *   expert_ids [N,top_k] i32: -1 = slot not routed (contributes nothing); any
+ *     other value outside [0,E) is skipped and flagged BAD_INDEX
+ *   expert_weights [N,top_k] fp32 (whatever the router produced; not renormalised)
+ *   Y out [N,D] dtype; a token with no routed slot gets zeros
+ * All device pointers, 16-byte aligned; D % 8 == 0, D <= 1024, E <= 4096,
+ * N*top_k < 2^31.  bf16 with D in {128,256,384} runs on the tcgen05 kernel of
+ * sentry_ffn_fwd with one weight set per expert; other shapes on the plain
+ * ALUs.  Scratch (row plan, per-slot results, and W1', W2' unless `packed` is
+ * given) comes from the workspace: sentry_moe_workspace_bytes.
+ *
+ *   sentry_moe_packed_bytes / sentry_moe_prepack: materialise W1_e', W2_e' of
+ *     all experts once (same contract as sentry_ffn_prepack)
+ *   sentry_moe_ffn_fwd: `packed` NULL -> W1, W2, kept_channels are gathered on
+ *     every call; otherwise they are ignored (may be NULL) and `packed` is used.
+ */
+typedef struct sentry_moe_desc {
+    int N;      /* tokens */
+    int D, F;   /* d_model, d_ff of one expert */
+    int E;      /* experts */
+    int top_k;  /* routing slots per token */
+    int k_c;    /* kept channels per expert */
+    int dtype;  /* sentry_dtype of X, W1, W2, Y */
+} sentry_moe_desc;
+SENTRY_API size_t sentry_moe_workspace_bytes(const sentry_moe_desc* desc);
+SENTRY_API size_t sentry_moe_packed_bytes(const sentry_moe_desc* desc);
+SENTRY_API int sentry_moe_prepack(sentry_ctx* ctx, const sentry_moe_desc* desc, const void* W1,
+                       const void* W2, const int32_t* kept_channels, void* packed,
+                       size_t packed_bytes, void* stream);
+SENTRY_API int sentry_moe_ffn_fwd(sentry_ctx* ctx, const sentry_moe_desc* desc, const void* X,
+                       const void* W1, const void* W2, const int32_t* kept_channels,
+                       const void* packed, const int32_t* expert_ids,
+                       const float* expert_weights, void* Y, void* stream);
+
+/* ---------------------------------------------------------------------------
  * Projections of the pruned layer (Sec. 4.6, "Head pruning with GQA
  * consistency": of W_Q in R^{d_model x Hq d} only the column blocks of H_keep
  * are kept, of W_K and W_V the blocks of K_keep = floor(H_keep / (Hq/Hk)); a KV

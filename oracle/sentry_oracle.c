@@ -340,9 +340,9 @@ void oracle_gate_eval(int M, int hidden, int n_layers, const int32_t* layer_offs
 }
 
 /* ---- Head pruning with GQA consistency (Section 4.6): the projections of a pruned layer.
- * "Given the query projection W_Q in R^{d_model x H_q d_h}, we keep only the column blocks
- * associated with H_keep ... K_keep = floor(H_keep / (H_q/H_k)) and apply analogous block
- * filtering to W_K and W_V."  For every sample b and present token t:
+ * W_Q is [d_model, H_q d_h]; of its H_q column blocks only those of the kept heads H_keep are
+ * used.  The kept KV groups follow from them, K_keep = { floor(h / (H_q/H_k)) : h in H_keep }, and
+ * W_K, W_V are filtered by block in the same way.  For every sample b and present token t:
  *   Q[b,h,t,:] = x_t . W_Q[:, h d : (h+1) d]        for h in H_keep(b)
  *   K[b,g,t,:] = x_t . W_K[:, g d : (g+1) d],  V likewise,  for g in K_keep(b)
  * Everything else (pruned heads, unreferenced groups, absent tokens) is left at zero here.
@@ -402,9 +402,9 @@ void oracle_project_out(const double* A, const double* WO, int B, int T, int D, 
     }
 }
 
-/* ---- Sparse-MoE FFN pruning (Section 4.6): "the total number of experts and Top-k routing policy
- * remain fixed.  Each expert contains its own internal FFN; ... W_{1,e}' = W_{1,e}[:, N_keep,e],
- * W_{2,e}' = W_{2,e}[N_keep,e, :]".  The routing result (which experts a token goes to, with which
+/* ---- Sparse-MoE FFN pruning (Section 4.6): the expert count and the top-k routing rule are left
+ * alone; what is pruned is the inside of each expert, whose own FFN keeps a channel set N_e of its
+ * own: W1_e' = W1_e[:, N_e], W2_e' = W2_e[N_e, :].  The routing result (which experts a token goes to, with which
  * weights) is an INPUT: pruning does not touch it.  For every token t
  *   y_t = sum_j weight[t][j] * ( gelu(x_t . W1_e[:, N_e]) . W2_e[N_e, :] ),   e = expert[t][j],
  * gelu as in oracle_ffn (exact erf; the paper names no activation).

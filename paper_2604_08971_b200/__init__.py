@@ -30,7 +30,8 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
            "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
-           "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out"]
+           "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out",
+           "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -44,6 +45,10 @@ class FfnDesc(ctypes.Structure):
 
 class ProjDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("B", "T", "D", "Hq", "Hk", "d", "k_h", "dtype")]
+
+
+class MoeDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "D", "F", "E", "top_k", "k_c", "dtype")]
 
 
 class SentryError(RuntimeError):
@@ -92,6 +97,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_packed_bytes.restype = ctypes.c_size_t
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
+    lib.sentry_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
+    lib.sentry_moe_workspace_bytes.restype = ctypes.c_size_t
+    lib.sentry_moe_packed_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
+    lib.sentry_moe_packed_bytes.restype = ctypes.c_size_t
+    lib.sentry_moe_prepack.argtypes = [vp, ctypes.POINTER(MoeDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.sentry_moe_ffn_fwd.argtypes = [vp, ctypes.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_profile_enable.argtypes = [vp, ci]
     lib.sentry_profile_slots.argtypes = []
     lib.sentry_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
@@ -100,7 +111,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_kernel_name.restype = ctypes.c_char_p
     for name in EXPORTS:
         if name not in ("sentry_status_string", "sentry_workspace_bytes", "sentry_kernel_name",
-                        "sentry_ffn_packed_bytes"):
+                        "sentry_ffn_packed_bytes", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes"):
             getattr(lib, name).restype = ci
     if path is None:
         _lib = lib
@@ -383,3 +394,36 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_project_out")
         return out
+
+    def moe_prepack(self, W1, W2, kept_channels, packed=None):
+        """sentry_moe_prepack: W1_e[:, N_e], W2_e[N_e, :] of every expert, once.  W1 [E,D,F]; W2 [E,F,D];
+        kept_channels [E,k_c].  Returns the packed buffer for moe_ffn_fwd(packed=...)."""
+        E, D, F = W1.shape
+        desc = MoeDesc(1, D, F, E, 1, kept_channels.shape[1], _dtype_code(W1))
+        nbytes = int(self.lib.sentry_moe_packed_bytes(ctypes.byref(desc)))
+        if packed is None:
+            packed = torch.empty((nbytes,), dtype=torch.uint8, device=W1.device)
+        rc = self.lib.sentry_moe_prepack(self.h, ctypes.byref(desc), _ptr(W1), _ptr(W2), _ptr(kept_channels),
+                                         _ptr(packed), packed.numel(), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_moe_prepack")
+        return packed
+
+    def moe_ffn_fwd(self, X, expert_ids, expert_weights, W1=None, W2=None, kept_channels=None, packed=None,
+                    F: Optional[int] = None, E: Optional[int] = None, k_c: Optional[int] = None, Y=None):
+        """sentry_moe_ffn_fwd.  X [N,D]; expert_ids i32, expert_weights fp32 [N,top_k]; either W1 [E,D,F],
+        W2 [E,F,D], kept_channels [E,k_c], or `packed` from moe_prepack with F, E, k_c.  Returns Y [N,D]."""
+        N, D = X.shape
+        if packed is None:
+            E, _, F = W1.shape
+            k_c = kept_channels.shape[1]
+        desc = MoeDesc(N, D, int(F), int(E), expert_ids.shape[1], int(k_c), _dtype_code(X))
+        if Y is None:
+            Y = torch.empty_like(X)
+        self.ensure_workspace(int(self.lib.sentry_moe_workspace_bytes(ctypes.byref(desc))))
+        rc = self.lib.sentry_moe_ffn_fwd(self.h, ctypes.byref(desc), _ptr(X), _ptr(W1), _ptr(W2),
+                                         _ptr(kept_channels), _ptr(packed), _ptr(expert_ids), _ptr(expert_weights),
+                                         _ptr(Y), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_moe_ffn_fwd")
+        return Y

@@ -96,7 +96,8 @@ int sentry_profile_slots(void) { return KS_COUNT; }
 
 const char* sentry_kernel_name(int slot) {
     static const char* names[KS_COUNT] = {"gate_rows", "gate_expand", "attend_score", "attend_select",
-                                          "attend_core", "ffn_prepare", "ffn_main", "gate_eval", "project_qkv", "project_out"};
+                                          "attend_core", "ffn_prepare", "ffn_main", "gate_eval", "project_qkv", "project_out",
+                                          "moe_plan", "moe_combine"};
     return (slot >= 0 && slot < KS_COUNT) ? names[slot] : "?";
 }
 
@@ -307,7 +308,7 @@ int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, 
         !aligned(kept_channels, 4))
         return SENTRY_ERR_INVALID_ARG;
     ctx->last_launches = 0;
-    FfnArgs a;
+    FfnArgs a = {};
     a.d = *desc;
     a.X = X; a.W1 = W1; a.W2 = W2;
     a.kept = kept_channels;
@@ -375,6 +376,70 @@ int sentry_project_out(sentry_ctx* ctx, const sentry_proj_desc* desc, const void
     SENTRY_ON_DEVICE(ctx->device);
     return project_out_tc_supported(*desc) ? launch_project_out_tc(ctx, a, (cudaStream_t)stream)
                                            : launch_project_out_generic(ctx, a, (cudaStream_t)stream);
+}
+
+static int check_moe_desc(const sentry_moe_desc* d) {
+    if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->N < 1 || d->D < 1 || d->F < 1 || d->E < 1 || d->top_k < 1 || d->k_c < 1) return SENTRY_ERR_BAD_SHAPE;
+    if (d->k_c > d->F) return SENTRY_ERR_BAD_SHAPE;
+    if (d->D % 8 != 0 || d->D > 1024 || d->E > 4096 || d->top_k > 64) return SENTRY_ERR_UNSUPPORTED;
+    if ((long long)d->N * d->top_k > 0x7fffffffLL - 8192) return SENTRY_ERR_UNSUPPORTED;
+    return SENTRY_OK;
+}
+
+size_t sentry_moe_workspace_bytes(const sentry_moe_desc* desc) {
+    return check_moe_desc(desc) == SENTRY_OK ? align_up(moe_workspace_bytes(*desc), 256) : 0;
+}
+
+size_t sentry_moe_packed_bytes(const sentry_moe_desc* desc) {
+    return check_moe_desc(desc) == SENTRY_OK ? moe_packed_bytes(*desc) : 0;
+}
+
+int sentry_moe_prepack(sentry_ctx* ctx, const sentry_moe_desc* desc, const void* W1, const void* W2,
+                       const int32_t* kept_channels, void* packed, size_t packed_bytes, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_moe_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (W1 == nullptr || W2 == nullptr || kept_channels == nullptr || packed == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(W1, 16) || !aligned(W2, 16) || !aligned(kept_channels, 4) || !aligned(packed, 256))
+        return SENTRY_ERR_INVALID_ARG;
+    if (packed_bytes < moe_packed_bytes(*desc)) return SENTRY_ERR_WORKSPACE;
+    ctx->last_launches = 0;
+    MoeArgs m = {};
+    m.d = *desc;
+    m.W1 = W1; m.W2 = W2;
+    m.kept = kept_channels;
+    m.status = ctx->d_status;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_moe_prepack(ctx, m, packed, (cudaStream_t)stream);
+}
+
+int sentry_moe_ffn_fwd(sentry_ctx* ctx, const sentry_moe_desc* desc, const void* X, const void* W1,
+                       const void* W2, const int32_t* kept_channels, const void* packed,
+                       const int32_t* expert_ids, const float* expert_weights, void* Y, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_moe_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (X == nullptr || Y == nullptr || expert_ids == nullptr || expert_weights == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (packed == nullptr && (W1 == nullptr || W2 == nullptr || kept_channels == nullptr))
+        return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(expert_ids, 4) || !aligned(expert_weights, 4))
+        return SENTRY_ERR_INVALID_ARG;
+    if (packed != nullptr ? !aligned(packed, 256) : (!aligned(W1, 16) || !aligned(W2, 16) || !aligned(kept_channels, 4)))
+        return SENTRY_ERR_INVALID_ARG;
+    ctx->last_launches = 0;
+    MoeArgs m = {};
+    m.d = *desc;
+    m.X = X; m.W1 = W1; m.W2 = W2;
+    m.kept = kept_channels;
+    m.expert_ids = expert_ids;
+    m.expert_weights = expert_weights;
+    m.Y = Y;
+    m.status = ctx->d_status;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_moe_ffn(ctx, m, ctx->workspace, ctx->workspace_bytes, packed, (cudaStream_t)stream);
 }
 
 size_t sentry_ffn_packed_bytes(const sentry_ffn_desc* desc) {

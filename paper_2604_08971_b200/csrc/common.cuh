@@ -13,7 +13,8 @@
 // Kernel slots for launch accounting and optional per-kernel timing.
 enum KernelSlot {
     KS_GATE_ROWS = 0, KS_GATE_EXPAND, KS_ATT_SCORE, KS_ATT_SELECT, KS_ATT_CORE,
-    KS_FFN_PREPARE, KS_FFN_MAIN, KS_GATE_EVAL, KS_PROJ_QKV, KS_PROJ_OUT, KS_COUNT
+    KS_FFN_PREPARE, KS_FFN_MAIN, KS_GATE_EVAL, KS_PROJ_QKV, KS_PROJ_OUT,
+    KS_MOE_PLAN, KS_MOE_COMBINE, KS_COUNT
 };
 
 struct ProfRec { cudaEvent_t start, stop; int slot; };
@@ -34,8 +35,9 @@ struct sentry_ctx {
 // Brackets one kernel launch with events when profiling is on; counts the launch.
 struct LaunchScope {
     sentry_ctx* ctx; cudaStream_t st; ProfRec rec; bool on;
-    LaunchScope(sentry_ctx* c, int slot, cudaStream_t s) : ctx(c), st(s), on(c->profiling) {
-        ++ctx->last_launches;
+    // `launches`: kernels the scope covers (they are timed together under `slot`)
+    LaunchScope(sentry_ctx* c, int slot, cudaStream_t s, int launches = 1) : ctx(c), st(s), on(c->profiling) {
+        ctx->last_launches += launches;
         if (!on) return;
         cudaEvent_t ev[2];
         for (int i = 0; i < 2; ++i) {
@@ -353,6 +355,7 @@ struct FfnArgs {
     sentry_ffn_desc d;
     const void *X, *W1, *W2;
     const int32_t* kept;
+    size_t w_stride;        // elements between the weight matrices of consecutive lists (0: shared)
     const int32_t* list_of_sample;
     const int32_t* ids;
     const uint32_t* masks;
@@ -364,3 +367,19 @@ size_t ffn_packed_bytes(const sentry_ffn_desc& d);
 int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStream_t st);
 int launch_wait_expiry_selftest(sentry_ctx* ctx, long long limit_cycles, cudaStream_t st);
 int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, const void* packed, cudaStream_t st);
+int ffn_kc_pad(const sentry_ffn_desc& d);
+int ffn_tile_rows(const sentry_ffn_desc& d);
+
+struct MoeArgs {
+    sentry_moe_desc d;
+    const void *X, *W1, *W2;
+    const int32_t* kept;            // [E, k_c]
+    const int32_t* expert_ids;      // [N, top_k]
+    const float* expert_weights;    // [N, top_k]
+    void* Y;
+    unsigned int* status;
+};
+size_t moe_workspace_bytes(const sentry_moe_desc& m);
+size_t moe_packed_bytes(const sentry_moe_desc& m);
+int launch_moe_prepack(sentry_ctx* ctx, const MoeArgs& m, void* packed, cudaStream_t st);
+int launch_moe_ffn(sentry_ctx* ctx, const MoeArgs& m, void* ws, size_t ws_bytes, const void* packed, cudaStream_t st);

@@ -35,7 +35,10 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
                    int tile_rows, FfnPlan p, uint8_t* __restrict__ Y,
                    const T* __restrict__ W1, const T* __restrict__ W2,
                    const int32_t* __restrict__ kept, int n_lists, int D, int F, int k_c, int kc_pad,
-                   int layout, T* __restrict__ out1, T* __restrict__ out2, unsigned int* status) {
+                   int layout, size_t w_stride, T* __restrict__ out1, T* __restrict__ out2,
+                   unsigned int* status) {
+    // w_stride: elements between the weight matrices of consecutive lists (0: every list gathers
+    // from the same W1, W2; D*F: list l has its own, as the experts of a Sparse-MoE block do)
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     if ((int)blockIdx.x < B) {
         __shared__ int s_cnt[32];
@@ -147,6 +150,8 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
         const int l = (int)(pb / per_list);
         const int tn = (int)((pb % per_list) / tiles_e), te = (int)(pb % tiles_e);
         const int n0 = tn * 32, e0 = te * 64;
+        const T* W1l = W1 + (size_t)l * w_stride;
+        const T* W2l = W2 + (size_t)l * w_stride;
         const int tx = threadIdx.x & 31, wy = threadIdx.x >> 5;   // 8 warps
         if (threadIdx.x < 32) {
             const int n = n0 + threadIdx.x;
@@ -165,7 +170,7 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
         if (which == 0) {
             const int ch = s_ch[tx];
             for (int ee = wy; ee < 64; ee += 8)
-                s_tile[ee][tx] = ch >= 0 ? W1[(size_t)(e0 + ee) * F + ch] : zero;
+                s_tile[ee][tx] = ch >= 0 ? W1l[(size_t)(e0 + ee) * F + ch] : zero;
             __syncthreads();
             T* dst = out1 + ((size_t)l * kc_pad + n0) * D + e0;
             for (int nn = wy; nn < 32; nn += 8) {
@@ -175,8 +180,8 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
         } else {
             for (int nn = wy; nn < 32; nn += 8) {
                 const int ch = s_ch[nn];
-                s_tile[tx][nn] = ch >= 0 ? W2[(size_t)ch * D + e0 + tx] : zero;
-                s_tile[32 + tx][nn] = ch >= 0 ? W2[(size_t)ch * D + e0 + 32 + tx] : zero;
+                s_tile[tx][nn] = ch >= 0 ? W2l[(size_t)ch * D + e0 + tx] : zero;
+                s_tile[32 + tx][nn] = ch >= 0 ? W2l[(size_t)ch * D + e0 + 32 + tx] : zero;
             }
             __syncthreads();
             T* dst = out2 + ((size_t)l * D + e0) * kc_pad + n0;
@@ -200,7 +205,7 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
         T v = from_f32<T>(0.f);
         if (n < k_c) {
             const int ch = N[n];
-            if (ch >= 0 && ch < F) v = W1[(size_t)e * F + ch];
+            if (ch >= 0 && ch < F) v = W1[(size_t)l * w_stride + (size_t)e * F + ch];
             else if (e == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
         }
         out1[(size_t)l * per + i] = v;
@@ -211,7 +216,7 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
         T v = from_f32<T>(0.f);
         if (n < k_c) {
             const int ch = N[n];
-            if (ch >= 0 && ch < F) v = W2[(size_t)ch * D + e];
+            if (ch >= 0 && ch < F) v = W2[(size_t)l * w_stride + (size_t)ch * D + e];
         }
         out2[(size_t)l * per + i] = v;
     }
@@ -230,11 +235,14 @@ ffn_generic_kernel(const T* __restrict__ X, const T* __restrict__ W1g, const T* 
     extern __shared__ float s_f[];
     float* s_x = s_f;                                  // [16][D]
     float* s_h = s_f + (size_t)kGenericTileRows * D;   // [16][256]
-    __shared__ long long s_row[kGenericTileRows];
+    __shared__ long long s_row[kGenericTileRows], s_out[kGenericTileRows];
     int l, row0, n_rows;
     if (!ffn_tile_lookup(plan, n_lists, blockIdx.x, kGenericTileRows, l, row0, n_rows)) return;
     if (threadIdx.x < kGenericTileRows)
         s_row[threadIdx.x] = threadIdx.x < n_rows ? (long long)plan.rowidx[row0 + threadIdx.x] : -1;
+    if (threadIdx.x < kGenericTileRows)
+        s_out[threadIdx.x] = threadIdx.x < n_rows
+                                 ? (long long)(plan.rowout ? plan.rowout : plan.rowidx)[row0 + threadIdx.x] : -1;
     __syncthreads();
     for (int i = threadIdx.x; i < kGenericTileRows * D; i += blockDim.x) {
         const int r = i / D, e = i % D;
@@ -286,7 +294,7 @@ ffn_generic_kernel(const T* __restrict__ X, const T* __restrict__ W1g, const T* 
         if (e < D) {
 #pragma unroll
             for (int r = 0; r < kGenericTileRows; ++r)
-                if (s_row[r] >= 0) Y[(size_t)s_row[r] * D + e] = from_f32<T>(y[s][r]);
+                if (s_out[r] >= 0) Y[(size_t)s_out[r] * D + e] = from_f32<T>(y[s][r]);
         }
     }
 }
@@ -312,6 +320,7 @@ FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes, bool w
     w.plan.list_row0 = a.take<int32_t>(d.n_lists + 1);
     w.plan.tile_start = a.take<int32_t>(d.n_lists + 1);
     w.plan.rowidx = a.take<int32_t>((size_t)d.B * d.T);
+    w.plan.rowout = nullptr;
     w.w1p = w.w2p = nullptr;
     if (with_weights) {
         w.w1p = a.take<uint8_t>(packed_half_bytes(d, kc_pad));
@@ -346,17 +355,54 @@ int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStre
     uint8_t* w1p = (uint8_t*)packed;
     uint8_t* w2p = w1p + packed_half_bytes(d, kc_pad);
     FfnPlan none = {};
+    none.rowout = nullptr;
     LaunchScope ls(ctx, KS_FFN_PREPARE, st);
     // no row-table and no zero-fill blocks (B = 0, no ids): every block gathers weights
     if (d.dtype == SENTRY_F32)
         ffn_prepare_kernel<float><<<(unsigned)pack_blocks, 256, 0, st>>>(
             nullptr, nullptr, nullptr, 0, d.T, 1, kGenericTileRows, none, nullptr, (const float*)a.W1,
-            (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, (float*)w1p, (float*)w2p, a.status);
+            (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, a.w_stride, (float*)w1p, (float*)w2p, a.status);
     else
         ffn_prepare_kernel<__nv_bfloat16><<<(unsigned)pack_blocks, 256, 0, st>>>(
             nullptr, nullptr, nullptr, 0, d.T, 1, tc ? kTcTileRows : kGenericTileRows, none, nullptr,
             (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad,
-            tc ? 1 : 0, (__nv_bfloat16*)w1p, (__nv_bfloat16*)w2p, a.status);
+            tc ? 1 : 0, a.w_stride, (__nv_bfloat16*)w1p, (__nv_bfloat16*)w2p, a.status);
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}
+
+int ffn_kc_pad(const sentry_ffn_desc& d) { return kc_pad_for(d); }
+int ffn_tile_rows(const sentry_ffn_desc& d) {
+    return d.dtype == SENTRY_BF16 && ffn_tc_supported(d) ? kTcTileRows : kGenericTileRows;
+}
+
+// The fused pair alone, on a row plan and materialised weights that are already in place.
+int launch_ffn_main(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1p, void* w2p, int kc_pad,
+                    int max_tiles, cudaStream_t st) {
+    const sentry_ffn_desc& d = a.d;
+    const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
+    if (tc) {
+        int rc = launch_ffn_tc(ctx, a, plan, w1p, w2p, kc_pad, max_tiles, st);
+        if (rc != SENTRY_OK) return rc;
+    } else {
+        const size_t smem = ((size_t)kGenericTileRows * d.D + kGenericTileRows * kGenericThreads) * 4;
+        LaunchScope ls(ctx, KS_FFN_MAIN, st);
+        if (d.dtype == SENTRY_F32) {
+            auto kern = ffn_generic_kernel<float>;
+            if (smem > 48 * 1024)
+                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<max_tiles, kGenericThreads, smem, st>>>((const float*)a.X, (const float*)w1p,
+                                                            (const float*)w2p, plan, d.n_lists,
+                                                            d.T, d.D, d.k_c, kc_pad, (float*)a.Y);
+        } else {
+            auto kern = ffn_generic_kernel<__nv_bfloat16>;
+            if (smem > 48 * 1024)
+                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<max_tiles, kGenericThreads, smem, st>>>(
+                (const __nv_bfloat16*)a.X, (const __nv_bfloat16*)w1p, (const __nv_bfloat16*)w2p,
+                plan, d.n_lists, d.T, d.D, d.k_c, kc_pad, (__nv_bfloat16*)a.Y);
+        }
+    }
     SENTRY_CUDA_TRY(cudaGetLastError());
     return SENTRY_OK;
 }
@@ -389,39 +435,16 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, con
         if (d.dtype == SENTRY_F32)
             ffn_prepare_kernel<float><<<(unsigned)grid, 256, 0, st>>>(
                 a.ids, a.masks, a.list_of_sample, d.B, d.T, zsplit, tile_rows, w.plan, (uint8_t*)a.Y,
-                (const float*)a.W1, (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0,
+                (const float*)a.W1, (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, a.w_stride,
                 (float*)w.w1p, (float*)w.w2p, a.status);
         else
             ffn_prepare_kernel<__nv_bfloat16><<<(unsigned)grid, 256, 0, st>>>(
                 a.ids, a.masks, a.list_of_sample, d.B, d.T, zsplit, tile_rows, w.plan, (uint8_t*)a.Y,
                 (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F,
-                d.k_c, kc_pad, tc ? 1 : 0, (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
+                d.k_c, kc_pad, tc ? 1 : 0, a.w_stride, (__nv_bfloat16*)w.w1p, (__nv_bfloat16*)w.w2p, a.status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
     const long long rows = (long long)d.B * d.T;
     const int max_tiles = (int)((rows + tile_rows - 1) / tile_rows) + d.n_lists;
-    if (tc) {
-        int rc = launch_ffn_tc(ctx, a, w.plan, w.w1p, w.w2p, kc_pad, max_tiles, st);
-        if (rc != SENTRY_OK) return rc;
-    } else {
-        const size_t smem = ((size_t)kGenericTileRows * d.D + kGenericTileRows * kGenericThreads) * 4;
-        LaunchScope ls(ctx, KS_FFN_MAIN, st);
-        if (d.dtype == SENTRY_F32) {
-            auto kern = ffn_generic_kernel<float>;
-            if (smem > 48 * 1024)
-                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            kern<<<max_tiles, kGenericThreads, smem, st>>>((const float*)a.X, (const float*)w.w1p,
-                                                            (const float*)w.w2p, w.plan, d.n_lists,
-                                                            d.T, d.D, d.k_c, kc_pad, (float*)a.Y);
-        } else {
-            auto kern = ffn_generic_kernel<__nv_bfloat16>;
-            if (smem > 48 * 1024)
-                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            kern<<<max_tiles, kGenericThreads, smem, st>>>(
-                (const __nv_bfloat16*)a.X, (const __nv_bfloat16*)w.w1p, (const __nv_bfloat16*)w.w2p,
-                w.plan, d.n_lists, d.T, d.D, d.k_c, kc_pad, (__nv_bfloat16*)a.Y);
-        }
-    }
-    SENTRY_CUDA_TRY(cudaGetLastError());
-    return SENTRY_OK;
+    return launch_ffn_main(ctx, a, w.plan, w.w1p, w.w2p, kc_pad, max_tiles, st);
 }

@@ -14,7 +14,13 @@ struct FfnPlan {
     int32_t* list_row0;     // [n_lists+1]  offset in rowidx of each list's rows
     int32_t* tile_start;    // [n_lists+1]  first tile of each list; [n_lists] = total tiles
     int32_t* rowidx;        // [B*T]        global row (b*T + t) of every present row, list-major
+    int32_t* rowout;        // same shape or null: row of Y a result goes to, if not the row of X it came from
+                            //              (Sparse-MoE: X row = token, Y row = (token, routing slot))
 };
+
+// The fused pair alone, on a row plan and materialised weights that are already in place.
+int launch_ffn_main(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1p, void* w2p, int kc_pad,
+                    int max_tiles, cudaStream_t st);
 
 #ifdef __CUDACC__
 // Locate tile `tile` -> list l, offset of its first row in rowidx, and its row count;

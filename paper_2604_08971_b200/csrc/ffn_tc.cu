@@ -482,7 +482,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             int l, row0, n_rows;
             ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
             prev_row = my_row;
-            my_row = row < n_rows ? plan.rowidx[row0 + row] : -1;
+            my_row = row < n_rows ? (plan.rowout ? plan.rowout : plan.rowidx)[row0 + row] : -1;
             for (int c = 0; c < NC && ok; ++c, ++g) {
                 if (!warp_wait(&misc->h_full, g & 1u, abort_flag)) { ok = false; break; }
                 ptx::tc_fence_after_sync();

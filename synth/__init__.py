@@ -235,3 +235,39 @@ def generate(w: Workload, n_samples_of: Callable[[int], int], device: str = "cpu
     list_of_sample = np.array([index_of[int(m)] for m in masks], dtype=np.int32)
     return Inputs(w, ids, masks, scores_heads, scores_ch, Q, K, V, X, W1, W2,
                   table, offsets, subsets, list_of_sample)
+
+
+@dataclass
+class MoeInputs:
+    X: torch.Tensor                 # [N,D]
+    W1: torch.Tensor                # [E,D,F]
+    W2: torch.Tensor                # [E,F,D]
+    kept: np.ndarray                # [E,k_c] int32, ascending per expert
+    expert_ids: np.ndarray          # [N,top_k] int32, distinct per token; -1 = slot not routed
+    expert_weights: np.ndarray      # [N,top_k] float32, sum to 1 per token
+
+
+def generate_moe(N: int, D: int, F: int, E: int, top_k: int, k_c: int, dtype: str = "bf16", seed: int = 0,
+                 skew: float = 1.0, unrouted: float = 0.0, x_std: float = 1.0, w_std: float = 0.05,
+                 device: str = "cpu") -> MoeInputs:
+    """One Sparse-MoE block's inputs with a routing result drawn at random (the router itself is
+    outside the pruned path).  Expert popularity follows p_e ~ (e+1)^-skew, shuffled, so that the
+    per-expert token counts are uneven the way trained routers' are (skew 0: uniform); each token
+    gets top_k DISTINCT experts without replacement and Dirichlet(1) weights; a fraction `unrouted`
+    of the slots is marked -1 (dropped by a capacity limit, or a token that is absent)."""
+    rng = np.random.default_rng(seed)
+    p = (np.arange(E) + 1.0) ** -skew
+    p = rng.permutation(p / p.sum())
+    # Gumbel top-k = sampling without replacement in proportion to p
+    keys = np.log(p)[None, :] + rng.gumbel(size=(N, E))
+    expert_ids = np.argsort(-keys, axis=1)[:, :top_k].astype(np.int32)
+    expert_weights = rng.dirichlet(np.ones(top_k), size=N).astype(np.float32)
+    if unrouted > 0.0:
+        expert_ids[rng.random((N, top_k)) < unrouted] = -1
+    kept = np.stack([np.sort(rng.permutation(F)[:k_c]) for _ in range(E)]).astype(np.int32)
+    dt = torch.float32 if dtype == "f32" else torch.bfloat16
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    normal = lambda shape, std: (torch.randn(shape, generator=gen, device=device, dtype=torch.float32) * std).to(dt)
+    return MoeInputs(normal((N, D), x_std), normal((E, D, F), w_std), normal((E, F, D), w_std), kept,
+                     expert_ids, expert_weights)
