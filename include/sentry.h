@@ -112,10 +112,30 @@ SENTRY_API int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, i
                        const uint32_t* masks, int n_masks, int k, int32_t* kept,
                        uint32_t* kv_groups, int heads_per_group, void* stream);
 
+/* Several selections over the same S mask values in ONE launch (the heads and
+ * the channels of a layer, or the units of several layers): every member of
+ * `sets` (host array, 1 <= n_sets <= SENTRY_GATE_MAX_SETS) has the meaning of
+ * the like-named sentry_gate_select arguments, and the result of each set is
+ * what sentry_gate_select would write for it.  A set with n_masks * k > 16384
+ * needs one more launch for its fan-out.  Workspace: the sum over the sets of
+ * S*k*4 + S*4 bytes, each rounded up to 256. */
+#define SENTRY_GATE_MAX_SETS 4
+typedef struct sentry_gate_set {
+    const float* scores;   /* [S, n_units] fp32 */
+    int n_units, k;
+    const uint32_t* masks; /* [n_masks] u32 */
+    int n_masks;
+    int32_t* kept;         /* out [n_masks, k] */
+    uint32_t* kv_groups;   /* out [n_masks] or NULL */
+    int heads_per_group;
+} sentry_gate_set;
+SENTRY_API int sentry_gate_select_multi(sentry_ctx* ctx, int S, const sentry_gate_set* sets, int n_sets,
+                             void* stream);
+
 /* ---------------------------------------------------------------------------
  * SentryGate on the device (Sec. 4.2, Eq. 1) and the cross-layer threshold of
- * Sec. 4.6 ("evaluate the gate outputs for all layers, then apply a global
- * threshold determined by a desired pruning ratio").
+ * Sec. 4.6 (the gate outputs of all layers are ranked together and cut by one
+ * threshold that the pruning ratio fixes).
  *
  * Units of all layers are concatenated: layer l owns the unit indices
  * [layer_offsets[l], layer_offsets[l+1]), layer_offsets[n_layers] = n_units.

@@ -31,7 +31,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
            "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
            "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out",
-           "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
+           "sentry_gate_select_multi", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -45,6 +45,15 @@ class FfnDesc(ctypes.Structure):
 
 class ProjDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("B", "T", "D", "Hq", "Hk", "d", "k_h", "dtype")]
+
+
+class GateSet(ctypes.Structure):
+    _fields_ = [("scores", ctypes.c_void_p), ("n_units", ctypes.c_int), ("k", ctypes.c_int),
+                ("masks", ctypes.c_void_p), ("n_masks", ctypes.c_int), ("kept", ctypes.c_void_p),
+                ("kv_groups", ctypes.c_void_p), ("heads_per_group", ctypes.c_int)]
+
+
+GATE_MAX_SETS = 4
 
 
 class MoeDesc(ctypes.Structure):
@@ -97,6 +106,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_packed_bytes.restype = ctypes.c_size_t
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
+    lib.sentry_gate_select_multi.argtypes = [vp, ci, ctypes.POINTER(GateSet), ci, vp]
     lib.sentry_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
     lib.sentry_moe_workspace_bytes.restype = ctypes.c_size_t
     lib.sentry_moe_packed_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
@@ -259,6 +269,32 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_gate_select")
         return (kept, groups) if heads_per_group > 0 else kept
+
+    def gate_select_multi(self, sets):
+        """sentry_gate_select_multi: several selections over the same mask values in one launch.
+        `sets`: list of (scores [S,n] fp32, masks [n_masks], k, heads_per_group[, kept]) tuples.  Returns one
+        entry per set: kept, or (kept, kv_groups) where heads_per_group > 0."""
+        arr = (GateSet * len(sets))()
+        outs = []
+        S = sets[0][0].shape[0]
+        need = 1024
+        for i, item in enumerate(sets):
+            scores, masks, k, hpg = item[:4]
+            kept = item[4] if len(item) > 4 else None
+            assert scores.shape[0] == S and scores.dtype == torch.float32
+            n_masks = masks.shape[0]
+            if kept is None:
+                kept = torch.empty((n_masks, k), dtype=torch.int32, device=scores.device)
+            groups = torch.empty((n_masks,), dtype=torch.int32, device=scores.device) if hpg > 0 else None
+            arr[i] = GateSet(_ptr(scores), scores.shape[1], int(k), _ptr(masks), n_masks, _ptr(kept), _ptr(groups),
+                             int(hpg))
+            outs.append((kept, groups) if hpg > 0 else kept)
+            need += S * k * 4 + S * 4 + 512
+        self.ensure_workspace(max(1 << 20, need))
+        rc = self.lib.sentry_gate_select_multi(self.h, S, arr, len(sets), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_gate_select_multi")
+        return outs
 
     def attend_desc(self, Q, K, k_h: int, c: int = 5, score_mode: int = 0) -> AttendDesc:
         B, Hq, T, d = Q.shape

@@ -213,6 +213,35 @@ int sentry_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                               heads_per_group, rows, groups, (cudaStream_t)stream);
 }
 
+int sentry_gate_select_multi(sentry_ctx* ctx, int S, const sentry_gate_set* sets, int n_sets, void* stream) {
+    if (ctx == nullptr || sets == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (n_sets < 1 || n_sets > SENTRY_GATE_MAX_SETS || S < 1) return SENTRY_ERR_BAD_SHAPE;
+    if (S > 65536 / SENTRY_GATE_MAX_SETS) return SENTRY_ERR_UNSUPPORTED;
+    WsAlloc a(ctx->workspace, ctx->workspace_bytes);
+    int32_t* rows[SENTRY_GATE_MAX_SETS];
+    uint32_t* groups[SENTRY_GATE_MAX_SETS];
+    bool any = false;
+    for (int i = 0; i < n_sets; ++i) {
+        const sentry_gate_set& g = sets[i];
+        if (g.scores == nullptr || g.masks == nullptr || g.kept == nullptr) return SENTRY_ERR_INVALID_ARG;
+        if (!aligned(g.scores, 4) || !aligned(g.masks, 4) || !aligned(g.kept, 4)) return SENTRY_ERR_INVALID_ARG;
+        if (g.n_units < 1 || g.n_masks < 0 || g.k < 1 || g.k > g.n_units) return SENTRY_ERR_BAD_SHAPE;
+        if (g.n_units > kMaxUnits) return SENTRY_ERR_UNSUPPORTED;
+        if (g.kv_groups != nullptr) {
+            if (g.heads_per_group < 1) return SENTRY_ERR_INVALID_ARG;
+            if ((g.n_units + g.heads_per_group - 1) / g.heads_per_group > 32) return SENTRY_ERR_BAD_SHAPE;
+        }
+        rows[i] = a.take<int32_t>((size_t)S * g.k);
+        groups[i] = a.take<uint32_t>((size_t)S);
+        any = any || g.n_masks > 0;
+    }
+    ctx->last_launches = 0;
+    if (!any) return SENTRY_OK;
+    if (!a.ok) return SENTRY_ERR_WORKSPACE;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_gate_select_multi(ctx, S, sets, n_sets, rows, groups, (cudaStream_t)stream);
+}
+
 int sentry_gate_eval(sentry_ctx* ctx, int M, int hidden, int n_layers, const int32_t* layer_offsets,
                      int n_units, const float* zeta, const float* gamma, const float* W1, const float* b1,
                      const float* w2, const float* b2, float* logits, float* gates, void* stream) {

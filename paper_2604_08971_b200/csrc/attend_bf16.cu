@@ -972,7 +972,13 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
         return SENTRY_OK;
     }
     const size_t valid_bytes = (((size_t)d.T * 2 + 127) / 128) * 128;
-    if (!a.selection_given) {
+    // scores and selection by one CTA per group with K resident, where the shape allows it; the
+    // streamed kernel then takes the active lists as given
+    const bool long_select = !a.selection_given && attend_long_select_supported(d);
+    if (long_select) {
+        int rc = launch_attend_long_select(ctx, a, st);
+        if (rc != SENTRY_OK) return rc;
+    } else if (!a.selection_given) {
         // K segment: 64 KB worth of rows, a power of two (at most 8 segments for T <= 8192)
         int seg_shift = 0;
         while ((2 << seg_shift) * D * 2 <= 64 * 1024) ++seg_shift;
@@ -994,15 +1000,16 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
         size_t smem = valid_bytes + (((size_t)d.T + 127) / 128) * 128 +
                       (((size_t)kMaxRK * words * 4 + 127) / 128) * 128;
         size_t uni = CoreSmem<D>::PIPE_BYTES;
-        if (!a.selection_given && (size_t)kMaxRK * d.T * 4 > uni) uni = (size_t)kMaxRK * d.T * 4;
+        const bool given = a.selection_given || long_select;
+        if (!given && (size_t)kMaxRK * d.T * 4 > uni) uni = (size_t)kMaxRK * d.T * 4;
         smem += uni;
         auto kern = attend_core_bf16_kernel<D>;
         SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         LaunchScope ls(ctx, KS_ATT_CORE, st);
         kern<<<d.B * d.Hk, kCoreThreads, smem, st>>>(
             (const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, a.kept_heads,
-            a.ids, a.masks, a.mscore, a.selection_given ? a.active : nullptr,
-            a.selection_given ? nullptr : a.active_out_user, d.T, d.Hq, d.Hk, d.k_h, d.c, a.U_max,
+            a.ids, a.masks, a.mscore, given ? a.active : nullptr,
+            given ? nullptr : a.active_out_user, d.T, d.Hq, d.Hk, d.k_h, d.c, a.U_max,
             (__nv_bfloat16*)a.O, a.status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());

@@ -300,6 +300,8 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 #endif  // __CUDACC__
 
 // ---- launchers implemented in the .cu files (host side; return sentry_status)
+int launch_gate_select_multi(sentry_ctx* ctx, int S, const sentry_gate_set* sets, int n_sets, int32_t* const* ws_rows,
+                             uint32_t* const* ws_groups, cudaStream_t st);
 int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                        const uint32_t* masks, int n_masks, int k, int32_t* kept,
                        uint32_t* kv_groups, int heads_per_group, int32_t* ws_rows,
@@ -330,6 +332,8 @@ struct AttendArgs {
 };
 int launch_attend_generic(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_tc_supported(const sentry_attend_desc& d);
+bool attend_long_select_supported(const sentry_attend_desc& d);
+int launch_attend_long_select(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 int launch_attend_tc(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_bf16_supported(const sentry_attend_desc& d);
 int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);

@@ -19,16 +19,15 @@ inline int gate_threads(int n_units) {
 // One block per score-table row s: rows[s, 0..k) and groups[s].  With fan_masks given (a small
 // fan-out), the block also copies its row to every sample whose mask selects it, which saves
 // the second launch: kept[m, :] = rows[s, :] for masks[m] == s.
-__global__ void __launch_bounds__(kGateMaxThreads)
-gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
-                 int32_t* __restrict__ rows, uint32_t* __restrict__ groups,
-                 int heads_per_group, const uint32_t* __restrict__ fan_masks = nullptr,
-                 int n_masks = 0, int S = 0, int32_t* __restrict__ kept = nullptr,
-                 uint32_t* __restrict__ kv_groups = nullptr, unsigned int* status = nullptr) {
+__device__ __forceinline__ void
+gate_row_block(int s, const float* __restrict__ scores, int n_units, int k,
+               int32_t* __restrict__ rows, uint32_t* __restrict__ groups,
+               int heads_per_group, const uint32_t* __restrict__ fan_masks,
+               int n_masks, int S, int32_t* __restrict__ kept,
+               uint32_t* __restrict__ kv_groups, unsigned int* status) {
     extern __shared__ uint32_t s_keys[];
     __shared__ int red[66];
     __shared__ uint32_t s_bits;
-    const int s = blockIdx.x;
     const float* row = scores + (size_t)s * n_units;
     for (int i = threadIdx.x; i < n_units; i += blockDim.x) s_keys[i] = sentry_order_key(row[i]);
     if (threadIdx.x == 0) s_bits = 0u;
@@ -72,6 +71,38 @@ gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
             atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
         }
     }
+}
+
+__global__ void __launch_bounds__(kGateMaxThreads)
+gate_rows_kernel(const float* __restrict__ scores, int n_units, int k,
+                 int32_t* __restrict__ rows, uint32_t* __restrict__ groups,
+                 int heads_per_group, const uint32_t* __restrict__ fan_masks = nullptr,
+                 int n_masks = 0, int S = 0, int32_t* __restrict__ kept = nullptr,
+                 uint32_t* __restrict__ kv_groups = nullptr, unsigned int* status = nullptr) {
+    gate_row_block(blockIdx.x, scores, n_units, k, rows, groups, heads_per_group, fan_masks, n_masks, S, kept,
+                   kv_groups, status);
+}
+
+// Several selections over the same S mask values (heads and channels of a layer, or several
+// layers) in one launch: block b works on row b % S of set b / S.
+struct GateSetDev {
+    const float* scores;
+    int n_units, k;
+    int32_t* rows;
+    uint32_t* groups;
+    int heads_per_group;
+    const uint32_t* fan_masks;   // null: no fan-out in this launch (the set is expanded afterwards)
+    int n_masks;
+    int32_t* kept;
+    uint32_t* kv_groups;
+};
+struct GateSetsDev { GateSetDev set[SENTRY_GATE_MAX_SETS]; };
+
+__global__ void __launch_bounds__(kGateMaxThreads)
+gate_rows_multi_kernel(const __grid_constant__ GateSetsDev sets, int S, unsigned int* status) {
+    const GateSetDev& g = sets.set[blockIdx.x / S];
+    gate_row_block((int)(blockIdx.x % S), g.scores, g.n_units, g.k, g.rows, g.groups, g.heads_per_group,
+                   g.fan_masks, g.n_masks, S, g.kept, g.kv_groups, status);
 }
 
 // kept[m, :] = rows[masks[m], :]  (and kv_groups[m] = groups[masks[m]]).
@@ -134,6 +165,55 @@ int launch_gate_select(sentry_ctx* ctx, const float* scores, int S, int n_units,
                                                    kv_groups, ctx->d_status);
     }
     SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}
+
+// All sets in one launch; a set whose fan-out is large gets its rows there and one expand launch.
+int launch_gate_select_multi(sentry_ctx* ctx, int S, const sentry_gate_set* sets, int n_sets, int32_t* const* ws_rows,
+                             uint32_t* const* ws_groups, cudaStream_t st) {
+    GateSetsDev dev = {};
+    size_t smem = 0;
+    int threads = 64;
+    bool expand[SENTRY_GATE_MAX_SETS] = {};
+    for (int i = 0; i < n_sets; ++i) {
+        const sentry_gate_set& g = sets[i];
+        const size_t total = (size_t)g.n_masks * g.k;
+        expand[i] = total > 16384;
+        GateSetDev& d = dev.set[i];
+        d.scores = g.scores; d.n_units = g.n_units; d.k = g.k;
+        d.rows = ws_rows[i];
+        d.groups = g.kv_groups ? ws_groups[i] : nullptr;
+        d.heads_per_group = g.heads_per_group > 0 ? g.heads_per_group : 1;
+        d.fan_masks = expand[i] ? nullptr : g.masks;
+        d.n_masks = g.n_masks; d.kept = g.kept; d.kv_groups = g.kv_groups;
+        if ((size_t)g.n_units * sizeof(uint32_t) > smem) smem = (size_t)g.n_units * sizeof(uint32_t);
+        int t = gate_threads(g.n_units);
+        if (!expand[i]) {
+            const int fan = g.k <= 32 ? g.n_masks : (int)(total < 1024 ? total : 1024);
+            while (t < 256 && t < fan) t *= 2;
+        }
+        if (t > threads) threads = t;
+    }
+    if (smem > 48 * 1024)
+        SENTRY_CUDA_TRY(cudaFuncSetAttribute(gate_rows_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem));
+    {
+        LaunchScope ls(ctx, KS_GATE_ROWS, st);
+        gate_rows_multi_kernel<<<S * n_sets, threads, smem, st>>>(dev, S, ctx->d_status);
+    }
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    for (int i = 0; i < n_sets; ++i) {
+        if (!expand[i]) continue;
+        const sentry_gate_set& g = sets[i];
+        const size_t total = (size_t)g.n_masks * g.k;
+        int blocks = (int)((total + 255) / 256);
+        const int cap = ctx->sm_count * 8;
+        if (blocks > cap) blocks = cap;
+        LaunchScope ls(ctx, KS_GATE_EXPAND, st);
+        gate_expand_kernel<<<blocks, 256, 0, st>>>(ws_rows[i], ws_groups[i], g.masks, S, g.n_masks, g.k, g.kept,
+                                                   g.kv_groups, ctx->d_status);
+        SENTRY_CUDA_TRY(cudaGetLastError());
+    }
     return SENTRY_OK;
 }
 

@@ -163,6 +163,18 @@ def test_config5_sweep_cells(sn, B, T):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("name,lengths,Hq,Hk,d,k_h", [
+    ("long_d64_segments", (700, 900, 600), 8, 2, 64, 6),    # K of a group: up to 275 KB -> walked in segments, up to 4 heads per group
+    ("long_d16_resident", (2100, 1500, 1400), 6, 3, 16, 4),  # 5000 tokens, K resident in one piece
+    ("long_d32_three_heads", (1300, 1100, 900), 12, 4, 32, 9),
+], ids=lambda v: v if isinstance(v, str) else None)
+def test_long_sequences_selection_by_one_cta_per_group(sn, name, lengths, Hq, Hk, d, k_h):
+    """Sequences whose K and V do not fit in shared memory together: scores and top-U by the
+    one-CTA-per-group kernel (K resident, or walked in segments), Eq. 6 by the streamed kernel."""
+    w = synth.Workload(name, "bf16", 7, lengths, 64, Hq, Hk, d, 128, k_h, 64, "cycle7", 60 + d)
+    _run_workload(sn, w, "all", "all")
+
+
 # ------------------------------------------------------------------ edge cases
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d", [16, 32, 64])
