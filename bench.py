@@ -33,6 +33,8 @@ if ROOT not in sys.path:
 import synth  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+TABLE_LAYOUT = "entry"   # set from --table-layout
+GATE_MULTI = False        # set from --gate-multi
 # fp32 FMA peak of the plain ALUs: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (unit counts and max SM clock)
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
@@ -295,7 +297,12 @@ class Workbench:
         self.subsets = torch.as_tensor(inp.subsets.astype(np.int64).astype(np.int32), device=dev)
         self.los = torch.as_tensor(inp.list_of_sample, device=dev)
         self.sh, self.sc = torch.as_tensor(inp.scores_heads, device=dev), torch.as_tensor(inp.scores_ch, device=dev)
-        self.tbl = torch.as_tensor(inp.sample_table, device=dev)
+        # the sample tables in the layout the kernels read with one 128-byte access per sample and warp
+        # (score_mode 2: entry-major; the same numbers, transposed once here, outside every timed region)
+        self.score_mode = 2 if TABLE_LAYOUT == "entry" else 0
+        tbl_np = synth.entry_major_tables(w, inp.sample_table, inp.table_offsets, self.n_s_of) \
+            if self.score_mode == 2 else inp.sample_table
+        self.tbl = torch.as_tensor(tbl_np, device=dev)
         self.offs = torch.as_tensor(inp.table_offsets, device=dev)
         self.W1, self.W2 = inp.W1, inp.W2
         base = DeviceSet(inp, dev)
@@ -324,8 +331,11 @@ class Workbench:
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
 
-    def ffn_branch(self, s: DeviceSet, ctx):
+    def ffn_branch(self, s: DeviceSet, ctx, gated=False):
         w = self.w
+        if gated:
+            ctx.ffn_fwd(s.X, self.W1, self.W2, s.kept_c, self.los, self.ids, self.masks, Y=s.Y)
+            return ctx.last_launch_count()
         if self.once:
             ctx.ffn_fwd_packed(s.X, self.packed, w.F, w.k_c, len(self.inp.subsets), self.los, self.ids, self.masks, Y=s.Y)
             return ctx.last_launch_count()
@@ -338,19 +348,25 @@ class Workbench:
         w, sn = self.w, self.sn
         n = 0
         two = fork and self.branch is not None
+        multi = GATE_MULTI and not self.once
+        if multi:   # heads and channels selected by one launch, ahead of the fork
+            sn.gate_select_multi([(self.sh, self.masks, w.k_h, 0, s.kept_h), (self.sc, self.subsets, w.k_c, 0, s.kept_c)])
+            n += sn.last_launch_count()
         if two:
             cur = torch.cuda.current_stream()
             self.branch.wait_stream(cur)
             with torch.cuda.stream(self.branch):
-                n += self.ffn_branch(s, self.sn2)
-        sn.gate_select(self.sh, self.masks, w.k_h, kept=s.kept_h)
-        n += sn.last_launch_count()
-        sn.attend_fwd(s.Q, s.K, s.V, s.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s.O)
+                n += self.ffn_branch(s, self.sn2, gated=multi)
+        if not multi:
+            sn.gate_select(self.sh, self.masks, w.k_h, kept=s.kept_h)
+            n += sn.last_launch_count()
+        sn.attend_fwd(s.Q, s.K, s.V, s.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s.O,
+                      score_mode=self.score_mode)
         n += sn.last_launch_count()
         if two:
             torch.cuda.current_stream().wait_stream(self.branch)
         else:
-            n += self.ffn_branch(s, sn)
+            n += self.ffn_branch(s, sn, gated=multi)
         if count:
             self.launches = n
 
@@ -411,7 +427,8 @@ class Workbench:
             sn.gate_select(self.sh, self.masks, w.k_h, kept=s0.kept_h); c += sn.last_launch_count()
             sn.project_qkv(s0.X, WQ, WK, WV, s0.kept_h, self.ids, self.masks, w.Hq, w.Hk, w.d, Q=Q, K=K, V=V)
             c += sn.last_launch_count()
-            sn.attend_fwd(Q, K, V, s0.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s0.O)
+            sn.attend_fwd(Q, K, V, s0.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s0.O,
+                          score_mode=self.score_mode)
             c += sn.last_launch_count()
             sn.project_out(s0.O, WO, s0.kept_h, self.ids, self.masks, w.Hq, out=H); c += sn.last_launch_count()
             sn.gate_select(self.sc, self.subsets, w.k_c, kept=s0.kept_c); c += sn.last_launch_count()
@@ -596,7 +613,7 @@ def run_ours(args, w: synth.Workload):
             cur.wait_event(ups[i])
             sn.gate_select(sh, masks[b0:b1], w.k_h, kept=base.kept_h[b0:b1])
             sn.attend_fwd(base.Q[b0:b1], base.K[b0:b1], base.V[b0:b1], base.kept_h[b0:b1], ids, masks[b0:b1],
-                          tbl, offs, c=w.c, O=base.O[b0:b1])
+                          tbl, offs, c=w.c, O=base.O[b0:b1], score_mode=wb.score_mode)
             sn.gate_select(sc, subsets, w.k_c, kept=kept_c_e2e)
             sn.ffn_fwd(base.X[b0:b1], W1, W2, kept_c_e2e, los[b0:b1], ids, masks[b0:b1], Y=base.Y[b0:b1])
             ev = torch.cuda.Event()
@@ -697,6 +714,8 @@ def run_ours(args, w: synth.Workload):
                    "streams": "attention branch and FFN branch forked inside the step" if two_streams
                               else "one stream",
                    "attend_kernel": args.attend_kernel,
+                   "sample_table_layout": "entry-major (score_mode 2), transposed once outside the timed region"
+                   if args.table_layout == "entry" else "query-major (score_mode 0)",
                    "step_includes": "gate selection for heads and channels, attention, FFN weight gather and FFN, "
                                     "every step (see materialised_once for the weights gathered once)",
                    "timing": "median of %d blocks of %d steps, each block bracketed by barrier + synchronise "
@@ -734,8 +753,16 @@ def main():
     ap.add_argument("--replays", type=int, default=5, help="timed blocks of --steps steps; the median is reported")
     ap.add_argument("--attend-kernel", default="auto", choices=sorted(ATTEND_KERNELS),
                     help="SENTRY_OPT_ATTEND_KERNEL for the attention call")
+    ap.add_argument("--gate-multi", action="store_true",
+                    help="select heads and channels with one sentry_gate_select_multi launch ahead of the fork")
+    ap.add_argument("--table-layout", default="entry", choices=["entry", "query"],
+                    help="layout of the sample tables handed to sentry_attend_fwd: entry-major (score_mode 2) "
+                         "or query-major (score_mode 0); the numbers are the same")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
+    global TABLE_LAYOUT, GATE_MULTI
+    TABLE_LAYOUT = args.table_layout
+    GATE_MULTI = args.gate_multi
     w = synth.by_name(args.config)
     if args.impl == "reference":
         run_reference(args, w)

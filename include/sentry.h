@@ -213,17 +213,21 @@ typedef struct sentry_attend_desc {
     int k_h;             /* kept heads per sample (same for every sample) */
     int dtype;           /* sentry_dtype of Q, K, V, O */
     int c;               /* sparsity constant of U = c*ceil(ln T_v); the paper uses 5 */
-    int score_mode;      /* 0: S_i from the sample table; 1: S_i = all present keys */
+    int score_mode;      /* 0: S_i from the sample table; 1: S_i = all present keys;
+                            2: as 0, the table of every subset stored entry-major */
 } sentry_attend_desc;
 
 /*   Q [B,Hq,T,d]; K, V [B,Hk,T,d]; O out [B,k_h,T,d] (heads in kept-list order)
  *   kept_heads [B,k_h] i32 ascending, in [0,Hq)
  *   token_modality_ids [T] i32 in [0,32); masks [B] u32
  *   sample_table i32 + sample_offsets i64 [2^M entries, indexed by mask value]
- *     (score_mode 0 only, else NULL): sample_table + sample_offsets[m] is the
+ *     (score_mode 0 and 2, else NULL): sample_table + sample_offsets[m] is the
  *     [T_v, U] table of the subset m; row i = the U key positions (indices into
  *     the present-token list, each in [0,T_v)) on which query position i is scored.
  *     Subsets with equal T_v may share one table.  n_subsets = entries of sample_offsets.
+ *     score_mode 2: the same numbers stored [U, T_v] (sample j of query position i
+ *     at j*T_v + i), so that the queries of a warp read one sample with one
+ *     128-byte access; the result is bit for bit that of score_mode 0.
  *   active_out [B,k_h,U_max] i32 or NULL, U_max = sentry_num_active_queries(T,c):
  *     the active token indices, ascending, padded with -1
  *   active_in  same shape or NULL: if given, step 1-2 are skipped and these

@@ -23,7 +23,7 @@ size_t attend_workspace_bytes(const sentry_attend_desc& d) {
 int check_attend_desc(const sentry_attend_desc* d) {
     if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
     if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
-    if (d->score_mode != 0 && d->score_mode != 1) return SENTRY_ERR_INVALID_ARG;
+    if (d->score_mode < 0 || d->score_mode > 2) return SENTRY_ERR_INVALID_ARG;
     if (d->B < 1 || d->T < 1 || d->Hq < 1 || d->Hk < 1 || d->k_h < 1 || d->c < 1)
         return SENTRY_ERR_BAD_SHAPE;
     if (d->Hq % d->Hk != 0 || d->k_h > d->Hq) return SENTRY_ERR_BAD_SHAPE;
@@ -281,7 +281,7 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) ||
         !aligned(kept_heads, 4) || !aligned(token_modality_ids, 4) || !aligned(masks, 4))
         return SENTRY_ERR_INVALID_ARG;
-    if (active_in == nullptr && desc->score_mode == 0) {
+    if (active_in == nullptr && desc->score_mode != 1) {
         if (sample_table == nullptr || sample_offsets == nullptr) return SENTRY_ERR_INVALID_ARG;
         if (n_subsets < 1) return SENTRY_ERR_BAD_SHAPE;
         if (!aligned(sample_table, 4) || !aligned(sample_offsets, 8)) return SENTRY_ERR_INVALID_ARG;

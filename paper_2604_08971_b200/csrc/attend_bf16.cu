@@ -36,7 +36,7 @@ template <int D, int NH>
 __device__ __forceinline__ void long_score_pass(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ Kg,
                                                 const uint16_t* s_valid, uint16_t* s_list, uint32_t ks_addr,
                                                 int seg_shift, int Tv, int Tlen, const size_t* q_base,
-                                                const int* khs, const int32_t* tbl_row, int cnt,
+                                                const int* khs, const int32_t* tbl_row, size_t tbl_es, int cnt,
                                                 int score_mode, int p, int b, int k_h,
                                                 float* __restrict__ mscore, unsigned int* status) {
     using S = Sw<D>;
@@ -58,10 +58,10 @@ __device__ __forceinline__ void long_score_pass(const __nv_bfloat16* __restrict_
                 qw[h][4 * cc] = v.x; qw[h][4 * cc + 1] = v.y; qw[h][4 * cc + 2] = v.z; qw[h][4 * cc + 3] = v.w;
             }
         }
-        if (score_mode == 0) {
+        if (score_mode != 1) {
             unsigned long long counts = 0ull;
             for (int a = 0; a < cnt; ++a) {
-                int pj = __ldg(tbl_row + a);
+                int pj = __ldg(tbl_row + (size_t)a * tbl_es);
                 if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
                 counts += 1ull << (8 * (pj >> seg_shift));
             }
@@ -73,7 +73,7 @@ __device__ __forceinline__ void long_score_pass(const __nv_bfloat16* __restrict_
             }
             unsigned long long fill = starts;
             for (int a = 0; a < cnt; ++a) {
-                int pj = __ldg(tbl_row + a);
+                int pj = __ldg(tbl_row + (size_t)a * tbl_es);
                 if (pj < 0 || pj >= Tv) pj = 0;
                 const int sgm = pj >> seg_shift;
                 const int pos = (int)((fill >> (8 * sgm)) & 255ull);
@@ -94,7 +94,7 @@ __device__ __forceinline__ void long_score_pass(const __nv_bfloat16* __restrict_
         ptx::cp_async_wait_all();
         __syncthreads();
         if (!act) continue;
-        if (score_mode == 0) {
+        if (score_mode != 1) {
             const int i0 = (int)((starts >> (8 * sgm)) & 255ull);
             const int i1 = sgm == 7 ? cnt : (seg0 + seg_rows >= Tv ? cnt : (int)((starts >> (8 * (sgm + 1))) & 255ull));
             for (int i = i0; i < i1; ++i) {
@@ -138,15 +138,16 @@ attend_score_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     if (bad && threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
     if (rk == 0) return;
     const int n_s = sentry_num_active(Tv, c);
-    const int cnt = score_mode == 0 ? n_s : Tv;
+    const int cnt = score_mode != 1 ? n_s : Tv;
     const int p = blockIdx.y * blockDim.x + threadIdx.x;
     const int32_t* tbl_row = nullptr;
-    if (score_mode == 0) {
+    const size_t tbl_es = score_mode == 2 ? (size_t)Tv : 1;   // entry-major table: entry a of row p at a * Tv + p
+    if (score_mode != 1) {
         if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) {
             if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
             return;
         }
-        tbl_row = table + offsets[mask] + (size_t)min(p, Tv - 1) * n_s;
+        tbl_row = table + offsets[mask] + (size_t)min(p, Tv - 1) * (score_mode == 2 ? 1 : n_s);
     }
     const __nv_bfloat16* Kg = K + ((size_t)b * Hk + g) * Tlen * D;
     constexpr int HPP = (D == 64) ? 1 : (D == 32 ? 2 : 4);   // heads per pass: packed q rows live in registers
@@ -160,7 +161,7 @@ attend_score_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
             khs_[j] = khs[hh];
         }
 #define LONG_PASS(N) long_score_pass<D, N>(Q, Kg, s_valid, s_list, ks_addr, seg_shift, Tv, Tlen, q_base, khs_, \
-                                           tbl_row, cnt, score_mode, p, b, k_h, mscore, status)
+                                           tbl_row, tbl_es, cnt, score_mode, p, b, k_h, mscore, status)
         if (nh == 1) LONG_PASS(1);
         else if (nh == 2) LONG_PASS(2);
         else if constexpr (HPP == 4) {
@@ -547,16 +548,18 @@ __device__ __forceinline__ void fused_score_pass(const __nv_bfloat16* __restrict
         // The sampled positions come four at a time, the next four requested before the current
         // four are used: a thread walks its own table row, and with most of the L1 given to
         // shared memory the row's lines do not survive from one use to the next.
-        const int32_t* row = score_mode == 0 ? tbl + (size_t)p * n_s : nullptr;
+        // query-major table: entry a of row p at p * n_s + a; entry-major (score_mode 2): a * Tv + p
+        const int32_t* row = score_mode != 1 ? tbl + (size_t)p * (score_mode == 2 ? 1 : n_s) : nullptr;
+        const size_t es = score_mode == 2 ? (size_t)Tv : 1;
         int nxt[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) nxt[u] = score_mode == 0 ? __ldg(row + min(u, cnt - 1)) : u;
+        for (int u = 0; u < 4; ++u) nxt[u] = score_mode != 1 ? __ldg(row + (size_t)min(u, cnt - 1) * es) : u;
         for (int a0 = 0; a0 < cnt; a0 += 4) {
             int cur[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 cur[u] = nxt[u];
-                nxt[u] = score_mode == 0 ? __ldg(row + min(a0 + 4 + u, cnt - 1)) : a0 + 4 + u;
+                nxt[u] = score_mode != 1 ? __ldg(row + (size_t)min(a0 + 4 + u, cnt - 1) * es) : a0 + 4 + u;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -712,10 +715,10 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     if (active_in == nullptr) {
         // ---- sparsity scores (Section 4.4) from the resident K rows
         const int n_s = U;
-        const int cnt = score_mode == 0 ? n_s : Tv;
+        const int cnt = score_mode != 1 ? n_s : Tv;
         const int32_t* tbl = nullptr;
         bool table_ok = true;
-        if (score_mode == 0) {
+        if (score_mode != 1) {
             if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) table_ok = false;
             else tbl = table + offsets[mask];
         }

@@ -64,7 +64,7 @@ attend_score_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     const int g = h / (Hq / Hk);
     const int n_s = sentry_num_active(Tv, c);
     const int32_t* tbl = nullptr;
-    if (score_mode == 0) {
+    if (score_mode != 1) {
         if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) {
             if (threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
             return;
@@ -77,10 +77,10 @@ attend_score_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     float q[D], kr[D];
     load_row<T, D>(Qh + (size_t)s_valid[p] * D, q);
     const float scale = 1.0f / sqrtf((float)D);
-    const int cnt = (score_mode == 0) ? n_s : Tv;
+    const int cnt = (score_mode != 1) ? n_s : Tv;
     float mx = -INFINITY, sum = 0.f;
     for (int a = 0; a < cnt; ++a) {
-        int pj = (score_mode == 0) ? tbl[(size_t)p * n_s + a] : a;
+        int pj = (score_mode == 0) ? tbl[(size_t)p * n_s + a] : (score_mode == 2 ? tbl[(size_t)a * Tv + p] : a);
         if (pj < 0 || pj >= Tv) { atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); pj = 0; }
         load_row<T, D>(Kg + (size_t)s_valid[pj] * D, kr);
         float dot = 0.f;

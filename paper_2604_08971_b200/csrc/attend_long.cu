@@ -41,18 +41,20 @@ __device__ __forceinline__ void long_score_segment(const __nv_bfloat16* __restri
             mx[h] = first ? -INFINITY : __uint_as_float(keys[h][p]);
             sum[h] = first ? 0.f : sums[h][p];
         }
-        if (score_mode == 0) {
-            // sampled positions, requested four ahead of their use (a thread walks its own table row)
-            const int32_t* row = tbl + (size_t)p * n_s;
+        if (score_mode != 1) {
+            // sampled positions, requested four ahead of their use.  Query-major table: entry a of
+            // row p at p * n_s + a; entry-major (score_mode 2): a * Tv + p
+            const int32_t* row = tbl + (size_t)p * (score_mode == 2 ? 1 : n_s);
+            const size_t es = score_mode == 2 ? (size_t)Tv : 1;
             int nxt[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) nxt[u] = __ldg(row + min(u, cnt - 1));
+            for (int u = 0; u < 4; ++u) nxt[u] = __ldg(row + (size_t)min(u, cnt - 1) * es);
             for (int a0 = 0; a0 < cnt; a0 += 4) {
                 int cur[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     cur[u] = nxt[u];
-                    nxt[u] = __ldg(row + min(a0 + 4 + u, cnt - 1));
+                    nxt[u] = __ldg(row + (size_t)min(a0 + 4 + u, cnt - 1) * es);
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -106,10 +108,10 @@ attend_long_select_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat
     }
     const int U = sentry_num_active(Tv, c);
     const int n_s = U;
-    const int cnt = score_mode == 0 ? n_s : Tv;
+    const int cnt = score_mode != 1 ? n_s : Tv;
     const int32_t* tbl = nullptr;
     bool table_ok = true;
-    if (score_mode == 0) {
+    if (score_mode != 1) {
         if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) table_ok = false;
         else tbl = table + offsets[mask];
     }

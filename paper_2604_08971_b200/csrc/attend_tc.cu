@@ -176,16 +176,17 @@ __device__ __forceinline__ void score_pass_gather(const __nv_bfloat16* __restric
         // The sampled positions come four at a time, the next four requested before the current
         // four are used: a thread walks its own 4 n_s-byte table row, and with most of the L1
         // given to shared memory the row's lines do not survive from one use to the next.
-        const int32_t* row = score_mode == 0 ? tbl + (size_t)p * n_s : nullptr;
+        const int32_t* row = score_mode != 1 ? tbl + (size_t)p * (score_mode == 2 ? 1 : n_s) : nullptr;
+        const size_t es = score_mode == 2 ? (size_t)Tv : 1;   // entry-major table: entry a of row p at a * Tv + p
         int nxt[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) nxt[u] = score_mode == 0 ? __ldg(row + min(u, cnt - 1)) : u;
+        for (int u = 0; u < 4; ++u) nxt[u] = score_mode != 1 ? __ldg(row + (size_t)min(u, cnt - 1) * es) : u;
         for (int a0 = 0; a0 < cnt; a0 += 4) {
             int cur[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 cur[u] = nxt[u];
-                nxt[u] = score_mode == 0 ? __ldg(row + min(a0 + 4 + u, cnt - 1)) : a0 + 4 + u;
+                nxt[u] = score_mode != 1 ? __ldg(row + (size_t)min(a0 + 4 + u, cnt - 1) * es) : a0 + 4 + u;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -422,10 +423,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_k64, const __grid_consta
     bool ok = __syncthreads_and(warp_wait(&misc->k_full, 0u, abort_flag) ? 1 : 0) != 0;   // block-uniform
 
     const int n_s = U;
-    const int cnt = score_mode == 0 ? n_s : Tv;
+    const int cnt = score_mode != 1 ? n_s : Tv;
     const int32_t* tbl = nullptr;
     bool table_ok = true;
-    if (score_mode == 0 && active_in == nullptr) {
+    if (score_mode != 1 && active_in == nullptr) {
         if (mask >= (uint32_t)n_subsets || offsets[mask] < 0) table_ok = false;
         else tbl = table + offsets[mask];
     }

@@ -180,6 +180,21 @@ def make_sample_tables(w: Workload, masks: np.ndarray, n_samples_of: Callable[[i
     return flat, offsets
 
 
+def entry_major_tables(w: Workload, flat: np.ndarray, offsets: np.ndarray,
+                       n_samples_of: Callable[[int], int]) -> np.ndarray:
+    """The same tables with every [T_v, n_s] block stored transposed ([n_s, T_v]); offsets unchanged."""
+    out = flat.copy()
+    done = set()
+    for s, off in enumerate(offsets):
+        if off < 0 or int(off) in done:
+            continue
+        done.add(int(off))
+        tv = present_count(w, s)
+        n_s = int(n_samples_of(tv))
+        out[off:off + tv * n_s] = flat[off:off + tv * n_s].reshape(tv, n_s).T.reshape(-1)
+    return out
+
+
 @dataclass
 class Inputs:
     w: Workload

@@ -175,6 +175,34 @@ def test_long_sequences_selection_by_one_cta_per_group(sn, name, lengths, Hq, Hk
     _run_workload(sn, w, "all", "all")
 
 
+@pytest.mark.parametrize("w,kernel", [
+    (synth.config1(), sentry.ATTEND_AUTO),                                         # fp32: plain-ALU kernels
+    (synth.config4().with_(B=9), sentry.ATTEND_AUTO),                              # fused warp-MMA kernel
+    (synth.config4().with_(B=9), sentry.ATTEND_TCGEN05),                           # tcgen05 kernel
+    (synth.config2().with_(B=12), sentry.ATTEND_AUTO),                             # short sequences, 128-thread CTAs
+    (synth.Workload("long_em", "bf16", 7, (1300, 1100, 900), 64, 8, 2, 32, 128, 4, 64, "cycle7", 91), sentry.ATTEND_AUTO),
+    (synth.Workload("long_em_d64", "bf16", 7, (700, 900, 600), 64, 8, 2, 64, 128, 6, 64, "cycle7", 92), sentry.ATTEND_AUTO),
+], ids=lambda v: v.name if isinstance(v, synth.Workload) else str(v))
+def test_entry_major_sample_table_gives_the_same_bits(sn, w, kernel):
+    """score_mode 2 reads the same sample sets from the transposed table, in the same order:
+    the output and the active lists must equal those of score_mode 0 bit for bit."""
+    inp = synth.generate(w, n_s_of)
+    kept_h, _ = parity.gate_lists(sn, inp)
+    ids, masks = dev(inp.ids), masks_dev(inp.masks)
+    tbl, offs = dev(inp.sample_table), dev(inp.table_offsets)
+    tbl_em = dev(synth.entry_major_tables(w, inp.sample_table, inp.table_offsets, n_s_of))
+    Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
+    sn.set_attend_kernel(kernel)
+    try:
+        O0, act0 = sn.attend_fwd(Q, K, V, kept_h, ids, masks, tbl, offs, c=w.c, score_mode=0, return_active=True)
+        O2, act2 = sn.attend_fwd(Q, K, V, kept_h, ids, masks, tbl_em, offs, c=w.c, score_mode=2, return_active=True)
+    finally:
+        sn.set_attend_kernel(sentry.ATTEND_AUTO)
+    assert sn.last_status() == 0
+    assert torch.equal(act0, act2)
+    assert torch.equal(O0, O2)
+
+
 # ------------------------------------------------------------------ edge cases
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d", [16, 32, 64])
