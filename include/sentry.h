@@ -360,6 +360,16 @@ SENTRY_API int sentry_project_out(sentry_ctx* ctx, const sentry_proj_desc* desc,
 #define SENTRY_ATTEND_AUTO 0
 #define SENTRY_ATTEND_WARP_MMA 1
 #define SENTRY_ATTEND_TCGEN05 2
+/* SENTRY_OPT_LONG_SELECT: sequences whose K and V do not fit in shared memory
+ * together take their scores and top-U selection either from a grid of
+ * 256-query blocks per (sample, KV group) (QUERY_BLOCKS) or from one CTA per
+ * group with the group's K rows resident (PER_GROUP: K staged once instead of
+ * once per query block; needs about a group per SM to pay).  AUTO: PER_GROUP
+ * when B*Hk >= the number of SMs.  Same results either way. */
+#define SENTRY_OPT_LONG_SELECT 2
+#define SENTRY_LONG_SELECT_AUTO 0
+#define SENTRY_LONG_SELECT_QUERY_BLOCKS 1
+#define SENTRY_LONG_SELECT_PER_GROUP 2
 SENTRY_API int sentry_set_option(sentry_ctx* ctx, int option, int value);
 
 /* ---------------------------------------------------------------------------

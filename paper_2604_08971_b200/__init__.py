@@ -23,6 +23,8 @@ SENTRY_F32, SENTRY_BF16 = 0, 1
 STATUS_BIT_TIMEOUT, STATUS_BIT_EMPTY_MASK, STATUS_BIT_BAD_INDEX = 1, 2, 4
 OPT_ATTEND_KERNEL = 1
 ATTEND_AUTO, ATTEND_WARP_MMA, ATTEND_TCGEN05 = 0, 1, 2
+OPT_LONG_SELECT = 2
+LONG_SELECT_AUTO, LONG_SELECT_QUERY_BLOCKS, LONG_SELECT_PER_GROUP = 0, 1, 2
 
 EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_status_string",
            "sentry_num_active_queries", "sentry_workspace_bytes", "sentry_set_workspace",
@@ -231,6 +233,11 @@ class Sentry:
     def set_attend_kernel(self, which: int):
         """SENTRY_OPT_ATTEND_KERNEL: ATTEND_AUTO, ATTEND_WARP_MMA or ATTEND_TCGEN05."""
         rc = self.lib.sentry_set_option(self.h, OPT_ATTEND_KERNEL, int(which))
+        if rc != 0:
+            raise SentryError(rc, "sentry_set_option")
+
+    def set_option(self, option: int, value: int):
+        rc = self.lib.sentry_set_option(self.h, int(option), int(value))
         if rc != 0:
             raise SentryError(rc, "sentry_set_option")
 

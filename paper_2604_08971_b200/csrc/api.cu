@@ -63,6 +63,7 @@ int sentry_create(sentry_ctx** out, int device) {
     c->last_launches = 0;
     c->profiling = false;
     c->attend_kernel = SENTRY_ATTEND_AUTO;
+    c->long_select = SENTRY_LONG_SELECT_AUTO;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return SENTRY_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
@@ -182,6 +183,10 @@ int sentry_set_option(sentry_ctx* ctx, int option, int value) {
         case SENTRY_OPT_ATTEND_KERNEL:
             if (value < SENTRY_ATTEND_AUTO || value > SENTRY_ATTEND_TCGEN05) return SENTRY_ERR_INVALID_ARG;
             ctx->attend_kernel = value;
+            return SENTRY_OK;
+        case SENTRY_OPT_LONG_SELECT:
+            if (value < SENTRY_LONG_SELECT_AUTO || value > SENTRY_LONG_SELECT_PER_GROUP) return SENTRY_ERR_INVALID_ARG;
+            ctx->long_select = value;
             return SENTRY_OK;
         default:
             return SENTRY_ERR_INVALID_ARG;

@@ -977,7 +977,11 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
     const size_t valid_bytes = (((size_t)d.T * 2 + 127) / 128) * 128;
     // scores and selection by one CTA per group with K resident, where the shape allows it; the
     // streamed kernel then takes the active lists as given
-    const bool long_select = !a.selection_given && attend_long_select_supported(d);
+    // (it needs about a CTA per SM to pay: with fewer groups than SMs the query-block score kernel,
+    // which spreads a group over T/256 CTAs, is the faster one -- 0.32 against 0.52 ms on B=16, T=4096)
+    const bool want_long = ctx->long_select == SENTRY_LONG_SELECT_PER_GROUP ||
+                           (ctx->long_select == SENTRY_LONG_SELECT_AUTO && d.B * d.Hk >= ctx->sm_count);
+    const bool long_select = !a.selection_given && want_long && attend_long_select_supported(d);
     if (long_select) {
         int rc = launch_attend_long_select(ctx, a, st);
         if (rc != SENTRY_OK) return rc;

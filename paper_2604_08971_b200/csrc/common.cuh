@@ -28,6 +28,7 @@ struct sentry_ctx {
     int sm_count;
     bool profiling;
     int attend_kernel;       // SENTRY_ATTEND_AUTO / _WARP_MMA / _TCGEN05
+    int long_select;         // SENTRY_LONG_SELECT_AUTO / _QUERY_BLOCKS / _PER_GROUP
     std::vector<ProfRec> prof;      // events recorded since profiling was enabled
     std::vector<cudaEvent_t> pool;  // reusable events
 };

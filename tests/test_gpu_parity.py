@@ -172,7 +172,12 @@ def test_long_sequences_selection_by_one_cta_per_group(sn, name, lengths, Hq, Hk
     """Sequences whose K and V do not fit in shared memory together: scores and top-U by the
     one-CTA-per-group kernel (K resident, or walked in segments), Eq. 6 by the streamed kernel."""
     w = synth.Workload(name, "bf16", 7, lengths, 64, Hq, Hk, d, 128, k_h, 64, "cycle7", 60 + d)
-    _run_workload(sn, w, "all", "all")
+    try:
+        for form in (sentry.LONG_SELECT_PER_GROUP, sentry.LONG_SELECT_QUERY_BLOCKS):
+            sn.set_option(sentry.OPT_LONG_SELECT, form)
+            _run_workload(sn, w, "all", "all")
+    finally:
+        sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_AUTO)
 
 
 @pytest.mark.parametrize("w,kernel", [
@@ -193,13 +198,19 @@ def test_entry_major_sample_table_gives_the_same_bits(sn, w, kernel):
     tbl_em = dev(synth.entry_major_tables(w, inp.sample_table, inp.table_offsets, n_s_of))
     Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
     sn.set_attend_kernel(kernel)
+    sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_PER_GROUP)
     try:
         O0, act0 = sn.attend_fwd(Q, K, V, kept_h, ids, masks, tbl, offs, c=w.c, score_mode=0, return_active=True)
         O2, act2 = sn.attend_fwd(Q, K, V, kept_h, ids, masks, tbl_em, offs, c=w.c, score_mode=2, return_active=True)
+        # the query-block form of the long-sequence selection reads the same table
+        sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_QUERY_BLOCKS)
+        O3 = sn.attend_fwd(Q, K, V, kept_h, ids, masks, tbl_em, offs, c=w.c, score_mode=2)
     finally:
         sn.set_attend_kernel(sentry.ATTEND_AUTO)
+        sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_AUTO)
     assert sn.last_status() == 0
     assert torch.equal(act0, act2)
+    assert torch.equal(O0, O3)
     assert torch.equal(O0, O2)
 
 
