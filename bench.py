@@ -33,8 +33,9 @@ if ROOT not in sys.path:
 import synth  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-TABLE_LAYOUT = "entry"   # set from --table-layout
+TABLE_LAYOUT = "auto"   # set from --table-layout
 GATE_MULTI = False        # set from --gate-multi
+LONG_SELECT = 0           # set from --long-select (SENTRY_OPT_LONG_SELECT)
 # fp32 FMA peak of the plain ALUs: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (unit counts and max SM clock)
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
@@ -287,6 +288,7 @@ class Workbench:
         self.sn2 = sentry.Sentry(local_rank) if overlap else self.sn
         for c in (self.sn, self.sn2):
             c.set_attend_kernel(attend_kernel)
+            c.set_option(sentry.OPT_LONG_SELECT, LONG_SELECT)
         self.branch = torch.cuda.Stream() if overlap else None
         self.once = materialise_once
         self.n_s_of = lambda tv: sentry.num_active_queries(tv, w.c)
@@ -299,10 +301,18 @@ class Workbench:
         self.sh, self.sc = torch.as_tensor(inp.scores_heads, device=dev), torch.as_tensor(inp.scores_ch, device=dev)
         # the sample tables in the layout the kernels read with one 128-byte access per sample and warp
         # (score_mode 2: entry-major; the same numbers, transposed once here, outside every timed region)
-        self.score_mode = 2 if TABLE_LAYOUT == "entry" else 0
+        layout = TABLE_LAYOUT
+        if layout == "auto":
+            # the bank-friendly order pays where a group's K and V rows sit in shared memory for the whole
+            # call (+3 %); kernels that walk K in segments want a query's samples in ascending order
+            layout = "arranged" if w.T * (4 * w.d + 20) + 4096 <= 200 * 1024 else "entry"
+        self.table_layout = layout
+        self.score_mode = 0 if layout == "query" else 2
         tbl_np = synth.entry_major_tables(w, inp.sample_table, inp.table_offsets, self.n_s_of) \
-            if self.score_mode == 2 else inp.sample_table
+            if layout == "entry" else inp.sample_table
         self.tbl = torch.as_tensor(tbl_np, device=dev)
+        if layout == "arranged":   # sentry_sample_table_arrange: entry-major, bank-friendly visiting order
+            self.tbl = self.sn.sample_table_arrange(self.ids, self.tbl, torch.as_tensor(inp.table_offsets, device=dev), c=w.c)
         self.offs = torch.as_tensor(inp.table_offsets, device=dev)
         self.W1, self.W2 = inp.W1, inp.W2
         base = DeviceSet(inp, dev)
@@ -714,8 +724,9 @@ def run_ours(args, w: synth.Workload):
                    "streams": "attention branch and FFN branch forked inside the step" if two_streams
                               else "one stream",
                    "attend_kernel": args.attend_kernel,
-                   "sample_table_layout": "entry-major (score_mode 2), transposed once outside the timed region"
-                   if args.table_layout == "entry" else "query-major (score_mode 0)",
+                   "sample_table_layout": {"arranged": "sentry_sample_table_arrange, once, outside the timed region (score_mode 2)",
+                                           "entry": "entry-major (score_mode 2), transposed once outside the timed region",
+                                           "query": "query-major (score_mode 0)"}[wb.table_layout],
                    "step_includes": "gate selection for heads and channels, attention, FFN weight gather and FFN, "
                                     "every step (see materialised_once for the weights gathered once)",
                    "timing": "median of %d blocks of %d steps, each block bracketed by barrier + synchronise "
@@ -753,14 +764,19 @@ def main():
     ap.add_argument("--replays", type=int, default=5, help="timed blocks of --steps steps; the median is reported")
     ap.add_argument("--attend-kernel", default="auto", choices=sorted(ATTEND_KERNELS),
                     help="SENTRY_OPT_ATTEND_KERNEL for the attention call")
+    ap.add_argument("--long-select", default="auto", choices=["auto", "query-blocks", "per-group"],
+                    help="SENTRY_OPT_LONG_SELECT: form of the score + selection step for sequences whose K/V do not fit in shared memory")
     ap.add_argument("--gate-multi", action="store_true",
                     help="select heads and channels with one sentry_gate_select_multi launch ahead of the fork")
-    ap.add_argument("--table-layout", default="entry", choices=["entry", "query"],
-                    help="layout of the sample tables handed to sentry_attend_fwd: entry-major (score_mode 2) "
-                         "or query-major (score_mode 0); the numbers are the same")
+    ap.add_argument("--table-layout", default="auto", choices=["auto", "arranged", "entry", "query"],
+                    help="sample tables handed to sentry_attend_fwd: prepared once by sentry_sample_table_arrange "
+                         "(score_mode 2), plainly transposed (score_mode 2), or query-major as generated (score_mode 0); "
+                         "auto: arranged where K and V of a group fit in shared memory, transposed otherwise; "
+                         "the sampled sets are the same")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
-    global TABLE_LAYOUT, GATE_MULTI
+    global TABLE_LAYOUT, GATE_MULTI, LONG_SELECT
+    LONG_SELECT = {"auto": 0, "query-blocks": 1, "per-group": 2}[args.long_select]
     TABLE_LAYOUT = args.table_layout
     GATE_MULTI = args.gate_multi
     w = synth.by_name(args.config)

@@ -242,6 +242,27 @@ SENTRY_API int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc
                       int n_subsets, void* O, int32_t* active_out,
                       const int32_t* active_in, void* stream);
 
+/* Preparation of the sample tables for score_mode 2, once per set of tables
+ * (Sec. 4.4 fixes WHICH keys a query is scored on, not the order they are
+ * visited in).  Reads the tables as score_mode 0 takes them ([T_v, U] per
+ * subset, offsets per mask value) and writes them entry-major into out_table
+ * (same size, same offsets, must not overlap sample_table), the U members of
+ * every query's set reordered so that the 8 queries of a shared-memory access
+ * phase read key rows on different banks wherever the sets allow it.  The sets
+ * themselves are unchanged; the sparsity scores change by the rounding of a
+ * different summation order only.  Subsets sharing one table are written
+ * twice with the same values.  Entries outside [0,T_v) are flagged BAD_INDEX
+ * and replaced by 0.  U(T, c) <= 64.  Where it pays: the kernels that keep a
+ * group's K rows in shared memory for the whole call (about -3 % on them:
+ * conflicts are a quarter of what they were, the gather is latency-bound
+ * otherwise).  Sequences long enough for K to be walked in segments are better
+ * served by the plain transposition of ascending tables, which keeps a warp's
+ * samples of one step in one segment. */
+SENTRY_API int sentry_sample_table_arrange(sentry_ctx* ctx, int T, int c,
+                                const int32_t* token_modality_ids, const int32_t* sample_table,
+                                const int64_t* sample_offsets, int n_subsets,
+                                int32_t* out_table, void* stream);
+
 /* The same with the pruned weights materialised ONCE, as Sec. 4.6 describes
  * ("materialize a pruned model" per modality mask and budget), instead of on
  * every call:

@@ -33,7 +33,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
            "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
            "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out",
-           "sentry_gate_select_multi", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
+           "sentry_gate_select_multi", "sentry_sample_table_arrange", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -109,6 +109,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_gate_select_multi.argtypes = [vp, ci, ctypes.POINTER(GateSet), ci, vp]
+    lib.sentry_sample_table_arrange.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp]
     lib.sentry_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
     lib.sentry_moe_workspace_bytes.restype = ctypes.c_size_t
     lib.sentry_moe_packed_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
@@ -302,6 +303,17 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_gate_select_multi")
         return outs
+
+    def sample_table_arrange(self, token_modality_ids, sample_table, sample_offsets, c: int = 5, out=None):
+        """sentry_sample_table_arrange: the tables for score_mode 2 (entry-major, bank-friendly order)."""
+        if out is None:
+            out = torch.empty_like(sample_table)
+        rc = self.lib.sentry_sample_table_arrange(self.h, token_modality_ids.shape[0], int(c), _ptr(token_modality_ids),
+                                                  _ptr(sample_table), _ptr(sample_offsets), sample_offsets.shape[0],
+                                                  _ptr(out), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_sample_table_arrange")
+        return out
 
     def attend_desc(self, Q, K, k_h: int, c: int = 5, score_mode: int = 0) -> AttendDesc:
         B, Hq, T, d = Q.shape

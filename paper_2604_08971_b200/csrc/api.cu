@@ -98,7 +98,7 @@ int sentry_profile_slots(void) { return KS_COUNT; }
 const char* sentry_kernel_name(int slot) {
     static const char* names[KS_COUNT] = {"gate_rows", "gate_expand", "attend_score", "attend_select",
                                           "attend_core", "ffn_prepare", "ffn_main", "gate_eval", "project_qkv", "project_out",
-                                          "moe_plan", "moe_combine"};
+                                          "moe_plan", "moe_combine", "table_arrange"};
     return (slot >= 0 && slot < KS_COUNT) ? names[slot] : "?";
 }
 
@@ -325,6 +325,22 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
                                         cudaMemcpyDeviceToDevice, st));
     }
     return SENTRY_OK;
+}
+
+int sentry_sample_table_arrange(sentry_ctx* ctx, int T, int c, const int32_t* token_modality_ids,
+                                const int32_t* sample_table, const int64_t* sample_offsets, int n_subsets,
+                                int32_t* out_table, void* stream) {
+    if (ctx == nullptr || token_modality_ids == nullptr || sample_table == nullptr || sample_offsets == nullptr ||
+        out_table == nullptr)
+        return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(sample_table, 4) || !aligned(out_table, 4) || !aligned(sample_offsets, 8)) return SENTRY_ERR_INVALID_ARG;
+    if (out_table == sample_table) return SENTRY_ERR_INVALID_ARG;
+    if (T < 1 || c < 1 || n_subsets < 1) return SENTRY_ERR_BAD_SHAPE;
+    if (T > 32768 || n_subsets > 65536) return SENTRY_ERR_UNSUPPORTED;
+    ctx->last_launches = 0;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_table_arrange(ctx, token_modality_ids, T, c, sample_table, sample_offsets, n_subsets, out_table,
+                                (cudaStream_t)stream);
 }
 
 int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, const void* W1,

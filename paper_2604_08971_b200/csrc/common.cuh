@@ -14,7 +14,7 @@
 enum KernelSlot {
     KS_GATE_ROWS = 0, KS_GATE_EXPAND, KS_ATT_SCORE, KS_ATT_SELECT, KS_ATT_CORE,
     KS_FFN_PREPARE, KS_FFN_MAIN, KS_GATE_EVAL, KS_PROJ_QKV, KS_PROJ_OUT,
-    KS_MOE_PLAN, KS_MOE_COMBINE, KS_COUNT
+    KS_MOE_PLAN, KS_MOE_COMBINE, KS_TABLE_ARRANGE, KS_COUNT
 };
 
 struct ProfRec { cudaEvent_t start, stop; int slot; };
@@ -333,6 +333,8 @@ struct AttendArgs {
 };
 int launch_attend_generic(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_tc_supported(const sentry_attend_desc& d);
+int launch_table_arrange(sentry_ctx* ctx, const int32_t* ids, int T, int c, const int32_t* table,
+                         const int64_t* offsets, int n_subsets, int32_t* out, cudaStream_t st);
 bool attend_long_select_supported(const sentry_attend_desc& d);
 int launch_attend_long_select(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 int launch_attend_tc(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);

@@ -127,10 +127,12 @@ def _pick(t: torch.Tensor, sel: np.ndarray) -> torch.Tensor:
 
 
 def attend_parity(sn, inp: synth.Inputs, kept_h: torch.Tensor, samples=None, score_mode: int = 0,
-                  full_batch: bool = False):
+                  full_batch: bool = False, arranged: bool = False):
     """Sparse-GQA parity on the samples `samples` (default: all).  With full_batch the CUDA call
     runs on the WHOLE batch (the launch shape the benchmark times) and the oracle checks the
     chosen samples of its output; otherwise the call itself only gets those samples.
+    With `arranged` the CUDA call gets the tables from sentry_sample_table_arrange (score_mode 2)
+    while the oracle keeps the tables as generated: the sets are the same, the visiting order is not.
     Returns (bounded relative error, number of near-tie selections)."""
     w = inp.w
     sel = np.arange(w.B) if samples is None else np.asarray(samples)
@@ -142,8 +144,13 @@ def attend_parity(sn, inp: synth.Inputs, kept_h: torch.Tensor, samples=None, sco
     kh_run = (kept_h if whole else _pick(kept_h, run)).contiguous()
     tbl = dev(inp.sample_table) if score_mode == 0 else None
     offs = dev(inp.table_offsets) if score_mode == 0 else None
+    gpu_mode = score_mode
+    if arranged:
+        assert score_mode == 0
+        tbl = sn.sample_table_arrange(dev(inp.ids), tbl, offs, c=w.c)
+        gpu_mode = 2
     O, act = sn.attend_fwd(Qd, Kd, Vd, kh_run, dev(inp.ids), masks_dev(inp.masks[run]), tbl, offs, c=w.c,
-                           score_mode=score_mode, return_active=True)
+                           score_mode=gpu_mode, return_active=True)
     assert sn.last_status() == 0
     pos = sel if whole else np.arange(len(sel))       # rows of the CUDA call that are compared
     Qc, Kc, Vc = (_pick(t, pos).cpu() for t in (Qd, Kd, Vd))
@@ -169,7 +176,7 @@ def attend_parity(sn, inp: synth.Inputs, kept_h: torch.Tensor, samples=None, sco
             a = act[i, j]
             active_rows[i, j, a[a >= 0]] = True
     err = rel_err(got, want, w.dtype, active_rows)
-    record(w.name, "attend", err, raw_rel_err(got, want),
+    record(w.name, "attend" + ("*" if arranged else ""), err, raw_rel_err(got, want),
            "%d of %d samples checked, call on %d, near-tie selections %d" % (len(sel), w.B, len(run), near_ties))
     return err, near_ties
 

@@ -214,6 +214,48 @@ def test_entry_major_sample_table_gives_the_same_bits(sn, w, kernel):
     assert torch.equal(O0, O2)
 
 
+@pytest.mark.parametrize("w", [
+    synth.config1(), synth.config2().with_(B=12), synth.config4().with_(B=9), synth.config3().with_(B=3),
+    synth.Workload("ragged_arr", "bf16", 5, (37, 5, 91), 72, 6, 3, 64, 200, 4, 77, "cycle7", 47),
+    synth.Workload("long_arr", "bf16", 7, (1300, 1100, 900), 64, 8, 2, 32, 128, 4, 64, "cycle7", 93),
+], ids=lambda w: w.name)
+def test_arranged_sample_tables_keep_the_sets_and_the_parity(sn, w):
+    """sentry_sample_table_arrange: every query keeps exactly its sampled set (bit-exact integer
+    work), stored entry-major; attention on the arranged tables meets the same bound against the
+    oracle, which reads the tables as generated."""
+    inp = synth.generate(w, n_s_of)
+    ids, tbl, offs = dev(inp.ids), dev(inp.sample_table), dev(inp.table_offsets)
+    arr = sn.sample_table_arrange(ids, tbl, offs, c=w.c)
+    assert sn.last_status() == 0
+    arr_np = arr.cpu().numpy()
+    seen = set()
+    worse = better = 0
+    for s, off in enumerate(inp.table_offsets):
+        if off < 0 or int(off) in seen:
+            continue
+        seen.add(int(off))
+        tv = synth.present_count(w, s)
+        n_s = n_s_of(tv)
+        orig = inp.sample_table[off:off + tv * n_s].reshape(tv, n_s)
+        got = arr_np[off:off + tv * n_s].reshape(n_s, tv).T
+        np.testing.assert_array_equal(np.sort(got, axis=1), np.sort(orig, axis=1))
+        # rows read in one access phase (8 consecutive queries, same step): fewer equal residues mod 8
+        for q0 in range(0, tv - 7, 8):
+            for a in range(n_s):
+                worse += np.bincount(orig[q0:q0 + 8, a] % 8, minlength=8).max()
+                better += np.bincount(got[q0:q0 + 8, a] % 8, minlength=8).max()
+    if worse:
+        assert better <= worse
+    kept_h, _ = parity.gate_lists(sn, inp)
+    try:
+        for form in (sentry.LONG_SELECT_PER_GROUP, sentry.LONG_SELECT_QUERY_BLOCKS):
+            sn.set_option(sentry.OPT_LONG_SELECT, form)
+            err, _ = parity.attend_parity(sn, inp, kept_h, None, 0, full_batch=True, arranged=True)
+            assert err <= TOL[w.dtype], (w.name, err)
+    finally:
+        sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_AUTO)
+
+
 # ------------------------------------------------------------------ edge cases
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d", [16, 32, 64])
