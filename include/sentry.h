@@ -62,7 +62,10 @@ typedef enum {
 #define SENTRY_STATUS_BIT_EMPTY_MASK 2u
 #define SENTRY_STATUS_BIT_BAD_INDEX 4u /* a kept index / token id out of range was skipped */
 
-typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1 } sentry_dtype;
+/* SENTRY_F16 (IEEE half; the FP16 post-training-quantisation point of Sec. 5): taken by the FFN, Sparse-MoE and
+ * projection entry points and by sentry_attend_fwd; the FFN pair runs on tcgen05 with fp16 operands, attention
+ * and the projections on the plain-ALU kernels. */
+typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1, SENTRY_F16 = 2 } sentry_dtype;
 
 /* Create / destroy a context bound to CUDA device `device`.  Creation
  * allocates one small device status word; nothing else. */
@@ -402,7 +405,8 @@ typedef struct sentry_ffn_desc {
     int B, T, D, F; /* batch, tokens per sample, d_model, d_ff */
     int k_c;        /* kept channels per list */
     int n_lists;    /* number of kept-channel lists (one per modality subset in use) */
-    int dtype;      /* sentry_dtype of X, W1, W2, Y */
+    int dtype;      /* sentry_dtype of X, W1, W2, Y (F32, BF16 or F16; the 16-bit types with D in
+                       {128,256,384} run on tcgen05, everything else on the plain ALUs) */
 } sentry_ffn_desc;
 
 /*   X [B,T,D]; W1 [D,F]; W2 [F,D]; Y out [B,T,D]

@@ -19,7 +19,7 @@ from . import build as _build
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsentry.so")
 
-SENTRY_F32, SENTRY_BF16 = 0, 1
+SENTRY_F32, SENTRY_BF16, SENTRY_F16 = 0, 1, 2
 STATUS_BIT_TIMEOUT, STATUS_BIT_EMPTY_MASK, STATUS_BIT_BAD_INDEX = 1, 2, 4
 OPT_ATTEND_KERNEL = 1
 ATTEND_AUTO, ATTEND_WARP_MMA, ATTEND_TCGEN05 = 0, 1, 2
@@ -158,6 +158,8 @@ def _dtype_code(t: torch.Tensor) -> int:
         return SENTRY_F32
     if t.dtype == torch.bfloat16:
         return SENTRY_BF16
+    if t.dtype == torch.float16:
+        return SENTRY_F16
     raise ValueError("unsupported dtype %s" % t.dtype)
 
 

@@ -22,7 +22,7 @@ size_t attend_workspace_bytes(const sentry_attend_desc& d) {
 
 int check_attend_desc(const sentry_attend_desc* d) {
     if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
-    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16 && d->dtype != SENTRY_F16) return SENTRY_ERR_INVALID_ARG;
     if (d->score_mode < 0 || d->score_mode > 2) return SENTRY_ERR_INVALID_ARG;
     if (d->B < 1 || d->T < 1 || d->Hq < 1 || d->Hk < 1 || d->k_h < 1 || d->c < 1)
         return SENTRY_ERR_BAD_SHAPE;
@@ -35,7 +35,7 @@ int check_attend_desc(const sentry_attend_desc* d) {
 
 int check_ffn_desc(const sentry_ffn_desc* d) {
     if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
-    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16 && d->dtype != SENTRY_F16) return SENTRY_ERR_INVALID_ARG;
     if (d->B < 1 || d->T < 1 || d->D < 1 || d->F < 1 || d->k_c < 1 || d->n_lists < 1)
         return SENTRY_ERR_BAD_SHAPE;
     if (d->k_c > d->F) return SENTRY_ERR_BAD_SHAPE;
@@ -373,7 +373,7 @@ int sentry_ffn_fwd(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, 
 
 static int check_proj_desc(const sentry_proj_desc* d) {
     if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
-    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16 && d->dtype != SENTRY_F16) return SENTRY_ERR_INVALID_ARG;
     if (d->B < 1 || d->T < 1 || d->D < 1 || d->Hq < 1 || d->Hk < 1 || d->d < 1 || d->k_h < 1) return SENTRY_ERR_BAD_SHAPE;
     if (d->Hq % d->Hk != 0 || d->k_h > d->Hq) return SENTRY_ERR_BAD_SHAPE;
     if (d->Hk > 32 || d->k_h > 64 || d->D > 8192 || d->k_h * d->d > 8192) return SENTRY_ERR_UNSUPPORTED;
@@ -430,7 +430,7 @@ int sentry_project_out(sentry_ctx* ctx, const sentry_proj_desc* desc, const void
 
 static int check_moe_desc(const sentry_moe_desc* d) {
     if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
-    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16 && d->dtype != SENTRY_F16) return SENTRY_ERR_INVALID_ARG;
     if (d->N < 1 || d->D < 1 || d->F < 1 || d->E < 1 || d->top_k < 1 || d->k_c < 1) return SENTRY_ERR_BAD_SHAPE;
     if (d->k_c > d->F) return SENTRY_ERR_BAD_SHAPE;
     if (d->D % 8 != 0 || d->D > 1024 || d->E > 4096 || d->top_k > 64) return SENTRY_ERR_UNSUPPORTED;

@@ -32,8 +32,14 @@ __device__ __forceinline__ void load_row(const T* __restrict__ p, float (&r)[D])
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                r[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
-                r[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                if constexpr (__is_same(T, __half)) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+                    r[8 * i + 2 * j] = f.x;
+                    r[8 * i + 2 * j + 1] = f.y;
+                } else {   // bf16: the upper half of an fp32
+                    r[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+                    r[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                }
             }
         }
     }
@@ -270,11 +276,11 @@ int launch_typed(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
 }  // namespace
 
 int launch_attend_generic(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
-    const bool f32 = a.d.dtype == SENTRY_F32;
+    const bool f32 = a.d.dtype == SENTRY_F32, f16 = a.d.dtype == SENTRY_F16;
     switch (a.d.d) {
-        case 16: return f32 ? launch_typed<float, 16>(ctx, a, st) : launch_typed<__nv_bfloat16, 16>(ctx, a, st);
-        case 32: return f32 ? launch_typed<float, 32>(ctx, a, st) : launch_typed<__nv_bfloat16, 32>(ctx, a, st);
-        case 64: return f32 ? launch_typed<float, 64>(ctx, a, st) : launch_typed<__nv_bfloat16, 64>(ctx, a, st);
+        case 16: return f32 ? launch_typed<float, 16>(ctx, a, st) : f16 ? launch_typed<__half, 16>(ctx, a, st) : launch_typed<__nv_bfloat16, 16>(ctx, a, st);
+        case 32: return f32 ? launch_typed<float, 32>(ctx, a, st) : f16 ? launch_typed<__half, 32>(ctx, a, st) : launch_typed<__nv_bfloat16, 32>(ctx, a, st);
+        case 64: return f32 ? launch_typed<float, 64>(ctx, a, st) : f16 ? launch_typed<__half, 64>(ctx, a, st) : launch_typed<__nv_bfloat16, 64>(ctx, a, st);
         default: return SENTRY_ERR_UNSUPPORTED;
     }
 }

@@ -332,7 +332,7 @@ FfnWs carve(const sentry_ffn_desc& d, int kc_pad, void* ws, size_t bytes, bool w
 }
 
 int kc_pad_for(const sentry_ffn_desc& d) {
-    if (d.dtype == SENTRY_BF16 && ffn_tc_supported(d)) return ffn_tc_kc_pad(d.D, d.k_c);
+    if (ffn_tc_supported(d)) return ffn_tc_kc_pad(d.D, d.k_c);
     return (d.k_c + 7) / 8 * 8;
 }
 
@@ -345,9 +345,11 @@ size_t ffn_workspace_bytes(const sentry_ffn_desc& d) {
 size_t ffn_packed_bytes(const sentry_ffn_desc& d) { return 2 * packed_half_bytes(d, kc_pad_for(d)); }
 
 // The weight gather alone: W1' = W1[:, N], W2' = W2[N, :] for every list into `packed`.
+// (The gather moves elements and writes zeros, no arithmetic: fp16 data goes through the 16-bit
+// instantiation unchanged.)
 int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStream_t st) {
     const sentry_ffn_desc& d = a.d;
-    const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
+    const bool tc = ffn_tc_supported(d);
     const int kc_pad = kc_pad_for(d);
     const size_t per = (size_t)kc_pad * d.D;
     const size_t pack_blocks = tc ? 2 * (size_t)d.n_lists * (kc_pad / 32) * (d.D / 64)
@@ -373,14 +375,14 @@ int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStre
 
 int ffn_kc_pad(const sentry_ffn_desc& d) { return kc_pad_for(d); }
 int ffn_tile_rows(const sentry_ffn_desc& d) {
-    return d.dtype == SENTRY_BF16 && ffn_tc_supported(d) ? kTcTileRows : kGenericTileRows;
+    return ffn_tc_supported(d) ? kTcTileRows : kGenericTileRows;
 }
 
 // The fused pair alone, on a row plan and materialised weights that are already in place.
 int launch_ffn_main(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1p, void* w2p, int kc_pad,
                     int max_tiles, cudaStream_t st) {
     const sentry_ffn_desc& d = a.d;
-    const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
+    const bool tc = ffn_tc_supported(d);
     if (tc) {
         int rc = launch_ffn_tc(ctx, a, plan, w1p, w2p, kc_pad, max_tiles, st);
         if (rc != SENTRY_OK) return rc;
@@ -394,6 +396,13 @@ int launch_ffn_main(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void
             kern<<<max_tiles, kGenericThreads, smem, st>>>((const float*)a.X, (const float*)w1p,
                                                             (const float*)w2p, plan, d.n_lists,
                                                             d.T, d.D, d.k_c, kc_pad, (float*)a.Y);
+        } else if (d.dtype == SENTRY_F16) {
+            auto kern = ffn_generic_kernel<__half>;
+            if (smem > 48 * 1024)
+                SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<max_tiles, kGenericThreads, smem, st>>>(
+                (const __half*)a.X, (const __half*)w1p, (const __half*)w2p,
+                plan, d.n_lists, d.T, d.D, d.k_c, kc_pad, (__half*)a.Y);
         } else {
             auto kern = ffn_generic_kernel<__nv_bfloat16>;
             if (smem > 48 * 1024)
@@ -411,7 +420,7 @@ int launch_ffn_main(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void
 // caller's materialised W1', W2' (launch_ffn_prepack) and only build the row plan.
 int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, const void* packed, cudaStream_t st) {
     const sentry_ffn_desc& d = a.d;
-    const bool tc = d.dtype == SENTRY_BF16 && ffn_tc_supported(d);
+    const bool tc = ffn_tc_supported(d);
     const int kc_pad = kc_pad_for(d);
     FfnWs w = carve(d, kc_pad, ws, ws_bytes, packed == nullptr);
     if (!w.ok) return SENTRY_ERR_WORKSPACE;

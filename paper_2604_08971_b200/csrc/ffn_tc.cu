@@ -126,7 +126,7 @@ __device__ __forceinline__ void cta_teardown(volatile int* abort_flag, unsigned 
     }
 }
 
-template <int D>
+template <int D, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2_256,
               const __grid_constant__ CUtensorMap tm_w2_128, const __nv_bfloat16* __restrict__ X,
@@ -262,8 +262,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         // two issuing warps were summed in an order that changed from run to run (results
         // differed in the last bit).  A second warp that did the waiting and handed the stage
         // number over through shared memory measured slower than the issuer waiting itself.
-        constexpr uint32_t idesc256 = ptx::umma_idesc_bf16(128, 256);
-        constexpr uint32_t idesc128 = ptx::umma_idesc_bf16(128, 128);
+        constexpr uint32_t idesc256 = F16 ? ptx::umma_idesc_f16(128, 256) : ptx::umma_idesc_bf16(128, 256);
+        constexpr uint32_t idesc128 = F16 ? ptx::umma_idesc_f16(128, 128) : ptx::umma_idesc_bf16(128, 128);
         constexpr uint32_t kBlkLo = kBlockBytes >> 4, kStageLo = kStageBytes >> 4;
         const uint32_t tm_h = tmem + C::H_COL0;
         const uint32_t xs_lo = desc_lo(xs), hs_lo = desc_lo(hs), w_lo = desc_lo(wsm);
@@ -451,16 +451,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + ((i ^ (lane & 7)) << 4)),
-                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i]), __uint_as_float(ra[8 * i + 1]))),
-                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i + 2]), __uint_as_float(ra[8 * i + 3]))),
-                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i + 4]), __uint_as_float(ra[8 * i + 5]))),
-                                 "r"(pack_bf16x2(__uint_as_float(ra[8 * i + 6]), __uint_as_float(ra[8 * i + 7])))
+                                 "r"(pack_16x2<F16>(__uint_as_float(ra[8 * i]), __uint_as_float(ra[8 * i + 1]))),
+                                 "r"(pack_16x2<F16>(__uint_as_float(ra[8 * i + 2]), __uint_as_float(ra[8 * i + 3]))),
+                                 "r"(pack_16x2<F16>(__uint_as_float(ra[8 * i + 4]), __uint_as_float(ra[8 * i + 5]))),
+                                 "r"(pack_16x2<F16>(__uint_as_float(ra[8 * i + 6]), __uint_as_float(ra[8 * i + 7])))
                                  : "memory");
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((4 + i) ^ (lane & 7)) << 4)),
-                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i]), __uint_as_float(rb[8 * i + 1]))),
-                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 2]), __uint_as_float(rb[8 * i + 3]))),
-                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 4]), __uint_as_float(rb[8 * i + 5]))),
-                                 "r"(pack_bf16x2(__uint_as_float(rb[8 * i + 6]), __uint_as_float(rb[8 * i + 7])))
+                                 "r"(pack_16x2<F16>(__uint_as_float(rb[8 * i]), __uint_as_float(rb[8 * i + 1]))),
+                                 "r"(pack_16x2<F16>(__uint_as_float(rb[8 * i + 2]), __uint_as_float(rb[8 * i + 3]))),
+                                 "r"(pack_16x2<F16>(__uint_as_float(rb[8 * i + 4]), __uint_as_float(rb[8 * i + 5]))),
+                                 "r"(pack_16x2<F16>(__uint_as_float(rb[8 * i + 6]), __uint_as_float(rb[8 * i + 7])))
                                  : "memory");
                 }
                 __syncwarp();
@@ -510,8 +510,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     uint32_t pk[32];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        pk[i] = gelu_erf_fast_bf16x2(__uint_as_float(h0[2 * i]), __uint_as_float(h0[2 * i + 1]));
-                        pk[16 + i] = gelu_erf_fast_bf16x2(__uint_as_float(h1[2 * i]), __uint_as_float(h1[2 * i + 1]));
+                        pk[i] = gelu_pack_16x2<F16>(__uint_as_float(h0[2 * i]), __uint_as_float(h0[2 * i + 1]));
+                        pk[16 + i] = gelu_pack_16x2<F16>(__uint_as_float(h1[2 * i]), __uint_as_float(h1[2 * i + 1]));
                     }
                     if (!warp_wait(&misc->hs_empty[blk], (g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t hrow = hs + blk * kBlockBytes + row * 128;
@@ -561,7 +561,7 @@ __global__ void __launch_bounds__(128, 1) wait_expiry_selftest_kernel(long long 
     cta_teardown(abort_flag, status, tmem, 32);
 }
 
-template <int D>
+template <int D, bool F16>
 int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c, int kc_pad,
              int max_tiles, cudaStream_t st) {
     const sentry_ffn_desc& d = a.d;
@@ -570,7 +570,7 @@ int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, 
     if (!make_weight_map(&m1, w1c, r1, D, Cfg<D>::CH == 256 ? 256 : 128)) return SENTRY_ERR_CUDA;
     if (!make_weight_map(&m2a, w2c, r2, kc_pad, D >= 256 ? 256 : 128)) return SENTRY_ERR_CUDA;
     if (!make_weight_map(&m2b, w2c, r2, kc_pad, 128)) return SENTRY_ERR_CUDA;
-    auto kern = ffn_tc_kernel<D>;
+    auto kern = ffn_tc_kernel<D, F16>;
     SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::SMEM_BYTES));
     int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;
     if (grid < 1) grid = 1;
@@ -583,7 +583,7 @@ int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, 
 }  // namespace
 
 bool ffn_tc_supported(const sentry_ffn_desc& d) {
-    return d.dtype == SENTRY_BF16 && (d.D == 128 || d.D == 256 || d.D == 384);
+    return (d.dtype == SENTRY_BF16 || d.dtype == SENTRY_F16) && (d.D == 128 || d.D == 256 || d.D == 384);
 }
 
 // kept channels are padded with zero columns / rows to a whole number of chunks
@@ -601,10 +601,16 @@ int launch_wait_expiry_selftest(sentry_ctx* ctx, long long limit_cycles, cudaStr
 int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,
                   int kc_pad, int max_tiles, cudaStream_t st) {
     int rc;
+    // the two 16-bit types share everything but the operand format of the UMMAs and the roundings
+    // (X, Y and the weight tiles are moved as 16-bit words)
+    const bool f16 = a.d.dtype == SENTRY_F16;
     switch (a.d.D) {
-        case 128: rc = launch_d<128>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
-        case 256: rc = launch_d<256>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
-        case 384: rc = launch_d<384>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
+        case 128: rc = f16 ? launch_d<128, true>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)
+                           : launch_d<128, false>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
+        case 256: rc = f16 ? launch_d<256, true>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)
+                           : launch_d<256, false>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
+        case 384: rc = f16 ? launch_d<384, true>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)
+                           : launch_d<384, false>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st); break;
         default: return SENTRY_ERR_UNSUPPORTED;
     }
     if (rc != SENTRY_OK) return rc;

@@ -95,6 +95,7 @@ moe_offsets_kernel(const int32_t* __restrict__ counts, int E, int tile_rows, Ffn
 template <typename T> struct Vec16;
 template <> struct Vec16<float> { static constexpr int N = 4; };
 template <> struct Vec16<__nv_bfloat16> { static constexpr int N = 8; };
+template <> struct Vec16<__half> { static constexpr int N = 8; };
 
 __device__ __forceinline__ void unpack16(const uint4& v, float (&f)[4]) {
     f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
@@ -121,6 +122,25 @@ __device__ __forceinline__ uint4 pack16(const float (&f)[8]) {
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+__device__ __forceinline__ void unpack16_half(const uint4& v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        f[2 * i] = p.x;
+        f[2 * i + 1] = p.y;
+    }
+}
+__device__ __forceinline__ uint4 pack16_half(const float (&f)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __half2 p = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
+        w[i] = *reinterpret_cast<const uint32_t*>(&p);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // y_t = sum_j weight[t][j] * staged[t*top_k + j]  over the routed slots, 16 bytes per thread.
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -128,6 +148,7 @@ moe_combine_kernel(const uint4* __restrict__ staged, const int32_t* __restrict__
                    const float* __restrict__ weights, long long N, int vpr, int E, int top_k,
                    uint4* __restrict__ Y) {
     constexpr int NV = Vec16<T>::N;
+    constexpr bool IS_BF16 = sizeof(T) == 2 && Vec16<T>::N == 8 && __is_same(T, __nv_bfloat16);
     const long long total = N * vpr;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -141,11 +162,14 @@ moe_combine_kernel(const uint4* __restrict__ staged, const int32_t* __restrict__
             if (e < 0 || e >= E) continue;
             const float g = weights[t * top_k + j];
             float f[NV];
-            unpack16(__ldg(&staged[(t * top_k + j) * vpr + v]), f);
+            const uint4 raw = __ldg(&staged[(t * top_k + j) * vpr + v]);
+            if constexpr (sizeof(T) == 2 && !IS_BF16) unpack16_half(raw, f);
+            else unpack16(raw, f);
 #pragma unroll
             for (int c = 0; c < NV; ++c) acc[c] = fmaf(g, f[c], acc[c]);
         }
-        Y[i] = pack16(acc);
+        if constexpr (sizeof(T) == 2 && !IS_BF16) Y[i] = pack16_half(acc);
+        else Y[i] = pack16(acc);
     }
 }
 
@@ -249,6 +273,9 @@ int launch_moe_ffn(sentry_ctx* ctx, const MoeArgs& m, void* ws, size_t ws_bytes,
         LaunchScope ls(ctx, KS_MOE_COMBINE, st);
         if (d.dtype == SENTRY_F32)
             moe_combine_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(
+                (const uint4*)w.staged, m.expert_ids, m.expert_weights, d.N, vpr, d.E, d.top_k, (uint4*)m.Y);
+        else if (d.dtype == SENTRY_F16)
+            moe_combine_kernel<__half><<<(unsigned)blocks, 256, 0, st>>>(
                 (const uint4*)w.staged, m.expert_ids, m.expert_weights, d.N, vpr, d.E, d.top_k, (uint4*)m.Y);
         else
             moe_combine_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(

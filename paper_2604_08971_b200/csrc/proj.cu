@@ -100,6 +100,10 @@ int launch_project_qkv_generic(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t 
         project_qkv_kernel<float><<<grid, kProjThreads, smem, st>>>(
             (const float*)a.X, (const float*)a.WQ, (const float*)a.WK, (const float*)a.WV, a.kept_heads, a.ids, a.masks,
             d.T, d.D, d.Hq, d.Hk, d.d, d.k_h, (float*)a.Q, (float*)a.K, (float*)a.V, a.status);
+    else if (d.dtype == SENTRY_F16)
+        project_qkv_kernel<__half><<<grid, kProjThreads, smem, st>>>(
+            (const __half*)a.X, (const __half*)a.WQ, (const __half*)a.WK, (const __half*)a.WV, a.kept_heads, a.ids,
+            a.masks, d.T, d.D, d.Hq, d.Hk, d.d, d.k_h, (__half*)a.Q, (__half*)a.K, (__half*)a.V, a.status);
     else
         project_qkv_kernel<__nv_bfloat16><<<grid, kProjThreads, smem, st>>>(
             (const __nv_bfloat16*)a.X, (const __nv_bfloat16*)a.WQ, (const __nv_bfloat16*)a.WK,
@@ -118,6 +122,10 @@ int launch_project_out_generic(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t 
         project_out_kernel<float><<<grid, kProjThreads, smem, st>>>(
             (const float*)a.A, (const float*)a.WO, a.kept_heads, a.ids, a.masks, d.T, d.D, d.Hq, d.d, d.k_h,
             (float*)a.out, a.status);
+    else if (d.dtype == SENTRY_F16)
+        project_out_kernel<__half><<<grid, kProjThreads, smem, st>>>(
+            (const __half*)a.A, (const __half*)a.WO, a.kept_heads, a.ids, a.masks, d.T, d.D, d.Hq, d.d, d.k_h,
+            (__half*)a.out, a.status);
     else
         project_out_kernel<__nv_bfloat16><<<grid, kProjThreads, smem, st>>>(
             (const __nv_bfloat16*)a.A, (const __nv_bfloat16*)a.WO, a.kept_heads, a.ids, a.masks, d.T, d.D, d.Hq, d.d,

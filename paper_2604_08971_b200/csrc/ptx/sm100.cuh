@@ -206,6 +206,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// The same with fp16 operands (format code 0 for A and B; both operands of one UMMA have the same type).
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N) {
+    return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
 // Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes
 // (64 bf16) with the 128-byte swizzle (16-byte chunk index XOR row-within-8), 8-row groups
 // 1024 bytes apart; the tile base must be 1024-byte aligned.

@@ -50,6 +50,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// Two floats -> one 32-bit pair of the storage type (low half = a): bf16, or IEEE half when F16.
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_16x2(float a, float b) {
+    if constexpr (F16) {
+        const __half2 v = __floats2half2_rn(a, b);
+        return *reinterpret_cast<const uint32_t*>(&v);
+    } else {
+        return pack_bf16x2(a, b);
+    }
+}
+// gelu of a pair, rounded to the storage type.  The half form keeps the erf of the math library:
+// the tanh form's 1.5e-4 relative error is of the size of half's own rounding (2.4e-4).
+template <bool F16>
+__device__ __forceinline__ uint32_t gelu_pack_16x2(float z0, float z1) {
+    if constexpr (F16) {
+        const float g0 = 0.5f * z0 * (1.0f + erff(z0 * 0.70710678118654752440f));
+        const float g1 = 0.5f * z1 * (1.0f + erff(z1 * 0.70710678118654752440f));
+        return pack_16x2<true>(g0, g1);
+    } else {
+        return gelu_erf_fast_bf16x2(z0, z1);
+    }
+}
 
 __device__ __forceinline__ void cp_async_wait_pending(int n) {
     if (n <= 0) ptx::cp_async_wait_group<0>();

@@ -108,7 +108,7 @@ def by_name(name: str) -> Workload:
 
 
 def torch_dtype(w: Workload):
-    return torch.float32 if w.dtype == "f32" else torch.bfloat16
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[w.dtype]
 
 
 def token_modality_ids(w: Workload) -> np.ndarray:
@@ -280,7 +280,7 @@ def generate_moe(N: int, D: int, F: int, E: int, top_k: int, k_c: int, dtype: st
     if unrouted > 0.0:
         expert_ids[rng.random((N, top_k)) < unrouted] = -1
     kept = np.stack([np.sort(rng.permutation(F)[:k_c]) for _ in range(E)]).astype(np.int32)
-    dt = torch.float32 if dtype == "f32" else torch.bfloat16
+    dt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[dtype]
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
     normal = lambda shape, std: (torch.randn(shape, generator=gen, device=device, dtype=torch.float32) * std).to(dt)

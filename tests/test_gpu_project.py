@@ -25,6 +25,7 @@ def _weights(w, seed):
 
 
 @pytest.mark.parametrize("w", [synth.config1(), synth.config4().with_(B=6), synth.config2().with_(B=9),
+                               synth.config2().with_(B=4, dtype="f16", name="cfg2_f16_proj"),
                                synth.Workload("ragged_p", "bf16", 5, (37, 5, 91), 72, 6, 3, 16, 200, 4, 77, "cycle7", 71)],
                          ids=lambda w: w.name)
 def test_projections_and_chained_layer(w):
@@ -33,7 +34,7 @@ def test_projections_and_chained_layer(w):
         inp = synth.generate(w, n_s_of)
         kept_h, _ = parity.gate_lists(sn, inp)
         WQ, WK, WV, WO = _weights(w, w.seed + 5)
-        X = inp.X if w.dtype == "f32" else (inp.X.float() * 1.0).to(torch.bfloat16)
+        X = inp.X
         ids, masks = dev(inp.ids), masks_dev(inp.masks)
         dt = synth.torch_dtype(w)
         sentinel = 7.0
