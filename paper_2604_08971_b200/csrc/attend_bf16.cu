@@ -629,6 +629,8 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     // heaviest first (every CTA finds the sample of its rank by itself with a counting sort on
     // the number of present modalities), so that the long ones do not end up alone in the tail
     // of the launch.
+    __shared__ int s_fill_next;
+    if (threadIdx.x == 0) s_fill_next = 0;
     int b = blockIdx.x / Hk;
     const int g = blockIdx.x % Hk;
     const int Bn = gridDim.x / Hk;
@@ -796,6 +798,7 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
             s_mean[threadIdx.x] = __float2bfloat16_rn(t / (float)Tv);
         }
     }
+    __syncthreads();   // s_mean is complete: warps without a row tile go straight to the fill
 
     // ---- Eq. 6 on the active rows: row tiles (head slot, 16 rows) over the warps
     const int WT = (min(U, kMaxActive) + 15) / 16;
@@ -930,16 +933,37 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
                 orow[n * 4 + tq] = pack2(acc[n][2 * h2] * inv, acc[n][2 * h2 + 1] * inv);
         }
     }
-    __syncthreads();   // s_mean is complete
-    // ---- context rows and zero rows, 16 bytes per store
+    // ---- context rows and zero rows, 16 bytes per store, in units of (head, 32 tokens) handed out
+    // from a shared counter: the warps that had no row tile above take most of them
     const uint4* mean4 = reinterpret_cast<const uint4*>(s_mean);
-    for (int hh = 0; hh < rk; ++hh) {
-        uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D);
-        const uint32_t* bits = s_abits + hh * words;
-        for (int i = threadIdx.x; i < Tlen * S::CPR; i += blockDim.x) {
-            const int t = i / S::CPR, cc = i % S::CPR;
-            if ((bits[t >> 5] >> (t & 31)) & 1u) continue;
-            dst[i] = s_kind[t] ? mean4[cc] : make_uint4(0, 0, 0, 0);
+    if (nwarps <= n_tiles) {
+        // every warp had a row tile: they arrive together, a fixed split is cheaper than the counter
+        for (int hh = 0; hh < rk; ++hh) {
+            uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D);
+            const uint32_t* bits = s_abits + hh * words;
+            for (int i = threadIdx.x; i < Tlen * S::CPR; i += blockDim.x) {
+                const int t = i / S::CPR, cc = i % S::CPR;
+                if ((bits[t >> 5] >> (t & 31)) & 1u) continue;
+                dst[i] = s_kind[t] ? mean4[cc] : make_uint4(0, 0, 0, 0);
+            }
+        }
+        return;
+    }
+    const int blocks_per_head = (Tlen + 31) / 32;
+    const int n_units = rk * blocks_per_head;
+    for (;;) {
+        int u = 0;
+        if (lane == 0) u = atomicAdd(&s_fill_next, 1);
+        u = __shfl_sync(0xffffffffu, u, 0);
+        if (u >= n_units) break;
+        const int hh = u / blocks_per_head, t0 = (u % blocks_per_head) * 32;
+        uint4* dst = reinterpret_cast<uint4*>(O + ((size_t)b * k_h + khs[hh]) * Tlen * D) + (size_t)t0 * S::CPR;
+        const uint32_t abits = s_abits[hh * words + (t0 >> 5)];
+#pragma unroll
+        for (int i = lane; i < 32 * S::CPR; i += 32) {
+            const int tl = i / S::CPR, cc = i % S::CPR;
+            if (t0 + tl >= Tlen || ((abits >> tl) & 1u)) continue;
+            dst[i] = s_kind[t0 + tl] ? mean4[cc] : make_uint4(0, 0, 0, 0);
         }
     }
 }
