@@ -36,6 +36,7 @@ L2_BYTES = 126 * 1024 * 1024
 TABLE_LAYOUT = "auto"   # set from --table-layout
 GATE_MULTI = False        # set from --gate-multi
 LONG_SELECT = 0           # set from --long-select (SENTRY_OPT_LONG_SELECT)
+SEPARATE_GATE = False     # set from --separate-gate
 # fp32 FMA peak of the plain ALUs: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (unit counts and max SM clock)
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
@@ -367,12 +368,18 @@ class Workbench:
             self.branch.wait_stream(cur)
             with torch.cuda.stream(self.branch):
                 n += self.ffn_branch(s, self.sn2, gated=multi)
-        if not multi:
-            sn.gate_select(self.sh, self.masks, w.k_h, kept=s.kept_h)
+        if not multi and not SEPARATE_GATE:
+            # head selection and attention in one call (one launch where K and V of a group fit in shared memory)
+            sn.gate_attend_fwd(self.sh, w.k_h, s.Q, s.K, s.V, self.ids, self.masks, self.tbl, self.offs, c=w.c,
+                               score_mode=self.score_mode, O=s.O, kept_heads=s.kept_h)
             n += sn.last_launch_count()
-        sn.attend_fwd(s.Q, s.K, s.V, s.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s.O,
-                      score_mode=self.score_mode)
-        n += sn.last_launch_count()
+        else:
+            if not multi:
+                sn.gate_select(self.sh, self.masks, w.k_h, kept=s.kept_h)
+                n += sn.last_launch_count()
+            sn.attend_fwd(s.Q, s.K, s.V, s.kept_h, self.ids, self.masks, self.tbl, self.offs, c=w.c, O=s.O,
+                          score_mode=self.score_mode)
+            n += sn.last_launch_count()
         if two:
             torch.cuda.current_stream().wait_stream(self.branch)
         else:
@@ -621,9 +628,8 @@ def run_ours(args, w: synth.Workload):
         for i in range(n_chunks):
             b0, b1 = bounds[i], bounds[i + 1]
             cur.wait_event(ups[i])
-            sn.gate_select(sh, masks[b0:b1], w.k_h, kept=base.kept_h[b0:b1])
-            sn.attend_fwd(base.Q[b0:b1], base.K[b0:b1], base.V[b0:b1], base.kept_h[b0:b1], ids, masks[b0:b1],
-                          tbl, offs, c=w.c, O=base.O[b0:b1], score_mode=wb.score_mode)
+            sn.gate_attend_fwd(sh, w.k_h, base.Q[b0:b1], base.K[b0:b1], base.V[b0:b1], ids, masks[b0:b1], tbl, offs, c=w.c,
+                               score_mode=wb.score_mode, O=base.O[b0:b1], kept_heads=base.kept_h[b0:b1])
             sn.gate_select(sc, subsets, w.k_c, kept=kept_c_e2e)
             sn.ffn_fwd(base.X[b0:b1], W1, W2, kept_c_e2e, los[b0:b1], ids, masks[b0:b1], Y=base.Y[b0:b1])
             ev = torch.cuda.Event()
@@ -728,7 +734,9 @@ def run_ours(args, w: synth.Workload):
                                            "entry": "entry-major (score_mode 2), transposed once outside the timed region",
                                            "query": "query-major (score_mode 0)"}[wb.table_layout],
                    "step_includes": "gate selection for heads and channels, attention, FFN weight gather and FFN, "
-                                    "every step (see materialised_once for the weights gathered once)",
+                                    "every step (see materialised_once for the weights gathered once); heads are selected "
+                                    + ("by a launch of their own" if args.separate_gate or args.gate_multi else
+                                       "through sentry_gate_attend_fwd (inside the attention launch where K/V of a group fit in shared memory)"),
                    "timing": "median of %d blocks of %d steps, each block bracketed by barrier + synchronise "
                              "and timed with CUDA events" % (args.replays, args.steps)},
         "block_ms": blocks, "replays": args.replays,
@@ -766,6 +774,8 @@ def main():
                     help="SENTRY_OPT_ATTEND_KERNEL for the attention call")
     ap.add_argument("--long-select", default="auto", choices=["auto", "query-blocks", "per-group"],
                     help="SENTRY_OPT_LONG_SELECT: form of the score + selection step for sequences whose K/V do not fit in shared memory")
+    ap.add_argument("--separate-gate", action="store_true",
+                    help="sentry_gate_select + sentry_attend_fwd instead of sentry_gate_attend_fwd")
     ap.add_argument("--gate-multi", action="store_true",
                     help="select heads and channels with one sentry_gate_select_multi launch ahead of the fork")
     ap.add_argument("--table-layout", default="auto", choices=["auto", "arranged", "entry", "query"],
@@ -775,7 +785,8 @@ def main():
                          "the sampled sets are the same")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
-    global TABLE_LAYOUT, GATE_MULTI, LONG_SELECT
+    global TABLE_LAYOUT, GATE_MULTI, LONG_SELECT, SEPARATE_GATE
+    SEPARATE_GATE = args.separate_gate
     LONG_SELECT = {"auto": 0, "query-blocks": 1, "per-group": 2}[args.long_select]
     TABLE_LAYOUT = args.table_layout
     GATE_MULTI = args.gate_multi

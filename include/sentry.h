@@ -245,6 +245,25 @@ SENTRY_API int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc
                       int n_subsets, void* O, int32_t* active_out,
                       const int32_t* active_in, void* stream);
 
+/* SentryGate's head selection and SentryAttend in one call: the kept heads of
+ * every sample are the k_h best of row masks[b] of head_scores [S, Hq] fp32
+ * (the rule of sentry_gate_select: score descending, equal scores -> lower
+ * index, NaN below every number; ascending output) and attention runs on them.
+ * kept_heads_out [B,k_h] i32 receives the lists (O's head axis follows them).
+ * Where K and V of a group fit in shared memory (bf16, Hq <= 64) and the batch
+ * is at most a few waves of CTAs (B*Hk <= 8 x the SM count) the attention
+ * kernel selects the heads itself -- one launch instead of two, which is what
+ * the short workloads' step time is made of; otherwise this is
+ * sentry_gate_select followed by sentry_attend_fwd.  A mask >= S is flagged
+ * BAD_INDEX (the one-launch form then uses row 0 for that sample, the
+ * two-launch form leaves its list unwritten).  No forced selection here. */
+SENTRY_API int sentry_gate_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc,
+                           const float* head_scores, int S, const void* Q, const void* K,
+                           const void* V, const int32_t* token_modality_ids,
+                           const uint32_t* masks, const int32_t* sample_table,
+                           const int64_t* sample_offsets, int n_subsets, void* O,
+                           int32_t* kept_heads_out, int32_t* active_out, void* stream);
+
 /* Preparation of the sample tables for score_mode 2, once per set of tables
  * (Sec. 4.4 fixes WHICH keys a query is scored on, not the order they are
  * visited in).  Reads the tables as score_mode 0 takes them ([T_v, U] per

@@ -33,7 +33,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
            "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
            "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out",
-           "sentry_gate_select_multi", "sentry_sample_table_arrange", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
+           "sentry_gate_select_multi", "sentry_sample_table_arrange", "sentry_gate_attend_fwd", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
 
 
 class AttendDesc(ctypes.Structure):
@@ -109,6 +109,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_gate_select_multi.argtypes = [vp, ci, ctypes.POINTER(GateSet), ci, vp]
+    lib.sentry_gate_attend_fwd.argtypes = [vp, ctypes.POINTER(AttendDesc), vp, ci, vp, vp, vp, vp, vp, vp, vp, ci, vp, vp, vp, vp]
     lib.sentry_sample_table_arrange.argtypes = [vp, ci, ci, vp, vp, vp, ci, vp, vp]
     lib.sentry_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeDesc)]
     lib.sentry_moe_workspace_bytes.restype = ctypes.c_size_t
@@ -305,6 +306,27 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_gate_select_multi")
         return outs
+
+    def gate_attend_fwd(self, head_scores, k_h: int, Q, K, V, token_modality_ids, masks, sample_table=None,
+                        sample_offsets=None, *, c: int = 5, score_mode: int = 0, O=None, kept_heads=None,
+                        active_out=None):
+        """sentry_gate_attend_fwd: head selection + attention.  Returns (O [B,k_h,T,d], kept_heads [B,k_h])."""
+        desc = self.attend_desc(Q, K, k_h, c, score_mode)
+        B, _, T, d = Q.shape
+        if O is None:
+            O = torch.empty((B, k_h, T, d), dtype=Q.dtype, device=Q.device)
+        if kept_heads is None:
+            kept_heads = torch.empty((B, k_h), dtype=torch.int32, device=Q.device)
+        S = head_scores.shape[0]
+        self.ensure_workspace(max(self.workspace_bytes(attend=desc), S * k_h * 4 + S * 4 + 1024))
+        n_subsets = 0 if sample_offsets is None else sample_offsets.shape[0]
+        rc = self.lib.sentry_gate_attend_fwd(self.h, ctypes.byref(desc), _ptr(head_scores), S, _ptr(Q), _ptr(K), _ptr(V),
+                                             _ptr(token_modality_ids), _ptr(masks), _ptr(sample_table),
+                                             _ptr(sample_offsets), n_subsets, _ptr(O), _ptr(kept_heads),
+                                             _ptr(active_out), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_gate_attend_fwd")
+        return O, kept_heads
 
     def sample_table_arrange(self, token_modality_ids, sample_table, sample_offsets, c: int = 5, out=None):
         """sentry_sample_table_arrange: the tables for score_mode 2 (entry-major, bank-friendly order)."""

@@ -271,12 +271,14 @@ int sentry_gate_layer_counts(sentry_ctx* ctx, const int32_t* kept, int n_masks, 
     return launch_layer_counts(ctx, kept, n_masks, k, layer_offsets, n_layers, counts, (cudaStream_t)stream);
 }
 
-int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const void* Q,
-                      const void* K, const void* V, const int32_t* kept_heads,
-                      const int32_t* token_modality_ids, const uint32_t* masks,
-                      const int32_t* sample_table, const int64_t* sample_offsets,
-                      int n_subsets, void* O, int32_t* active_out, const int32_t* active_in,
-                      void* stream) {
+// Body of sentry_attend_fwd and sentry_gate_attend_fwd.  gate_scores != null: the kept heads are
+// selected from that table (into kept_heads, which is then an output) instead of being given.
+static int attend_body(sentry_ctx* ctx, const sentry_attend_desc* desc, const void* Q,
+                       const void* K, const void* V, int32_t* kept_heads,
+                       const int32_t* token_modality_ids, const uint32_t* masks,
+                       const int32_t* sample_table, const int64_t* sample_offsets,
+                       int n_subsets, void* O, int32_t* active_out, const int32_t* active_in,
+                       const float* gate_scores, int gate_S, void* stream) {
     if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
     int rc = check_attend_desc(desc);
     if (rc != SENTRY_OK) return rc;
@@ -291,8 +293,14 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
         if (n_subsets < 1) return SENTRY_ERR_BAD_SHAPE;
         if (!aligned(sample_table, 4) || !aligned(sample_offsets, 8)) return SENTRY_ERR_INVALID_ARG;
     }
+    if (gate_scores != nullptr) {
+        if (!aligned(gate_scores, 4)) return SENTRY_ERR_INVALID_ARG;
+        if (gate_S < 1) return SENTRY_ERR_BAD_SHAPE;
+        if (gate_S > 65536 || desc->Hq > kMaxUnits) return SENTRY_ERR_UNSUPPORTED;
+    }
     ctx->last_launches = 0;
     AttendArgs a;
+    a.gate_scores = nullptr; a.gate_S = 0; a.kept_out = nullptr;
     a.d = *desc;
     a.Q = Q; a.K = K; a.V = V;
     a.kept_heads = kept_heads;
@@ -314,6 +322,24 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
     SENTRY_ON_DEVICE(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
     a.active_out_user = active_out;
+    if (gate_scores != nullptr) {
+        // inside the attention launch where that saves a launch worth saving: up to a few waves of
+        // CTAs (beyond, the selection repeated in every CTA costs more than one small launch: +5 %
+        // on B = 4096)
+        const bool inside = ctx->attend_kernel != SENTRY_ATTEND_TCGEN05 && attend_bf16_gate_fusable(*desc) &&
+                            (long long)desc->B * desc->Hk <= 8LL * ctx->sm_count;
+        if (inside) {   // the fused attention kernel selects the heads itself
+            a.gate_scores = gate_scores; a.gate_S = gate_S; a.kept_out = kept_heads;
+        } else {        // a gate launch first; its scratch rows are dead before the attention kernels start
+            WsAlloc g(ctx->workspace, ctx->workspace_bytes);
+            int32_t* rows = g.take<int32_t>((size_t)gate_S * desc->k_h);
+            uint32_t* groups = g.take<uint32_t>((size_t)gate_S);
+            if (!g.ok) return SENTRY_ERR_WORKSPACE;
+            rc = launch_gate_select(ctx, gate_scores, gate_S, desc->Hq, masks, desc->B, desc->k_h, kept_heads, nullptr, 0,
+                                    rows, groups, st);
+            if (rc != SENTRY_OK) return rc;
+        }
+    }
     // AUTO takes the kernel that measured faster for the shape: at present the warp-MMA kernels
     // on every shape they support (the tcgen05 kernel is within 10-20 % on T >= 512)
     if (ctx->attend_kernel == SENTRY_ATTEND_TCGEN05 && attend_tc_supported(*desc)) rc = launch_attend_tc(ctx, a, st);
@@ -325,6 +351,25 @@ int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const voi
                                         cudaMemcpyDeviceToDevice, st));
     }
     return SENTRY_OK;
+}
+
+int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const void* Q,
+                      const void* K, const void* V, const int32_t* kept_heads,
+                      const int32_t* token_modality_ids, const uint32_t* masks,
+                      const int32_t* sample_table, const int64_t* sample_offsets,
+                      int n_subsets, void* O, int32_t* active_out, const int32_t* active_in,
+                      void* stream) {
+    return attend_body(ctx, desc, Q, K, V, const_cast<int32_t*>(kept_heads), token_modality_ids, masks, sample_table,
+                       sample_offsets, n_subsets, O, active_out, active_in, nullptr, 0, stream);
+}
+
+int sentry_gate_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc, const float* head_scores, int S,
+                           const void* Q, const void* K, const void* V, const int32_t* token_modality_ids,
+                           const uint32_t* masks, const int32_t* sample_table, const int64_t* sample_offsets,
+                           int n_subsets, void* O, int32_t* kept_heads_out, int32_t* active_out, void* stream) {
+    if (head_scores == nullptr || kept_heads_out == nullptr) return SENTRY_ERR_INVALID_ARG;
+    return attend_body(ctx, desc, Q, K, V, kept_heads_out, token_modality_ids, masks, sample_table, sample_offsets,
+                       n_subsets, O, active_out, nullptr, head_scores, S, stream);
 }
 
 int sentry_sample_table_arrange(sentry_ctx* ctx, int T, int c, const int32_t* token_modality_ids,

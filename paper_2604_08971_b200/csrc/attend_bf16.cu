@@ -603,13 +603,15 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
                          const int32_t* __restrict__ table, const int64_t* __restrict__ offsets,
                          int n_subsets, const int32_t* __restrict__ active_in,
                          int32_t* __restrict__ active_out, int Tlen, int Hq, int Hk, int k_h, int c,
-                         int score_mode, int U_max, __nv_bfloat16* __restrict__ O, unsigned int* status) {
+                         int score_mode, int U_max, __nv_bfloat16* __restrict__ O, unsigned int* status,
+                         const float* __restrict__ gate_scores, int gate_S, int32_t* __restrict__ kept_out) {
     using S = Sw<D>;
     constexpr int NT = D / 8;        // n-tiles of the output (8 dims each)
     constexpr int KS = D / 16;       // k-steps of q.k
     constexpr int TILE_BYTES = kKeyTile * D * 2;
     extern __shared__ __align__(128) uint8_t s_raw[];
     __shared__ int red[66];
+    __shared__ int32_t s_kept[64];
     __shared__ int32_t s_act[kMaxRK][kMaxActive];
     __shared__ float s_vpart[512 / (D / 2)][D];
     __shared__ __align__(16) __nv_bfloat16 s_mean[D];
@@ -672,9 +674,37 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const uint32_t mask = masks[b];
     const int Tv = block_build_valid(ids, Tlen, mask, s_valid, red);
+    const int32_t* kept_row = kept_heads + (size_t)b * k_h;
+    if (gate_scores != nullptr) {
+        // SentryGate's head selection for this sample's mask, done here instead of by a launch of
+        // its own: the k_h best of the Hq <= 64 scores of row `mask` (score descending, equal
+        // scores -> lower index, NaN below every number), ascending.  Every CTA of the sample
+        // computes the same list; the CTA of group 0 leaves it in kept_out.
+        if (warp == 0) {
+            uint32_t row = mask;
+            if (row >= (uint32_t)gate_S) { if (lane == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX); row = 0; }
+            const float* sr = gate_scores + (size_t)row * Hq;
+            const uint32_t k0 = lane < Hq ? sentry_order_key(sr[lane]) : 0u;
+            const uint32_t k1 = lane + 32 < Hq ? sentry_order_key(sr[lane + 32]) : 0u;
+            int r0 = 0, r1 = 0;
+            for (int j = 0; j < Hq; ++j) {
+                const uint32_t kj = __shfl_sync(0xffffffffu, j < 32 ? k0 : k1, j & 31);
+                r0 += (kj > k0 || (kj == k0 && j < lane)) ? 1 : 0;
+                r1 += (kj > k1 || (kj == k1 && j < lane + 32)) ? 1 : 0;
+            }
+            const bool keep0 = lane < Hq && r0 < k_h, keep1 = lane + 32 < Hq && r1 < k_h;
+            const unsigned b0 = __ballot_sync(0xffffffffu, keep0), b1 = __ballot_sync(0xffffffffu, keep1);
+            const unsigned lt = (1u << lane) - 1u;
+            if (keep0) s_kept[__popc(b0 & lt)] = lane;
+            if (keep1) s_kept[__popc(b0) + __popc(b1 & lt)] = lane + 32;
+        }
+        __syncthreads();
+        if (g == 0 && kept_out != nullptr && (int)threadIdx.x < k_h) kept_out[(size_t)b * k_h + threadIdx.x] = s_kept[threadIdx.x];
+        kept_row = s_kept;
+    }
     int hs[kMaxRK], khs[kMaxRK];
     bool bad;
-    const int rk = group_heads(kept_heads + (size_t)b * k_h, k_h, Hq / Hk, g, Hq, hs, khs, bad);
+    const int rk = group_heads(kept_row, k_h, Hq / Hk, g, Hq, hs, khs, bad);
     if (bad && threadIdx.x == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
     if (rk == 0) return;
     if (Tv == 0) {  // no modality present: zero rows, flag
@@ -994,10 +1024,12 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
             (const __nv_bfloat16*)a.Q, (const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, a.kept_heads,
             a.ids, a.masks, a.sample_table, a.sample_offsets, a.n_subsets,
             a.selection_given ? a.active : nullptr, a.selection_given ? nullptr : a.active_out_user, d.T,
-            d.Hq, d.Hk, d.k_h, d.c, d.score_mode, a.U_max, (__nv_bfloat16*)a.O, a.status);
+            d.Hq, d.Hk, d.k_h, d.c, d.score_mode, a.U_max, (__nv_bfloat16*)a.O, a.status, a.gate_scores, a.gate_S,
+            a.kept_out);
         SENTRY_CUDA_TRY(cudaGetLastError());
         return SENTRY_OK;
     }
+    if (a.gate_scores != nullptr) return SENTRY_ERR_UNSUPPORTED;   // the caller checks attend_bf16_gate_fusable
     const size_t valid_bytes = (((size_t)d.T * 2 + 127) / 128) * 128;
     // scores and selection by one CTA per group with K resident, where the shape allows it; the
     // streamed kernel then takes the active lists as given
@@ -1056,6 +1088,18 @@ bool attend_bf16_supported(const sentry_attend_desc& d) {
     if (sentry_num_active(d.T, d.c) > kMaxActive) return false;
     if (d.T > 8192) return false;
     return d.d == 16 || d.d == 32 || d.d == 64;
+}
+
+// Whether the head selection can ride inside the attention launch: the fused kernel (K and V of a
+// group resident in shared memory) with at most 64 heads.
+bool attend_bf16_gate_fusable(const sentry_attend_desc& d) {
+    if (!attend_bf16_supported(d) || d.Hq > 64 || d.k_h > 64) return false;
+    switch (d.d) {
+        case 16: return fused_smem_bytes<16>(d.T) <= 200 * 1024;
+        case 32: return fused_smem_bytes<32>(d.T) <= 200 * 1024;
+        case 64: return fused_smem_bytes<64>(d.T) <= 200 * 1024;
+        default: return false;
+    }
 }
 
 int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {

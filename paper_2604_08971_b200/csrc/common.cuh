@@ -333,6 +333,10 @@ struct AttendArgs {
     float* mscore;          // workspace [B,k_h,T]
     int U_max;
     unsigned int* status;
+    // head selection inside the attention launch (null: kept_heads is given)
+    const float* gate_scores;   // [gate_S, Hq] score table of the heads
+    int gate_S;
+    int32_t* kept_out;          // [B,k_h] where the kernel leaves the lists it selected
 };
 int launch_attend_generic(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_tc_supported(const sentry_attend_desc& d);
@@ -342,6 +346,7 @@ bool attend_long_select_supported(const sentry_attend_desc& d);
 int launch_attend_long_select(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 int launch_attend_tc(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_bf16_supported(const sentry_attend_desc& d);
+bool attend_bf16_gate_fusable(const sentry_attend_desc& d);
 int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 
 struct ProjArgs {

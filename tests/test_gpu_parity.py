@@ -256,6 +256,41 @@ def test_arranged_sample_tables_keep_the_sets_and_the_parity(sn, w):
         sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_AUTO)
 
 
+@pytest.mark.parametrize("w,kernel", [
+    (synth.config2().with_(B=24), sentry.ATTEND_AUTO),       # heads selected inside the fused kernel (128-thread CTAs)
+    (synth.config4().with_(B=20), sentry.ATTEND_AUTO),       # the same, 256-thread CTAs, three subsets
+    (synth.config3().with_(B=3), sentry.ATTEND_AUTO),        # 512-thread CTAs
+    (synth.config4().with_(B=6), sentry.ATTEND_TCGEN05),     # gate launch + tcgen05 kernel
+    (synth.config1(), sentry.ATTEND_AUTO),                   # fp32: gate launch + plain-ALU kernels
+    (synth.Workload("long_ga", "bf16", 4, (1300, 1100, 900), 64, 8, 2, 32, 128, 4, 64, "cycle7", 94), sentry.ATTEND_AUTO),
+], ids=lambda v: v.name if isinstance(v, synth.Workload) else str(v))
+def test_gate_and_attention_in_one_call(sn, w, kernel):
+    """sentry_gate_attend_fwd == sentry_gate_select followed by sentry_attend_fwd, bit for bit:
+    kept-head lists, active lists and output."""
+    inp = synth.generate(w, n_s_of)
+    ids, masks = dev(inp.ids), masks_dev(inp.masks)
+    tbl, offs = dev(inp.sample_table), dev(inp.table_offsets)
+    sh = dev(inp.scores_heads)
+    Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
+    U_max = n_s_of(w.T)
+    sn.set_attend_kernel(kernel)
+    try:
+        kept = sn.gate_select(sh, masks, w.k_h)
+        O1, act1 = sn.attend_fwd(Q, K, V, kept, ids, masks, tbl, offs, c=w.c, return_active=True)
+        act2 = torch.full((w.B, w.k_h, U_max), -7, dtype=torch.int32, device="cuda")
+        O2, kept2 = sn.gate_attend_fwd(sh, w.k_h, Q, K, V, ids, masks, tbl, offs, c=w.c, active_out=act2)
+        launches = sn.last_launch_count()
+    finally:
+        sn.set_attend_kernel(sentry.ATTEND_AUTO)
+    assert sn.last_status() == 0
+    np.testing.assert_array_equal(kept2.cpu().numpy(), oracle.gate_select(inp.scores_heads, inp.masks, w.k_h))
+    assert torch.equal(kept, kept2)
+    assert torch.equal(act1, act2)
+    assert torch.equal(O1, O2)
+    if w.dtype == "bf16" and kernel == sentry.ATTEND_AUTO and w.T <= 1024:
+        assert launches == 1   # B * Hk is far below the bound beyond which the gate gets its own launch
+
+
 # ------------------------------------------------------------------ edge cases
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d", [16, 32, 64])
