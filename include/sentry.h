@@ -62,9 +62,9 @@ typedef enum {
 #define SENTRY_STATUS_BIT_EMPTY_MASK 2u
 #define SENTRY_STATUS_BIT_BAD_INDEX 4u /* a kept index / token id out of range was skipped */
 
-/* SENTRY_F16 (IEEE half; the FP16 post-training-quantisation point of Sec. 5): taken by the FFN, Sparse-MoE and
- * projection entry points and by sentry_attend_fwd; the FFN pair runs on tcgen05 with fp16 operands, attention
- * and the projections on the plain-ALU kernels. */
+/* SENTRY_F16 (IEEE half; the FP16 post-training-quantisation point of Sec. 5): taken by every entry point.  The
+ * FFN pair and the Sparse-MoE block run on tcgen05 with fp16 operands, attention on the warp-MMA kernels with fp16
+ * operands (the tcgen05 attention kernel is bf16 only), the projections on the plain-ALU kernels. */
 typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1, SENTRY_F16 = 2 } sentry_dtype;
 
 /* Create / destroy a context bound to CUDA device `device`.  Creation

@@ -326,7 +326,8 @@ static int attend_body(sentry_ctx* ctx, const sentry_attend_desc* desc, const vo
         // inside the attention launch where that saves a launch worth saving: up to a few waves of
         // CTAs (beyond, the selection repeated in every CTA costs more than one small launch: +5 %
         // on B = 4096)
-        const bool inside = ctx->attend_kernel != SENTRY_ATTEND_TCGEN05 && attend_bf16_gate_fusable(*desc) &&
+        const bool inside = ctx->attend_kernel != SENTRY_ATTEND_TCGEN05 &&
+                            (attend_bf16_gate_fusable(*desc) || attend_f16_gate_fusable(*desc)) &&
                             (long long)desc->B * desc->Hk <= 8LL * ctx->sm_count;
         if (inside) {   // the fused attention kernel selects the heads itself
             a.gate_scores = gate_scores; a.gate_S = gate_S; a.kept_out = kept_heads;
@@ -343,7 +344,9 @@ static int attend_body(sentry_ctx* ctx, const sentry_attend_desc* desc, const vo
     // AUTO takes the kernel that measured faster for the shape: at present the warp-MMA kernels
     // on every shape they support (the tcgen05 kernel is within 10-20 % on T >= 512)
     if (ctx->attend_kernel == SENTRY_ATTEND_TCGEN05 && attend_tc_supported(*desc)) rc = launch_attend_tc(ctx, a, st);
-    else rc = attend_bf16_supported(*desc) ? launch_attend_bf16(ctx, a, st) : launch_attend_generic(ctx, a, st);
+    else rc = attend_bf16_supported(*desc)  ? launch_attend_bf16(ctx, a, st)
+              : attend_f16_supported(*desc) ? launch_attend_f16(ctx, a, st)
+                                            : launch_attend_generic(ctx, a, st);
     if (rc != SENTRY_OK) return rc;
     if (a.selection_given && active_out != nullptr && active_out != active_in) {
         SENTRY_CUDA_TRY(cudaMemcpyAsync(active_out, active_in,

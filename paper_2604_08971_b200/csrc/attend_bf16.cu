@@ -176,7 +176,7 @@ attend_score_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
 // ------------------------------------------------------------------------------------- core
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "mma.sync.aligned.m16n8k16.row.col.f32." ATT_PTX_TYPE "." ATT_PTX_TYPE ".f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
         "{%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -370,8 +370,8 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
         for (int row = vs_k0; row < kKeyTile; row += VS_STRIDE) {
             uint32_t w;
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(vbase + S::off(row, vs_dp >> 2) + (vs_dp & 3) * 4));
-            vsum0 += __uint_as_float(w << 16);
-            vsum1 += __uint_as_float(w & 0xffff0000u);
+            vsum0 += att_lo(w);
+            vsum1 += att_hi(w);
         }
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
@@ -470,7 +470,7 @@ attend_core_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     if (threadIdx.x < D) {
         float t = 0.f;
         for (int i = 0; i < VS_STRIDE; ++i) t += s_vpart[i][threadIdx.x];
-        s_mean[threadIdx.x] = __float2bfloat16_rn(t / (float)Tv);
+        reinterpret_cast<unsigned short*>(s_mean)[threadIdx.x] = att_bits(t / (float)Tv);
     }
     // ---- active rows: normalise and store
 #pragma unroll
@@ -816,8 +816,8 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         for (int row = vs_k0; row < rows_staged; row += stride) {
             uint32_t w;
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(vs_addr + S::off(row, vs_dp >> 2) + (vs_dp & 3) * 4));
-            v0 += __uint_as_float(w << 16);
-            v1 += __uint_as_float(w & 0xffff0000u);
+            v0 += att_lo(w);
+            v1 += att_hi(w);
         }
         s_vpart[vs_k0][2 * vs_dp] = v0;
         s_vpart[vs_k0][2 * vs_dp + 1] = v1;
@@ -825,7 +825,7 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         if (threadIdx.x < D) {
             float t = 0.f;
             for (int i = 0; i < stride; ++i) t += s_vpart[i][threadIdx.x];
-            s_mean[threadIdx.x] = __float2bfloat16_rn(t / (float)Tv);
+            reinterpret_cast<unsigned short*>(s_mean)[threadIdx.x] = att_bits(t / (float)Tv);
         }
     }
     __syncthreads();   // s_mean is complete: warps without a row tile go straight to the fill
@@ -1083,7 +1083,7 @@ int launch_d(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st) {
 
 // bf16, at most 4 query heads per KV group, U <= 48 and shared memory within reach.
 bool attend_bf16_supported(const sentry_attend_desc& d) {
-    if (d.dtype != SENTRY_BF16) return false;
+    if (d.dtype != ATT_DTYPE) return false;
     if (d.Hq / d.Hk > kMaxRK) return false;
     if (sentry_num_active(d.T, d.c) > kMaxActive) return false;
     if (d.T > 8192) return false;

@@ -6,7 +6,42 @@
 #include "common.cuh"
 #include "ptx/sm100.cuh"
 
+// The kernels that include this header exist twice: for bf16 tensors, and -- compiled again with
+// SENTRY_ATT_F16 defined, under other entry-point names (attend_f16.cu, attend_long_f16.cu) -- for
+// IEEE-half tensors.  The two builds differ only in the helpers below: the operand type of the
+// mixed-precision FMA and of the warp MMA, and the 16-bit packing / unpacking.
+#ifdef SENTRY_ATT_F16
+#define ATT_PTX_TYPE "f16"
+#define ATT_DTYPE SENTRY_F16
+#else
+#define ATT_PTX_TYPE "bf16"
+#define ATT_DTYPE SENTRY_BF16
+#endif
+
 namespace {
+
+// Low / high element of a packed 16-bit pair as fp32, and fp32 -> the 16 storage bits.
+__device__ __forceinline__ float att_lo(uint32_t w) {
+#ifdef SENTRY_ATT_F16
+    return __half2float(__ushort_as_half((unsigned short)(w & 0xffffu)));
+#else
+    return __uint_as_float(w << 16);
+#endif
+}
+__device__ __forceinline__ float att_hi(uint32_t w) {
+#ifdef SENTRY_ATT_F16
+    return __half2float(__ushort_as_half((unsigned short)(w >> 16)));
+#else
+    return __uint_as_float(w & 0xffff0000u);
+#endif
+}
+__device__ __forceinline__ unsigned short att_bits(float x) {
+#ifdef SENTRY_ATT_F16
+    return __half_as_ushort(__float2half_rn(x));
+#else
+    return __bfloat16_as_ushort(__float2bfloat16_rn(x));
+#endif
+}
 
 constexpr int kMaxRK = 4;          // kept heads of one KV group handled per CTA
 constexpr int kScoreThreads = 256;
@@ -55,7 +90,7 @@ __device__ __forceinline__ int group_heads(const int32_t* kept, int k_h, int r, 
 __device__ __forceinline__ void fma_bf16_pair(float& acc_lo, float& acc_hi, uint32_t a, uint32_t b) {
     asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
         "mov.b32 {al, ah}, %2;\n\tmov.b32 {bl, bh}, %3;\n\t"
-        "fma.rn.f32.bf16 %0, al, bl, %0;\n\tfma.rn.f32.bf16 %1, ah, bh, %1;\n\t}"
+        "fma.rn.f32." ATT_PTX_TYPE " %0, al, bl, %0;\n\tfma.rn.f32." ATT_PTX_TYPE " %1, ah, bh, %1;\n\t}"
         : "+f"(acc_lo), "+f"(acc_hi)
         : "r"(a), "r"(b));
 }
@@ -93,12 +128,16 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+#ifdef SENTRY_ATT_F16
+    __half2 v = __floats2half2_rn(lo, hi);
+#else
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+#endif
     return *reinterpret_cast<uint32_t*>(&v);
 }
 // bf16 pair of what the packed pair `head` = pack2(lo, hi) leaves of lo and hi
 __device__ __forceinline__ uint32_t pack2_rem(float lo, float hi, uint32_t head) {
-    return pack2(lo - __uint_as_float(head << 16), hi - __uint_as_float(head & 0xffff0000u));
+    return pack2(lo - att_lo(head), hi - att_hi(head));
 }
 
 // Warp-level top-k by radix selection over n order keys in shared memory (larger key first,

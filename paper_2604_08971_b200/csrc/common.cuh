@@ -348,6 +348,12 @@ int launch_attend_tc(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 bool attend_bf16_supported(const sentry_attend_desc& d);
 bool attend_bf16_gate_fusable(const sentry_attend_desc& d);
 int launch_attend_bf16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
+// the same kernels compiled for IEEE-half tensors (attend_f16.cu, attend_long_f16.cu)
+bool attend_long_select_f16_supported(const sentry_attend_desc& d);
+int launch_attend_long_select_f16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
+bool attend_f16_supported(const sentry_attend_desc& d);
+bool attend_f16_gate_fusable(const sentry_attend_desc& d);
+int launch_attend_f16(sentry_ctx* ctx, const AttendArgs& a, cudaStream_t st);
 
 struct ProjArgs {
     sentry_proj_desc d;

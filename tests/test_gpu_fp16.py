@@ -1,6 +1,7 @@
 """IEEE-half storage (the FP16 point of the paper's post-training-quantisation axis, Section 5): the
-pruned FFN pair on tcgen05 with fp16 operands, the Sparse-MoE block on the same kernel, and attention /
-projections on the plain-ALU kernels, each against the float64 oracle fed the same fp16 values."""
+pruned FFN pair on tcgen05 with fp16 operands, the Sparse-MoE block on the same kernel, attention on the
+warp-MMA kernels compiled for fp16 operands, projections on the plain-ALU kernels, each against the
+float64 oracle fed the same fp16 values."""
 import numpy as np
 import pytest
 import torch
@@ -43,17 +44,34 @@ def test_fp16_ffn_and_attention(sn, w):
     packed = sn.ffn_prepack(W1, W2, kept_c)
     Y2 = sn.ffn_fwd_packed(X, packed, w.F, w.k_c, kept_c.shape[0], los, ids, masks)
     assert torch.equal(Y1, Y2)
-    if w.B * w.T <= 4096:   # attention on the plain-ALU kernels: small cases only
-        err_a, _ = parity.attend_parity(sn, inp, kept_h, None, 0, full_batch=True)
-        assert err_a <= TOL["f16"], err_a
-
-
-def test_fp16_attention_small(sn):
-    w = synth.Workload("att_f16", "f16", 4, (40, 24, 33), 64, 8, 2, 32, 128, 5, 64, "cycle7", 49)
-    inp = synth.generate(w, n_s_of)
-    kept_h, _ = parity.gate_lists(sn, inp)
+    # attention: the warp-MMA kernels compiled for fp16 operands
     err_a, _ = parity.attend_parity(sn, inp, kept_h, None, 0, full_batch=True)
     assert err_a <= TOL["f16"], err_a
+
+
+@pytest.mark.parametrize("w", [
+    synth.Workload("att_f16", "f16", 4, (40, 24, 33), 64, 8, 2, 32, 128, 5, 64, "cycle7", 49),
+    synth.Workload("att_f16_d64", "f16", 4, (140, 124, 133), 64, 8, 2, 64, 128, 5, 64, "cycle7", 50),
+    synth.Workload("att_f16_long", "f16", 5, (1300, 1100, 900), 64, 8, 2, 32, 128, 4, 64, "cycle7", 51),   # streamed Eq. 6
+    synth.Workload("att_f16_5heads", "f16", 3, (60, 70), 64, 10, 2, 16, 128, 9, 64, "all", 52),   # 5 heads per group: plain-ALU kernels
+], ids=lambda w: w.name)
+def test_fp16_attention(sn, w):
+    inp = synth.generate(w, n_s_of)
+    kept_h, _ = parity.gate_lists(sn, inp)
+    try:
+        for form in (sentry.LONG_SELECT_PER_GROUP, sentry.LONG_SELECT_QUERY_BLOCKS):
+            sn.set_option(sentry.OPT_LONG_SELECT, form)
+            err_a, _ = parity.attend_parity(sn, inp, kept_h, None, 0, full_batch=True)
+            assert err_a <= TOL["f16"], err_a
+    finally:
+        sn.set_option(sentry.OPT_LONG_SELECT, sentry.LONG_SELECT_AUTO)
+    # heads selected inside the attention launch: same bits as the two-call form
+    ids, masks = dev(inp.ids), masks_dev(inp.masks)
+    tbl, offs = dev(inp.sample_table), dev(inp.table_offsets)
+    Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
+    O1 = sn.attend_fwd(Q, K, V, kept_h, ids, masks, tbl, offs, c=w.c)
+    O2, kept2 = sn.gate_attend_fwd(dev(inp.scores_heads), w.k_h, Q, K, V, ids, masks, tbl, offs, c=w.c)
+    assert torch.equal(kept2, kept_h) and torch.equal(O1, O2)
 
 
 def test_fp16_moe(sn):
