@@ -678,7 +678,7 @@ def run_ours(args, w: synth.Workload):
         fl = wm["kernel_flops"]["ffn_main"]
         by = wm["kernel_bytes"]["ffn_main"]
         t_tensor, t_hbm = fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)
-        if t_tensor >= t_hbm and w.dtype == "bf16":
+        if t_tensor >= t_hbm and w.dtype in ("bf16", "f16"):
             roof = {"bound": "tensor", "achieved": fl / t_launch / 1e12, "peak": peaks["bf16_tflops"],
                     "unit": "TFLOP/s"}
         else:
@@ -701,7 +701,7 @@ def run_ours(args, w: synth.Workload):
     # ---- the other named workloads and the sweep cells, each measured briefly in this same run
     table = {}
     if world == 1 and not args.no_configs:
-        names = ["2", "3a", "3b", "3c", "4"] + ["5:%dx%d" % bt for bt in synth.CONFIG5_CELLS]
+        names = ["2", "3a", "3b", "3c", "4"] + ["5:%dx%d" % bt for bt in synth.CONFIG5_CELLS] + ["3b:f16", "4:f16"]
         for name in names:
             try:
                 table[name] = quick_config(sentry, name, dev, local_rank, peaks, args)

@@ -64,7 +64,7 @@ typedef enum {
 
 /* SENTRY_F16 (IEEE half; the FP16 post-training-quantisation point of Sec. 5): taken by every entry point.  The
  * FFN pair and the Sparse-MoE block run on tcgen05 with fp16 operands, attention on the warp-MMA kernels with fp16
- * operands (the tcgen05 attention kernel is bf16 only), the projections on the plain-ALU kernels. */
+ * operands (the tcgen05 attention kernel is bf16 only), the projections on tcgen05 with fp16 operands. */
 typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1, SENTRY_F16 = 2 } sentry_dtype;
 
 /* Create / destroy a context bound to CUDA device `device`.  Creation

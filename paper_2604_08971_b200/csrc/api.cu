@@ -450,6 +450,7 @@ int sentry_project_qkv(sentry_ctx* ctx, const sentry_proj_desc* desc, const void
     a.Q = Q; a.K = K; a.V = V;
     a.status = ctx->d_status;
     SENTRY_ON_DEVICE(ctx->device);
+    if (project_qkv_tc_f16_supported(*desc)) return launch_project_qkv_tc_f16(ctx, a, (cudaStream_t)stream);
     return project_qkv_tc_supported(*desc) ? launch_project_qkv_tc(ctx, a, (cudaStream_t)stream)
                                            : launch_project_qkv_generic(ctx, a, (cudaStream_t)stream);
 }
@@ -472,6 +473,7 @@ int sentry_project_out(sentry_ctx* ctx, const sentry_proj_desc* desc, const void
     a.out = out;
     a.status = ctx->d_status;
     SENTRY_ON_DEVICE(ctx->device);
+    if (project_out_tc_f16_supported(*desc)) return launch_project_out_tc_f16(ctx, a, (cudaStream_t)stream);
     return project_out_tc_supported(*desc) ? launch_project_out_tc(ctx, a, (cudaStream_t)stream)
                                            : launch_project_out_generic(ctx, a, (cudaStream_t)stream);
 }

@@ -371,6 +371,10 @@ bool project_qkv_tc_supported(const sentry_proj_desc& d);
 bool project_out_tc_supported(const sentry_proj_desc& d);
 int launch_project_qkv_tc(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
 int launch_project_out_tc(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
+bool project_qkv_tc_f16_supported(const sentry_proj_desc& d);   // the same for IEEE-half tensors (proj_tc_f16.cu)
+bool project_out_tc_f16_supported(const sentry_proj_desc& d);
+int launch_project_qkv_tc_f16(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
+int launch_project_out_tc_f16(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st);
 
 struct FfnArgs {
     sentry_ffn_desc d;

@@ -15,6 +15,14 @@
 #include "attend_common.cuh"
 #include "tc_common.cuh"
 
+// Compiled a second time for IEEE-half tensors (proj_tc_f16.cu): the operand format of the UMMAs
+// and the packing of the results (pack2, attend_common.cuh) are what differs.
+#ifdef SENTRY_ATT_F16
+#define PROJ_IDESC ptx::umma_idesc_f16_major
+#else
+#define PROJ_IDESC ptx::umma_idesc_bf16_major
+#endif
+
 namespace {
 
 constexpr int kPThreads = 256;
@@ -128,7 +136,7 @@ proj_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- UMMA issuer
-        constexpr uint32_t idesc = ptx::umma_idesc_bf16_major(128, DH, false, true);
+        constexpr uint32_t idesc = PROJ_IDESC(128, DH, false, true);
         bool ok = true;
         for (int s = 0; s < n_slices && ok; ++s) {
             const uint32_t st = (uint32_t)s % kPStages, use = (uint32_t)s / kPStages;
@@ -307,7 +315,7 @@ proj_out_tc_kernel(const __grid_constant__ CUtensorMap tm_o, const __nv_bfloat16
             __syncwarp();
         }
     } else if (warp == 1) {
-        constexpr uint32_t idesc = ptx::umma_idesc_bf16_major(128, 64, false, true);
+        constexpr uint32_t idesc = PROJ_IDESC(128, 64, false, true);
         bool ok = true;
         for (int s = 0; s < n_slices && ok; ++s) {
             const uint32_t st = (uint32_t)s % kPStages, use = (uint32_t)s / kPStages;
@@ -424,7 +432,7 @@ int launch_qkv_d(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st) {
 // bf16, head dim 16/32/64, d_model a multiple of 64, everything within one SM's shared memory,
 // and one CTA's tile count within the grid limit
 bool project_qkv_tc_supported(const sentry_proj_desc& d) {
-    if (d.dtype != SENTRY_BF16) return false;
+    if (d.dtype != ATT_DTYPE) return false;
     if (d.d != 16 && d.d != 32 && d.d != 64) return false;
     if (d.D % 64 != 0 || d.T > 65535) return false;
     if (d.k_h + 2 * d.Hk > kMaxSlicesTc) return false;
@@ -441,7 +449,7 @@ int launch_project_qkv_tc(sentry_ctx* ctx, const ProjArgs& a, cudaStream_t st) {
 }
 
 bool project_out_tc_supported(const sentry_proj_desc& d) {
-    if (d.dtype != SENTRY_BF16) return false;
+    if (d.dtype != ATT_DTYPE) return false;
     if (d.d != 16 && d.d != 32 && d.d != 64) return false;
     if (d.D % 64 != 0 || d.D > 512 || d.T > 65535 || d.k_h > kMaxSlicesTc) return false;
     return out_smem_bytes(d.D, d.d, d.k_h, d.T) <= 220 * 1024;

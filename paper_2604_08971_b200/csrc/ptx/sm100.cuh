@@ -250,5 +250,8 @@ __device__ __forceinline__ uint64_t umma_smem_desc_rows(uint32_t smem_addr, int 
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_major(int M, int N, bool a_mn_major, bool b_mn_major) {
     return umma_idesc_bf16(M, N) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u);
 }
+__host__ __device__ constexpr uint32_t umma_idesc_f16_major(int M, int N, bool a_mn_major, bool b_mn_major) {
+    return umma_idesc_f16(M, N) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u);
+}
 
 }  // namespace ptx

@@ -29,7 +29,8 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
-__device__ __forceinline__ uint32_t gelu_erf_fast_bf16x2(float z0, float z1) {
+// gelu of a pair by the tanh form above, as two floats
+__device__ __forceinline__ void gelu_erf_fast_x2(float z0, float z1, float& g0, float& g1) {
     const uint64_t Z = f32x2(z0, z1), zero = f32x2(0.f, 0.f);
     const uint64_t Z2 = fma_f32x2(Z, Z, zero);
     const uint64_t P = fma_f32x2(Z2, f32x2(0.03538746f, 0.03538746f), f32x2(0.7985835f, 0.7985835f));
@@ -40,8 +41,11 @@ __device__ __forceinline__ uint32_t gelu_erf_fast_bf16x2(float z0, float z1) {
     asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(u1));
     const uint64_t H = fma_f32x2(Z, f32x2(0.5f, 0.5f), zero);
     const uint64_t G = fma_f32x2(H, f32x2(t0, t1), H);
-    float g0, g1;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(g0), "=f"(g1) : "l"(G));
+}
+__device__ __forceinline__ uint32_t gelu_erf_fast_bf16x2(float z0, float z1) {
+    float g0, g1;
+    gelu_erf_fast_x2(z0, z1, g0, g1);
     __nv_bfloat162 v = __floats2bfloat162_rn(g0, g1);
     return *reinterpret_cast<uint32_t*>(&v);
 }
@@ -60,13 +64,15 @@ __device__ __forceinline__ uint32_t pack_16x2(float a, float b) {
         return pack_bf16x2(a, b);
     }
 }
-// gelu of a pair, rounded to the storage type.  The half form keeps the erf of the math library:
-// the tanh form's 1.5e-4 relative error is of the size of half's own rounding (2.4e-4).
+// gelu of a pair, rounded to the storage type.  Both types take the tanh form: its error (1.5e-4
+// of the value plus the tanh unit's 2^-11) is of the size of half's own rounding (2^-12 to 2^-11),
+// and the erf of the math library costs five times the issue slots, which the epilogue -- the
+// stage the tensor pipe waits for -- does not have (measured: 92 against 55 us on a D = 256 shape).
 template <bool F16>
 __device__ __forceinline__ uint32_t gelu_pack_16x2(float z0, float z1) {
     if constexpr (F16) {
-        const float g0 = 0.5f * z0 * (1.0f + erff(z0 * 0.70710678118654752440f));
-        const float g1 = 0.5f * z1 * (1.0f + erff(z1 * 0.70710678118654752440f));
+        float g0, g1;
+        gelu_erf_fast_x2(z0, z1, g0, g1);
         return pack_16x2<true>(g0, g1);
     } else {
         return gelu_erf_fast_bf16x2(z0, z1);

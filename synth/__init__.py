@@ -92,6 +92,9 @@ CONFIG5_CELLS = [(B, T) for B in (1, 16, 256, 4096) for T in (64, 256, 1024, 409
 
 
 def by_name(name: str) -> Workload:
+    if name.endswith(":f16"):   # the same workload with IEEE-half tensors
+        w = by_name(name[:-4])
+        return w.with_(dtype="f16", name=w.name + "_f16")
     if name in ("1", "cfg1"):
         return config1()
     if name in ("2", "cfg2"):
