@@ -510,6 +510,52 @@ def stage_fractions(wm, prof, n_prof, peaks):
                 "useful_tflops": wm["ffn_flops"] / max(t_ffn, 1e-12) / 1e12}}
 
 
+def quick_moe(sentry, dev: str, local_rank: int, peaks):
+    """The Sparse-MoE block (Section 4.6) on a synthetic shape of its own (the paper gives none): 32 768 tokens,
+    d_model 256, 8 experts of d_ff 1024 pruned to 512 channels each, top-2 routing with skewed expert popularity.
+    Median of 5 blocks of 20 calls on rotating inputs; weights gathered per call, and materialised once."""
+    N, D, F, E, top_k, k_c = 32768, 256, 1024, 8, 2, 512
+    m = synth.generate_moe(N, D, F, E, top_k, k_c, "bf16", seed=11, skew=1.0, device=dev)
+    sn = sentry.Sentry(local_rank)
+    kept = torch.as_tensor(m.kept, device=dev)
+    ids = torch.as_tensor(m.expert_ids, device=dev)
+    wts = torch.as_tensor(m.expert_weights, device=dev)
+    n_sets = 8   # 8 x (X + Y) = 268 MB of rotating activations (> L2) beside the 8 MB of expert weights
+    Xs = [m.X] + [torch.randn_like(m.X, dtype=torch.float32).to(m.X.dtype) for _ in range(n_sets - 1)]
+    Ys = [torch.empty_like(m.X) for _ in range(n_sets)]
+    packed = sn.moe_prepack(m.W1, m.W2, kept)
+    out = {"workload": "moe_N32768_D256_F1024_E8_top2_kc512", "tokens": N}
+
+    def run(i, once):
+        if once:
+            sn.moe_ffn_fwd(Xs[i % n_sets], ids, wts, packed=packed, F=F, E=E, k_c=k_c, Y=Ys[i % n_sets])
+        else:
+            sn.moe_ffn_fwd(Xs[i % n_sets], ids, wts, W1=m.W1, W2=m.W2, kept_channels=kept, Y=Ys[i % n_sets])
+
+    flops = 4.0 * D * k_c * N * top_k
+    for once in (False, True):
+        for i in range(5):
+            run(i, once)
+        launches = sn.last_launch_count()
+        torch.cuda.synchronize()
+        blocks = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for r in range(5):
+            e0.record()
+            for i in range(20):
+                run(r * 20 + i, once)
+            e1.record()
+            torch.cuda.synchronize()
+            blocks.append(e0.elapsed_time(e1) / 20)
+        ms = float(np.median(blocks))
+        key = "materialised_once" if once else "per_call_gather"
+        out[key] = {"ms_per_call": ms, "tokens_per_s": N / (ms * 1e-3), "launches_per_call": launches,
+                    "tensor_frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+    out["device_status"] = sn.last_status()
+    sn.close()
+    return out
+
+
 def quick_config(sentry, name: str, dev: str, local_rank: int, peaks, args):
     """Short measurement of one other workload for the `configs` table: median of 3 blocks of at
     least ~10 ms, plus the per-kernel pass."""
@@ -707,6 +753,10 @@ def run_ours(args, w: synth.Workload):
                 table[name] = quick_config(sentry, name, dev, local_rank, peaks, args)
             except Exception as ex:   # a cell that does not fit or fails must not take the line down
                 table[name] = {"error": repr(ex)[:200]}
+        try:
+            table["moe"] = quick_moe(sentry, dev, local_rank, peaks)
+        except Exception as ex:
+            table["moe"] = {"error": repr(ex)[:200]}
     sampler.stop_flag = True
 
     cpu = {"value": None, "unit": "tokens/s", "cores": None, "kind": "oracle", "sample": "skipped"}
