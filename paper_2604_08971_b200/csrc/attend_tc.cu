@@ -5,7 +5,7 @@
 //   1. Present tokens of the sample -> runs of consecutive tokens.  K, V (and later Q) rows sit in
 //      shared memory in present-token order, in the swizzled row layout the tensor core reads.
 //      The part of every run between 8-row boundaries comes by TMA tensor copies (boxes of 64
-//      and of 8 rows, no multicast); the few rows before and behind it, and everything when the
+//      and of 8 rows, each CTA fetching its own copy); the few rows before and behind it, and everything when the
 //      present tokens are scattered over more than kMaxRuns runs, come by 16-byte async copies
 //      into the same layout.  K and V are read from HBM once per group.
 //   2. Sparsity scores (max minus mean of q.k/sqrt(d) over the sampled keys of every query): one
