@@ -256,7 +256,9 @@ SENTRY_API int sentry_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc
  * the short workloads' step time is made of; otherwise this is
  * sentry_gate_select followed by sentry_attend_fwd.  A mask >= S is flagged
  * BAD_INDEX (the one-launch form then uses row 0 for that sample, the
- * two-launch form leaves its list unwritten).  No forced selection here. */
+ * two-launch form leaves its list unwritten).  No forced selection here.
+ * Workspace: what sentry_attend_fwd needs for the descriptor, and at least
+ * S*k_h*4 + S*4 + 512 bytes (the two-launch form's gate rows). */
 SENTRY_API int sentry_gate_attend_fwd(sentry_ctx* ctx, const sentry_attend_desc* desc,
                            const float* head_scores, int S, const void* Q, const void* K,
                            const void* V, const int32_t* token_modality_ids,
