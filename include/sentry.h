@@ -305,6 +305,14 @@ SENTRY_API size_t sentry_ffn_packed_bytes(const sentry_ffn_desc* desc);
 SENTRY_API int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* W1,
                        const void* W2, const int32_t* kept_channels, void* packed,
                        size_t packed_bytes, void* stream);
+/* The weights kept in FP8 (Sec. 5: the FP8 point of the quantisation axis is the one that pays in STORAGE): W1 [D,F]
+ * and W2 [F,D] as e4m3 codes (one byte each: sign, 4 exponent bits with bias 7, 3 fraction bits, no infinities), each
+ * with one fp32 scale; an element is decode(code) * scale.  sentry_ffn_prepack_fp8 materialises W1[:, N], W2[N, :]
+ * of every list from them into `packed`, rounded once to desc->dtype, in the layout sentry_ffn_fwd_packed reads: the
+ * FFN then runs as for 16-bit weights (the arithmetic is not FP8: weights-only quantisation). */
+SENTRY_API int sentry_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const uint8_t* W1_e4m3,
+                           const uint8_t* W2_e4m3, float scale_w1, float scale_w2,
+                           const int32_t* kept_channels, void* packed, size_t packed_bytes, void* stream);
 SENTRY_API int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X,
                           const void* packed, const int32_t* list_of_sample,
                           const int32_t* token_modality_ids, const uint32_t* masks, void* Y,

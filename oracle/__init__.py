@@ -216,3 +216,25 @@ def moe_ffn(X, W1, W2, kept_channels, expert_ids, expert_weights) -> np.ndarray:
     Y = np.empty((N, D), dtype=np.float64)
     _load().oracle_moe_ffn(_p(X), _p(W1), _p(W2), N, D, F, E, _p(kc), kc.shape[1], _p(ex), _p(wt), ex.shape[1], _p(Y))
     return Y
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Value of every FP8 e4m3 code (Section 5's FP8 storage point; the format is the published
+    8-bit one: sign, 4 exponent bits with bias 7, 3 fraction bits, subnormals at exponent 0, no
+    infinities, exponent 15 with fraction 7 is NaN, largest finite value 448).  float64, exact."""
+    c = np.asarray(codes).astype(np.uint8).astype(np.int64)
+    sign = np.where((c >> 7) & 1, -1.0, 1.0)
+    e = (c >> 3) & 15
+    m = c & 7
+    val = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2(e.astype(np.float64) - 7.0))
+    val = np.where((e == 15) & (m == 7), np.nan, val)
+    return sign * val
+
+
+def dequantise_e4m3(codes, scale: float, dtype: str = "bf16"):
+    """decode(code) * scale as the pruned FFN takes FP8-stored weights: the product in fp32 (both
+    factors are exact in fp32), rounded once to the compute type by the library's conversion."""
+    import torch   # only for the library's rounding to the 16-bit types
+    prod = e4m3_decode(codes).astype(np.float32) * np.float32(scale)
+    t = torch.from_numpy(prod)
+    return t.to({"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[dtype])

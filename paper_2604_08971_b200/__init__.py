@@ -31,7 +31,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
-           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_fwd_packed",
+           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_prepack_fp8", "sentry_ffn_fwd_packed",
            "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out",
            "sentry_gate_select_multi", "sentry_sample_table_arrange", "sentry_gate_attend_fwd", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
 
@@ -107,6 +107,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_packed_bytes.argtypes = [ctypes.POINTER(FfnDesc)]
     lib.sentry_ffn_packed_bytes.restype = ctypes.c_size_t
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.sentry_ffn_prepack_fp8.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, ctypes.c_float, ctypes.c_float, vp, vp,
+                                           ctypes.c_size_t, vp]
     lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_gate_select_multi.argtypes = [vp, ci, ctypes.POINTER(GateSet), ci, vp]
     lib.sentry_gate_attend_fwd.argtypes = [vp, ctypes.POINTER(AttendDesc), vp, ci, vp, vp, vp, vp, vp, vp, vp, ci, vp, vp, vp, vp]
@@ -401,6 +403,24 @@ class Sentry:
                                          _ptr(packed), packed.numel(), _stream())
         if rc != 0:
             raise SentryError(rc, "sentry_ffn_prepack")
+        return packed
+
+    def ffn_prepack_fp8(self, W1q, W2q, scale_w1: float, scale_w2: float, kept_channels, dtype=torch.bfloat16,
+                        packed=None):
+        """sentry_ffn_prepack_fp8: W1q [D,F], W2q [F,D] uint8 e4m3 codes -> packed buffer of `dtype` weights."""
+        if kept_channels.dim() == 1:
+            kept_channels = kept_channels[None, :]
+        D, F = W1q.shape
+        n_lists, k_c = kept_channels.shape
+        code = {torch.float32: SENTRY_F32, torch.bfloat16: SENTRY_BF16, torch.float16: SENTRY_F16}[dtype]
+        desc = FfnDesc(1, 1, D, F, k_c, n_lists, code)
+        nbytes = int(self.lib.sentry_ffn_packed_bytes(ctypes.byref(desc)))
+        if packed is None:
+            packed = torch.empty((nbytes,), dtype=torch.uint8, device=W1q.device)
+        rc = self.lib.sentry_ffn_prepack_fp8(self.h, ctypes.byref(desc), _ptr(W1q), _ptr(W2q), float(scale_w1),
+                                             float(scale_w2), _ptr(kept_channels), _ptr(packed), packed.numel(), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_ffn_prepack_fp8")
         return packed
 
     def ffn_fwd_packed(self, X, packed, F: int, k_c: int, n_lists: int, list_of_sample=None,

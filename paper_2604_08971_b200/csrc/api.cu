@@ -565,6 +565,22 @@ int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void*
     return launch_ffn_prepack(ctx, a, packed, (cudaStream_t)stream);
 }
 
+int sentry_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const uint8_t* W1_e4m3, const uint8_t* W2_e4m3,
+                           float scale_w1, float scale_w2, const int32_t* kept_channels, void* packed,
+                           size_t packed_bytes, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_ffn_desc(desc);
+    if (rc != SENTRY_OK) return rc;
+    if (W1_e4m3 == nullptr || W2_e4m3 == nullptr || kept_channels == nullptr || packed == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(kept_channels, 4) || !aligned(packed, 256)) return SENTRY_ERR_INVALID_ARG;
+    if (!(scale_w1 == scale_w1) || !(scale_w2 == scale_w2)) return SENTRY_ERR_INVALID_ARG;   // NaN scales
+    if (packed_bytes < ffn_packed_bytes(*desc)) return SENTRY_ERR_WORKSPACE;
+    ctx->last_launches = 0;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_ffn_prepack_fp8(ctx, *desc, W1_e4m3, W2_e4m3, scale_w1, scale_w2, kept_channels, packed,
+                                  (cudaStream_t)stream);
+}
+
 int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X, const void* packed,
                           const int32_t* list_of_sample, const int32_t* token_modality_ids,
                           const uint32_t* masks, void* Y, void* stream) {

@@ -390,6 +390,8 @@ struct FfnArgs {
 size_t ffn_workspace_bytes(const sentry_ffn_desc& d);
 size_t ffn_packed_bytes(const sentry_ffn_desc& d);
 int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStream_t st);
+int launch_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc& d, const uint8_t* W1q, const uint8_t* W2q, float s1,
+                           float s2, const int32_t* kept, void* packed, cudaStream_t st);
 int launch_wait_expiry_selftest(sentry_ctx* ctx, long long limit_cycles, cudaStream_t st);
 int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, const void* packed, cudaStream_t st);
 int ffn_kc_pad(const sentry_ffn_desc& d);

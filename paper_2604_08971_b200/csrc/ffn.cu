@@ -5,6 +5,8 @@
 #include <math.h>
 
 #include "common.cuh"
+#include <cuda_fp8.h>
+
 #include "ffn_plan.cuh"
 
 int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c,
@@ -222,6 +224,47 @@ ffn_prepare_kernel(const int32_t* __restrict__ ids, const uint32_t* __restrict__
     }
 }
 
+// The weight gather from FP8 storage: W1q [D,F] and W2q [F,D] hold e4m3 codes (4 exponent bits, 3
+// fraction bits, bias 7, no infinities), each with one fp32 scale; element = decode(code) * scale,
+// rounded once to the compute type T.  Same destination layouts as the gather above; a one-off
+// (materialise-once) step, so one thread per destination element is enough.
+template <typename T>
+__global__ void __launch_bounds__(256)
+ffn_prepack_fp8_kernel(const uint8_t* __restrict__ W1q, const uint8_t* __restrict__ W2q, float s1, float s2,
+                       const int32_t* __restrict__ kept, int n_lists, int D, int F, int k_c, int kc_pad,
+                       int layout, T* __restrict__ out1, T* __restrict__ out2, unsigned int* status) {
+    const size_t per = (size_t)kc_pad * D;
+    const size_t blocks_per = (per + 255) / 256;
+    size_t pb = blockIdx.x;
+    const int which = (int)(pb / (blocks_per * n_lists));
+    pb -= (size_t)which * blocks_per * n_lists;
+    const int l = (int)(pb / blocks_per);
+    const size_t i = (pb % blocks_per) * 256 + threadIdx.x;
+    if (i >= per) return;
+    const int32_t* N = kept + (size_t)l * k_c;
+    auto decode = [](uint8_t code) {
+        __nv_fp8_e4m3 q;
+        q.__x = code;
+        return float(q);
+    };
+    int n, e;
+    if (which == 0) {
+        if (layout == 0) { e = (int)(i / kc_pad); n = (int)(i % kc_pad); }
+        else             { n = (int)(i / D);      e = (int)(i % D); }
+    } else {
+        if (layout == 0) { n = (int)(i / D);      e = (int)(i % D); }
+        else             { e = (int)(i / kc_pad); n = (int)(i % kc_pad); }
+    }
+    T v = from_f32<T>(0.f);
+    if (n < k_c) {
+        const int ch = N[n];
+        if (ch >= 0 && ch < F)
+            v = which == 0 ? from_f32<T>(decode(W1q[(size_t)e * F + ch]) * s1) : from_f32<T>(decode(W2q[(size_t)ch * D + e]) * s2);
+        else if (which == 0 && e == 0) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+    }
+    (which == 0 ? out1 : out2)[(size_t)l * per + i] = v;
+}
+
 __device__ __forceinline__ float gelu_erf(float z) {
     return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f));
 }
@@ -369,6 +412,30 @@ int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStre
             nullptr, nullptr, nullptr, 0, d.T, 1, tc ? kTcTileRows : kGenericTileRows, none, nullptr,
             (const __nv_bfloat16*)a.W1, (const __nv_bfloat16*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad,
             tc ? 1 : 0, a.w_stride, (__nv_bfloat16*)w1p, (__nv_bfloat16*)w2p, a.status);
+    SENTRY_CUDA_TRY(cudaGetLastError());
+    return SENTRY_OK;
+}
+
+int launch_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc& d, const uint8_t* W1q, const uint8_t* W2q, float s1,
+                           float s2, const int32_t* kept, void* packed, cudaStream_t st) {
+    const bool tc = ffn_tc_supported(d);
+    const int kc_pad = kc_pad_for(d);
+    const size_t per = (size_t)kc_pad * d.D;
+    const unsigned grid = (unsigned)(2 * (size_t)d.n_lists * ((per + 255) / 256));
+    uint8_t* w1p = (uint8_t*)packed;
+    uint8_t* w2p = w1p + packed_half_bytes(d, kc_pad);
+    const int layout = tc ? 1 : 0;
+    LaunchScope ls(ctx, KS_FFN_PREPARE, st);
+    if (d.dtype == SENTRY_F32)
+        ffn_prepack_fp8_kernel<float><<<grid, 256, 0, st>>>(W1q, W2q, s1, s2, kept, d.n_lists, d.D, d.F, d.k_c, kc_pad,
+                                                           layout, (float*)w1p, (float*)w2p, ctx->d_status);
+    else if (d.dtype == SENTRY_F16)
+        ffn_prepack_fp8_kernel<__half><<<grid, 256, 0, st>>>(W1q, W2q, s1, s2, kept, d.n_lists, d.D, d.F, d.k_c, kc_pad,
+                                                            layout, (__half*)w1p, (__half*)w2p, ctx->d_status);
+    else
+        ffn_prepack_fp8_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(W1q, W2q, s1, s2, kept, d.n_lists, d.D, d.F, d.k_c,
+                                                                   kc_pad, layout, (__nv_bfloat16*)w1p,
+                                                                   (__nv_bfloat16*)w2p, ctx->d_status);
     SENTRY_CUDA_TRY(cudaGetLastError());
     return SENTRY_OK;
 }

@@ -523,3 +523,21 @@ def test_moe_ffn_equals_library_form_and_reduces_to_plain_ffn():
     a = oracle.moe_ffn(X, W1, W2, kept, ex, wt0)
     b = oracle.moe_ffn(X, W1, W2, kept, ex[:, :1], wt[:, :1])
     np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+
+
+def test_e4m3_decode_matches_the_library_and_the_format_constants():
+    """Every one of the 256 codes against the library's float8 conversion, plus the values the
+    format fixes by definition (1.0, the largest finite value 448, the smallest subnormal 2^-9,
+    the smallest normal 2^-6, signed zero, the NaN code)."""
+    codes = np.arange(256, dtype=np.uint8)
+    got = oracle.e4m3_decode(codes)
+    lib = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    np.testing.assert_array_equal(np.isnan(got), np.isnan(lib))
+    ok = ~np.isnan(lib)
+    np.testing.assert_array_equal(got[ok], lib[ok])
+    assert got[0x38] == 1.0 and got[0x7E] == 448.0 and got[0x01] == 2.0 ** -9 and got[0x08] == 2.0 ** -6
+    assert got[0x00] == 0.0 and got[0x80] == 0.0 and np.signbit(got[0x80]) and got[0xB8] == -1.0
+    assert np.isnan(got[0x7F]) and np.isnan(got[0xFF])
+    # dequantisation: fp32 product, one rounding to the compute type
+    w = oracle.dequantise_e4m3(np.array([0x38, 0x3C, 0xC9], dtype=np.uint8), 0.5, "bf16")
+    np.testing.assert_array_equal(w.float().numpy(), np.array([0.5, 0.75, -2.25], dtype=np.float32))   # 0xC9 = -(1 + 1/8) * 2^(9-7)
