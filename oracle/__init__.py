@@ -6,8 +6,12 @@ reference arm may import this package; the CUDA library never does, and this
 package never imports the CUDA library.
 
 Inputs may be numpy arrays or torch CPU tensors of any float dtype; they are
-widened to float64 exactly (bf16 and fp32 values are representable), so the
+widened to float64 exactly (bf16, fp16 and fp32 values are representable), so the
 oracle sees the same numbers the GPU reads.
+
+Besides the wrapper, two numpy functions of their own: ``e4m3_decode`` (the FP8
+format written out from its definition; pinned against the library's float8
+conversion on all 256 codes, tests/test_oracle_pins.py) and ``dequantise_e4m3``.
 """
 from __future__ import annotations
 
