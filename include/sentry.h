@@ -65,7 +65,7 @@ typedef enum {
 /* SENTRY_F16 (IEEE half; the FP16 post-training-quantisation point of Sec. 5): taken by every entry point.  The
  * FFN pair and the Sparse-MoE block run on tcgen05 with fp16 operands, attention on the warp-MMA kernels with fp16
  * operands (the tcgen05 attention kernel is bf16 only), the projections on tcgen05 with fp16 operands. */
-typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1, SENTRY_F16 = 2 } sentry_dtype;
+typedef enum { SENTRY_F32 = 0, SENTRY_BF16 = 1, SENTRY_F16 = 2, SENTRY_FP8_E4M3 = 3 /* FFN only, see sentry_ffn_fwd_fp8 */ } sentry_dtype;
 
 /* Create / destroy a context bound to CUDA device `device`.  Creation
  * allocates one small device status word; nothing else. */
@@ -313,6 +313,18 @@ SENTRY_API int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, 
 SENTRY_API int sentry_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const uint8_t* W1_e4m3,
                            const uint8_t* W2_e4m3, float scale_w1, float scale_w2,
                            const int32_t* kept_channels, void* packed, size_t packed_bytes, void* stream);
+/* FP8 ARITHMETIC (Sec. 5, the FP8 point taken to the tensor cores; desc->dtype = SENTRY_FP8_E4M3, D = 256 only):
+ * X [B,T,D] and the weights are e4m3 codes with per-tensor scales scale_x, scale_w1, scale_w2; the hidden
+ * activations are requantised to e4m3 with scale_h (a calibration constant of the caller); Y is bf16:
+ *   z = (x_q . W1_q[:, N]) * (scale_x*scale_w1);  h_q = e4m3(gelu(z) / scale_h)   (nearest, saturating at 448)
+ *   y = (h_q . W2_q[N, :]) * (scale_h*scale_w2)
+ * with exact e4m3 x e4m3 products accumulated in fp32 (tcgen05 kind::f8f6f4).  The weights come from
+ * sentry_ffn_prepack called with the same FP8 descriptor on the e4m3 W1 [D,F], W2 [F,D] (it gathers bytes).
+ * All scales > 0.  Other shapes: SENTRY_ERR_UNSUPPORTED. */
+SENTRY_API int sentry_ffn_fwd_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X_e4m3,
+                       const void* packed, const int32_t* list_of_sample,
+                       const int32_t* token_modality_ids, const uint32_t* masks, float scale_x,
+                       float scale_w1, float scale_w2, float scale_h, void* Y_bf16, void* stream);
 SENTRY_API int sentry_ffn_fwd_packed(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X,
                           const void* packed, const int32_t* list_of_sample,
                           const int32_t* token_modality_ids, const uint32_t* masks, void* Y,

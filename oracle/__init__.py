@@ -242,3 +242,55 @@ def dequantise_e4m3(codes, scale: float, dtype: str = "bf16"):
     prod = e4m3_decode(codes).astype(np.float32) * np.float32(scale)
     t = torch.from_numpy(prod)
     return t.to({"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[dtype])
+
+
+def e4m3_encode(values) -> np.ndarray:
+    """Nearest e4m3 code of every value (ties to even, magnitudes beyond 448 saturate to 448;
+    NaN -> the NaN code), from the format's definition: below 2^-6 the spacing is 2^-9, above it
+    2^(e-3) in the binade [2^e, 2^(e+1)).  uint8."""
+    v = np.asarray(values, dtype=np.float64)
+    a = np.minimum(np.abs(v), 448.0)
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))
+    quantum = np.exp2(e - 3.0)
+    q = np.rint(a / quantum) * quantum          # numpy rounds halves to even
+    q = np.minimum(q, 448.0)
+    # back to (exponent, fraction) fields
+    e2 = np.floor(np.log2(np.maximum(q, 2.0 ** -6)))
+    sub = q < 2.0 ** -6
+    frac = np.where(sub, np.rint(q / 2.0 ** -9), np.rint(q / np.exp2(e2 - 3.0)) - 8.0)
+    expf = np.where(sub, 0.0, e2 + 7.0)
+    code = (expf.astype(np.int64) << 3) | frac.astype(np.int64)
+    code = np.where(np.signbit(v), code | 0x80, code)
+    code = np.where(np.isnan(v), 0x7F, code)
+    return code.astype(np.uint8)
+
+
+def ffn_fp8(Xq, W1q, W2q, kept_channels, list_of_sample, ids, masks, scale_x, scale_w1, scale_w2, scale_h) -> np.ndarray:
+    """The channel-compacted FFN with FP8 (e4m3) operands and per-tensor scales (Section 5's FP8
+    point taken to the arithmetic): for a present row x of sample b with kept list N,
+        z   = (x_q . W1_q[:, N]) * (scale_x * scale_w1)            exact products, exact sum
+        h_q = e4m3( gelu(z) / scale_h )                            exact erf; nearest e4m3, saturating
+        y   = (h_q . W2_q[N, :]) * (scale_h * scale_w2)
+    Scale products and the requantisation argument are taken in fp32, the precision the device
+    takes them in.  Xq [B,T,D], W1q [D,F], W2q [F,D] uint8 codes; returns Y [B,T,D] float64."""
+    from math import sqrt
+    from scipy.special import erf
+    X = e4m3_decode(Xq)
+    W1 = e4m3_decode(W1q)
+    W2 = e4m3_decode(W2q)
+    kc = _i32(kept_channels)
+    los = _i32(list_of_sample) if list_of_sample is not None else np.zeros(X.shape[0], dtype=np.int32)
+    B, T, D = X.shape
+    a_scale = np.float32(scale_x) * np.float32(scale_w1)
+    h_inv = np.float32(1.0) / np.float32(scale_h)
+    y_scale = np.float32(scale_h) * np.float32(scale_w2)
+    Y = np.zeros((B, T, D), dtype=np.float64)
+    for b in range(B):
+        N = kc[los[b]]
+        present = np.ones(T, dtype=bool) if ids is None else ((int(masks[b]) >> np.asarray(ids)) & 1).astype(bool)
+        xb = X[b][present]
+        z = (xb @ W1[:, N]).astype(np.float32) * a_scale
+        g = 0.5 * z.astype(np.float64) * (1.0 + erf(z.astype(np.float64) / sqrt(2.0)))
+        hq = e4m3_decode(e4m3_encode(g.astype(np.float32) * h_inv))
+        Y[b][present] = (hq @ W2[N, :]) * np.float64(y_scale)
+    return Y

@@ -19,7 +19,7 @@ from . import build as _build
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsentry.so")
 
-SENTRY_F32, SENTRY_BF16, SENTRY_F16 = 0, 1, 2
+SENTRY_F32, SENTRY_BF16, SENTRY_F16, SENTRY_FP8_E4M3 = 0, 1, 2, 3
 STATUS_BIT_TIMEOUT, STATUS_BIT_EMPTY_MASK, STATUS_BIT_BAD_INDEX = 1, 2, 4
 OPT_ATTEND_KERNEL = 1
 ATTEND_AUTO, ATTEND_WARP_MMA, ATTEND_TCGEN05 = 0, 1, 2
@@ -31,7 +31,7 @@ EXPORTS = ["sentry_create", "sentry_destroy", "sentry_get_last_status", "sentry_
            "sentry_gate_select", "sentry_attend_fwd", "sentry_ffn_fwd", "sentry_last_launch_count",
            "sentry_profile_enable", "sentry_profile_slots", "sentry_profile_read",
            "sentry_kernel_name", "sentry_gate_select_static", "sentry_selftest_wait_expiry", "sentry_set_option",
-           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_prepack_fp8", "sentry_ffn_fwd_packed",
+           "sentry_ffn_packed_bytes", "sentry_ffn_prepack", "sentry_ffn_prepack_fp8", "sentry_ffn_fwd_fp8", "sentry_ffn_fwd_packed",
            "sentry_gate_eval", "sentry_gate_layer_counts", "sentry_project_qkv", "sentry_project_out",
            "sentry_gate_select_multi", "sentry_sample_table_arrange", "sentry_gate_attend_fwd", "sentry_moe_workspace_bytes", "sentry_moe_packed_bytes", "sentry_moe_prepack", "sentry_moe_ffn_fwd"]
 
@@ -109,6 +109,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sentry_ffn_prepack.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.sentry_ffn_prepack_fp8.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, ctypes.c_float, ctypes.c_float, vp, vp,
                                            ctypes.c_size_t, vp]
+    lib.sentry_ffn_fwd_fp8.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
+                                       ctypes.c_float, ctypes.c_float, vp, vp]
     lib.sentry_ffn_fwd_packed.argtypes = [vp, ctypes.POINTER(FfnDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.sentry_gate_select_multi.argtypes = [vp, ci, ctypes.POINTER(GateSet), ci, vp]
     lib.sentry_gate_attend_fwd.argtypes = [vp, ctypes.POINTER(AttendDesc), vp, ci, vp, vp, vp, vp, vp, vp, vp, ci, vp, vp, vp, vp]
@@ -422,6 +424,40 @@ class Sentry:
         if rc != 0:
             raise SentryError(rc, "sentry_ffn_prepack_fp8")
         return packed
+
+    def ffn_prepack_e4m3(self, W1q, W2q, kept_channels, packed=None):
+        """sentry_ffn_prepack with dtype FP8: gathers W1q[:, N], W2q[N, :] (uint8 e4m3 codes) for sentry_ffn_fwd_fp8."""
+        if kept_channels.dim() == 1:
+            kept_channels = kept_channels[None, :]
+        D, F = W1q.shape
+        n_lists, k_c = kept_channels.shape
+        desc = FfnDesc(1, 1, D, F, k_c, n_lists, SENTRY_FP8_E4M3)
+        nbytes = int(self.lib.sentry_ffn_packed_bytes(ctypes.byref(desc)))
+        if nbytes == 0:
+            raise SentryError(-4, "sentry_ffn_packed_bytes (FP8 shape)")
+        if packed is None:
+            packed = torch.empty((nbytes,), dtype=torch.uint8, device=W1q.device)
+        rc = self.lib.sentry_ffn_prepack(self.h, ctypes.byref(desc), _ptr(W1q), _ptr(W2q), _ptr(kept_channels),
+                                         _ptr(packed), packed.numel(), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_ffn_prepack (FP8)")
+        return packed
+
+    def ffn_fwd_fp8(self, Xq, packed, F: int, k_c: int, n_lists: int, scale_x: float, scale_w1: float, scale_w2: float,
+                    scale_h: float, list_of_sample=None, token_modality_ids=None, masks=None, Y=None):
+        """sentry_ffn_fwd_fp8: Xq [B,T,D] uint8 e4m3 codes, packed from ffn_prepack_e4m3.  Returns Y [B,T,D] bf16."""
+        B, T, D = Xq.shape
+        desc = FfnDesc(B, T, D, int(F), int(k_c), int(n_lists), SENTRY_FP8_E4M3)
+        if Y is None:
+            Y = torch.empty((B, T, D), dtype=torch.bfloat16, device=Xq.device)
+        desc16 = FfnDesc(B, T, D, int(F), int(k_c), int(n_lists), SENTRY_BF16)
+        self.ensure_workspace(self.workspace_bytes(ffn=desc16))
+        rc = self.lib.sentry_ffn_fwd_fp8(self.h, ctypes.byref(desc), _ptr(Xq), _ptr(packed), _ptr(list_of_sample),
+                                         _ptr(token_modality_ids), _ptr(masks), float(scale_x), float(scale_w1),
+                                         float(scale_w2), float(scale_h), _ptr(Y), _stream())
+        if rc != 0:
+            raise SentryError(rc, "sentry_ffn_fwd_fp8")
+        return Y
 
     def ffn_fwd_packed(self, X, packed, F: int, k_c: int, n_lists: int, list_of_sample=None,
                        token_modality_ids=None, masks=None, Y=None):

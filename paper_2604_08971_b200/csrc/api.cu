@@ -33,9 +33,13 @@ int check_attend_desc(const sentry_attend_desc* d) {
     return SENTRY_OK;
 }
 
-int check_ffn_desc(const sentry_ffn_desc* d) {
+int check_ffn_desc(const sentry_ffn_desc* d, bool fp8_ok = false) {
     if (d == nullptr) return SENTRY_ERR_INVALID_ARG;
-    if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16 && d->dtype != SENTRY_F16) return SENTRY_ERR_INVALID_ARG;
+    if (d->dtype == SENTRY_FP8_E4M3) {
+        if (!fp8_ok) return SENTRY_ERR_UNSUPPORTED;
+    } else if (d->dtype != SENTRY_F32 && d->dtype != SENTRY_BF16 && d->dtype != SENTRY_F16) {
+        return SENTRY_ERR_INVALID_ARG;
+    }
     if (d->B < 1 || d->T < 1 || d->D < 1 || d->F < 1 || d->k_c < 1 || d->n_lists < 1)
         return SENTRY_ERR_BAD_SHAPE;
     if (d->k_c > d->F) return SENTRY_ERR_BAD_SHAPE;
@@ -543,13 +547,14 @@ int sentry_moe_ffn_fwd(sentry_ctx* ctx, const sentry_moe_desc* desc, const void*
 }
 
 size_t sentry_ffn_packed_bytes(const sentry_ffn_desc* desc) {
-    return check_ffn_desc(desc) == SENTRY_OK ? ffn_packed_bytes(*desc) : 0;
+    return check_ffn_desc(desc, true) == SENTRY_OK ? ffn_packed_bytes(*desc) : 0;
 }
 
 int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* W1, const void* W2,
                        const int32_t* kept_channels, void* packed, size_t packed_bytes, void* stream) {
     if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
-    int rc = check_ffn_desc(desc);
+    int rc = check_ffn_desc(desc, true);
+    if (rc == SENTRY_OK && desc->dtype == SENTRY_FP8_E4M3 && !ffn_tc_fp8_supported(*desc)) rc = SENTRY_ERR_UNSUPPORTED;
     if (rc != SENTRY_OK) return rc;
     if (W1 == nullptr || W2 == nullptr || kept_channels == nullptr || packed == nullptr) return SENTRY_ERR_INVALID_ARG;
     if (!aligned(W1, 16) || !aligned(W2, 16) || !aligned(kept_channels, 4) || !aligned(packed, 256))
@@ -563,6 +568,35 @@ int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void*
     a.status = ctx->d_status;
     SENTRY_ON_DEVICE(ctx->device);
     return launch_ffn_prepack(ctx, a, packed, (cudaStream_t)stream);
+}
+
+int sentry_ffn_fwd_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const void* X_e4m3, const void* packed,
+                       const int32_t* list_of_sample, const int32_t* token_modality_ids, const uint32_t* masks,
+                       float scale_x, float scale_w1, float scale_w2, float scale_h, void* Y_bf16, void* stream) {
+    if (ctx == nullptr) return SENTRY_ERR_INVALID_ARG;
+    int rc = check_ffn_desc(desc, true);
+    if (rc != SENTRY_OK) return rc;
+    if (desc->dtype != SENTRY_FP8_E4M3) return SENTRY_ERR_INVALID_ARG;
+    if (!ffn_tc_fp8_supported(*desc)) return SENTRY_ERR_UNSUPPORTED;
+    if (X_e4m3 == nullptr || packed == nullptr || Y_bf16 == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if ((token_modality_ids == nullptr) != (masks == nullptr)) return SENTRY_ERR_INVALID_ARG;
+    if (desc->n_lists > 1 && list_of_sample == nullptr) return SENTRY_ERR_INVALID_ARG;
+    if (!aligned(X_e4m3, 16) || !aligned(Y_bf16, 16) || !aligned(packed, 256)) return SENTRY_ERR_INVALID_ARG;
+    if (!(scale_x > 0.f) || !(scale_w1 > 0.f) || !(scale_w2 > 0.f) || !(scale_h > 0.f)) return SENTRY_ERR_INVALID_ARG;
+    ctx->last_launches = 0;
+    FfnArgs a = {};
+    a.d = *desc;
+    a.X = X_e4m3;
+    a.list_of_sample = list_of_sample;
+    a.ids = token_modality_ids;
+    a.masks = masks;
+    a.Y = Y_bf16;
+    a.status = ctx->d_status;
+    a.fp8_a_scale = scale_x * scale_w1;
+    a.fp8_h_inv = 1.0f / scale_h;
+    a.fp8_y_scale = scale_h * scale_w2;
+    SENTRY_ON_DEVICE(ctx->device);
+    return launch_ffn(ctx, a, ctx->workspace, ctx->workspace_bytes, packed, (cudaStream_t)stream);
 }
 
 int sentry_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const uint8_t* W1_e4m3, const uint8_t* W2_e4m3,

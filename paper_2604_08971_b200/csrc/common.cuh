@@ -301,6 +301,7 @@ template <typename T> __device__ __forceinline__ T from_f32(float x);
 template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 template <> __device__ __forceinline__ __half from_f32<__half>(float x) { return __float2half_rn(x); }
+template <> __device__ __forceinline__ uint8_t from_f32<uint8_t>(float) { return 0; }   // only the zero of the FP8 weight gather
 #endif  // __CUDACC__
 
 // ---- launchers implemented in the .cu files (host side; return sentry_status)
@@ -381,6 +382,7 @@ struct FfnArgs {
     const void *X, *W1, *W2;
     const int32_t* kept;
     size_t w_stride;        // elements between the weight matrices of consecutive lists (0: shared)
+    float fp8_a_scale, fp8_h_inv, fp8_y_scale;   // FP8 form: scale of GEMM1's accumulator, 1 / hidden scale, scale of Y
     const int32_t* list_of_sample;
     const int32_t* ids;
     const uint32_t* masks;
@@ -389,6 +391,7 @@ struct FfnArgs {
 };
 size_t ffn_workspace_bytes(const sentry_ffn_desc& d);
 size_t ffn_packed_bytes(const sentry_ffn_desc& d);
+bool ffn_tc_fp8_supported(const sentry_ffn_desc& d);
 int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStream_t st);
 int launch_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc& d, const uint8_t* W1q, const uint8_t* W2q, float s1,
                            float s2, const int32_t* kept, void* packed, cudaStream_t st);

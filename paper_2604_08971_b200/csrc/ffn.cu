@@ -351,7 +351,7 @@ struct FfnWs {
 
 // One of W1', W2' (all lists), rounded so that the second starts 256-byte aligned.
 size_t packed_half_bytes(const sentry_ffn_desc& d, int kc_pad) {
-    const size_t esz = d.dtype == SENTRY_F32 ? 4 : 2;
+    const size_t esz = d.dtype == SENTRY_F32 ? 4 : (d.dtype == SENTRY_FP8_E4M3 ? 1 : 2);
     return align_up((size_t)d.n_lists * kc_pad * d.D * esz, 256);
 }
 
@@ -403,7 +403,12 @@ int launch_ffn_prepack(sentry_ctx* ctx, const FfnArgs& a, void* packed, cudaStre
     none.rowout = nullptr;
     LaunchScope ls(ctx, KS_FFN_PREPARE, st);
     // no row-table and no zero-fill blocks (B = 0, no ids): every block gathers weights
-    if (d.dtype == SENTRY_F32)
+    if (d.dtype == SENTRY_FP8_E4M3) {
+        if (!tc) return SENTRY_ERR_UNSUPPORTED;
+        ffn_prepare_kernel<uint8_t><<<(unsigned)pack_blocks, 256, 0, st>>>(
+            nullptr, nullptr, nullptr, 0, d.T, 1, kTcTileRows, none, nullptr, (const uint8_t*)a.W1, (const uint8_t*)a.W2,
+            a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 1, a.w_stride, w1p, w2p, a.status);
+    } else if (d.dtype == SENTRY_F32)
         ffn_prepare_kernel<float><<<(unsigned)pack_blocks, 256, 0, st>>>(
             nullptr, nullptr, nullptr, 0, d.T, 1, kGenericTileRows, none, nullptr, (const float*)a.W1,
             (const float*)a.W2, a.kept, d.n_lists, d.D, d.F, d.k_c, kc_pad, 0, a.w_stride, (float*)w1p, (float*)w2p, a.status);
@@ -489,6 +494,7 @@ int launch_ffn(sentry_ctx* ctx, const FfnArgs& a, void* ws, size_t ws_bytes, con
     const sentry_ffn_desc& d = a.d;
     const bool tc = ffn_tc_supported(d);
     const int kc_pad = kc_pad_for(d);
+    if (d.dtype == SENTRY_FP8_E4M3 && (packed == nullptr || !tc)) return SENTRY_ERR_UNSUPPORTED;   // FP8: prepacked weights only
     FfnWs w = carve(d, kc_pad, ws, ws_bytes, packed == nullptr);
     if (!w.ok) return SENTRY_ERR_WORKSPACE;
     if (packed != nullptr) {

@@ -43,15 +43,20 @@ constexpr int kLoaderWarp0 = 3, kLoaderWarps = 4, kLoaderThreads = kLoaderWarps 
 constexpr int kEpiWarp0 = 7, kEpiWarps = 8;
 constexpr int kTmemCols = 512;
 
-template <int D>
+// FP8: X, the weights and the hidden activations are e4m3 bytes (a 128-byte operand row then
+// holds 128 elements instead of 64), the accumulators stay fp32, Y is stored as bf16.
+template <int D, bool FP8 = false>
 struct Cfg {
+    static constexpr int EPB = FP8 ? 128 : 64;         // elements per 128-byte operand row
     static constexpr int CH = (D == 384) ? 128 : 256;  // kept channels per chunk
-    static constexpr int KB1 = D / 64;                 // X blocks per tile = K blocks of GEMM1
+    static constexpr int CH16 = FP8 ? CH / 2 : CH;     // a chunk's width in the 16-bit units of the weight maps
+    static constexpr int KB1 = D / EPB;                // X blocks per tile = K blocks of GEMM1
     static constexpr int H_COL0 = (D == 384) ? 384 : 256;  // TMEM column of the hidden accumulator
-    static constexpr int NXS = (D == 128) ? 4 : KB1;   // X block slots (D = 128: two tiles' worth)
-    static constexpr int NHS = CH / 64;                // hidden blocks per chunk (64 channels each)
+    static constexpr int NXS = (D == 128 || FP8) ? 4 : KB1;   // X block slots (two tiles' worth where they are few)
+    static constexpr int NHS = CH / EPB;               // hidden blocks per chunk
     static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
     static constexpr int SPG = (D == 384) ? 3 : KB1;   // weight stages per chunk of GEMM1 (= of GEMM2)
+    static_assert(!FP8 || D == 256, "the FP8 form is built for d_model = 256");
     static constexpr int OFF_H = NXS * kBlockBytes;
     static constexpr int OFF_W = OFF_H + NHS * kBlockBytes;
     static constexpr int OFF_MISC = OFF_W + kStages * kStageBytes;
@@ -79,24 +84,29 @@ static_assert(sizeof(Misc) <= 2048, "misc block too large");
 #define MISC_BAR(base, field) ((base) + (uint32_t)offsetof(Misc, field))
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // upper word of umma_smem_desc_sw128
 __device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3fffu) | (1u << 16); }
-// D (+)= A . B^T for one 64-wide K block = four K=16 steps; descriptors from their low words
-__device__ __forceinline__ void mma_kblock_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
-                                              uint32_t accumulate_first) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
-        "setp.ne.b32 p, 1, 0;\n\t"
-        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
-        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
-        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        :
-        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(kDescHi), "r"(accumulate_first)
-        : "memory");
+// D (+)= A . B^T for one 128-byte K block = four 32-byte K steps (K = 16 16-bit or 32 8-bit elements);
+// descriptors from their low words
+#define SENTRY_MMA_KBLOCK(KIND)                                                                                       \
+    asm volatile(                                                                                                     \
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"                                            \
+        "setp.ne.b32 p, %5, 0;\n\t"                                                                                   \
+        "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\t"                                                          \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, p;\n\t"                                             \
+        "setp.ne.b32 p, 1, 0;\n\t"                                                                                    \
+        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"              \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, p;\n\t"                                             \
+        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"              \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, p;\n\t"                                             \
+        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"              \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, p;\n\t}"                                            \
+        :                                                                                                             \
+        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(kDescHi), "r"(accumulate_first)                          \
+        : "memory")
+template <bool FP8>
+__device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                           uint32_t accumulate_first) {
+    if constexpr (FP8) SENTRY_MMA_KBLOCK("f8f6f4");
+    else SENTRY_MMA_KBLOCK("f16");
 }
 // Slow path of a stage's combined wait: the barriers one after the other, bounded (0 = none).
 static __device__ __noinline__ bool wait_each_slow(uint32_t b0, uint32_t p0, uint32_t b1, uint32_t p1, uint32_t b2,
@@ -126,13 +136,16 @@ __device__ __forceinline__ void cta_teardown(volatile int* abort_flag, unsigned 
     }
 }
 
-template <int D, bool F16>
+// F16: X, W and Y are IEEE half instead of bf16.  FP8: X and the weights are e4m3 bytes with
+// per-tensor scales, the hidden activations are requantised to e4m3 (gelu(acc * a_scale) * h_inv),
+// Y = acc * y_scale is stored as bf16.
+template <int D, bool F16, bool FP8 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2_256,
               const __grid_constant__ CUtensorMap tm_w2_128, const __nv_bfloat16* __restrict__ X,
               __nv_bfloat16* __restrict__ Y, FfnPlan plan, int n_lists, int kc_pad,
-              unsigned int* status) {
-    using C = Cfg<D>;
+              unsigned int* status, float a_scale, float h_inv, float y_scale) {
+    using C = Cfg<D, FP8>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;   // 1024-byte aligned operand blocks
@@ -233,7 +246,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 n += SPG;
             }
             if (q > 0) {
-                const int pl = c ? l_cur : l_last, x = (c ? c - 1 : NC - 1) * C::CH, y = pl * D;
+                const int pl = c ? l_cur : l_last, x = (c ? c - 1 : NC - 1) * C::CH16, y = pl * D;
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
                     if (ok && ((n + i) & 1u) == me) {
@@ -262,8 +275,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         // two issuing warps were summed in an order that changed from run to run (results
         // differed in the last bit).  A second warp that did the waiting and handed the stage
         // number over through shared memory measured slower than the issuer waiting itself.
-        constexpr uint32_t idesc256 = F16 ? ptx::umma_idesc_f16(128, 256) : ptx::umma_idesc_bf16(128, 256);
-        constexpr uint32_t idesc128 = F16 ? ptx::umma_idesc_f16(128, 128) : ptx::umma_idesc_bf16(128, 128);
+        // (kind::f8f6f4 with both operand formats e4m3 has the same descriptor bits as kind::f16 with fp16 operands:
+        // format code 0 for A and B, fp32 accumulator)
+        constexpr uint32_t idesc256 = (F16 || FP8) ? ptx::umma_idesc_f16(128, 256) : ptx::umma_idesc_bf16(128, 256);
+        constexpr uint32_t idesc128 = (F16 || FP8) ? ptx::umma_idesc_f16(128, 128) : ptx::umma_idesc_bf16(128, 128);
         constexpr uint32_t kBlkLo = kBlockBytes >> 4, kStageLo = kStageBytes >> 4;
         const uint32_t tm_h = tmem + C::H_COL0;
         const uint32_t xs_lo = desc_lo(xs), hs_lo = desc_lo(hs), w_lo = desc_lo(wsm);
@@ -287,8 +302,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             ptx::tc_fence_after_sync();   // orders the UMMAs after the epilogue's TMEM reads and operand writes
             if (elect_one()) {
                 const uint32_t b_lo = w_lo + sl * kStageLo;
-                mma_kblock_lo(d_tm, a_lo0, b_lo, idesc, overwrite ? 0u : 1u);
-                if (a_lo1 != 0u) mma_kblock_lo(d_tm, a_lo1, b_lo + kBlkLo, idesc, 1u);
+                mma_kblock<FP8>(d_tm, a_lo0, b_lo, idesc, overwrite ? 0u : 1u);
+                if (a_lo1 != 0u) mma_kblock<FP8>(d_tm, a_lo1, b_lo + kBlkLo, idesc, 1u);
                 if (cb0 != 0u) ptx::umma_commit(cb0);
                 if (cb1 != 0u) ptx::umma_commit(cb1);
                 ptx::umma_commit(MISC_BAR(mb, w_empty) + 8u * sl);
@@ -402,7 +417,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     const int r = idx >> 3, ci = idx & 7;
                     const uint32_t dst = xs + slot * kBlockBytes + r * 128 + ((ci ^ (r & 7)) << 4);
                     if (rows[j] >= 0) {
-                        ptx::cp_async_16(dst, X + (size_t)rows[j] * D + kb * 64 + ci * 8);
+                        if constexpr (FP8)
+                            ptx::cp_async_16(dst, reinterpret_cast<const uint8_t*>(X) + (size_t)rows[j] * D + kb * 128 + ci * 16);
+                        else
+                            ptx::cp_async_16(dst, X + (size_t)rows[j] * D + kb * 64 + ci * 8);
                     } else {
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
                     }
@@ -428,7 +446,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         // hidden-block buffer (free while Y is complete and this warp has not yet written its
         // next hidden block there) so that the global stores cover whole 128-byte row segments.
         constexpr int kDrainBlk = C::NBATCH - 1;
-        const uint32_t stg = hs + (uint32_t)(half * C::NBATCH + kDrainBlk) * kBlockBytes + (uint32_t)quarter * 4096u;
+        // (FP8: a warp writes one 128-channel hidden block, rows of its own quarter: that piece)
+        const uint32_t stg = FP8 ? hs + (uint32_t)half * kBlockBytes + (uint32_t)quarter * 4096u
+                                 : hs + (uint32_t)(half * C::NBATCH + kDrainBlk) * kBlockBytes + (uint32_t)quarter * 4096u;
         auto drain_y = [&](uint32_t t_idx, int32_t grow) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
@@ -448,6 +468,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 ptx::tmem_ld_32x32(lane_base + col0, ra);
                 ptx::tmem_ld_32x32(lane_base + col0 + 32, rb);
                 ptx::tmem_ld_wait();
+                if constexpr (FP8) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        ra[i] = __float_as_uint(__uint_as_float(ra[i]) * y_scale);
+                        rb[i] = __float_as_uint(__uint_as_float(rb[i]) * y_scale);
+                    }
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + ((i ^ (lane & 7)) << 4)),
@@ -489,11 +516,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
 #pragma unroll 1
                 for (int j = 0; j < C::NBATCH && ok; ++j) {
                     // 32 rows x 64 columns of the hidden accumulator -> registers
-                    const int blk = half * C::NBATCH + j;        // hidden block = 64 channels
+                    const int blk = half * C::NBATCH + j;        // hidden block = 64 channels (FP8: column batch)
                     // Y of the previous tile is complete about now (its last GEMM2 was queued right
                     // after this tile's first GEMM1): store it before this warp's last batch of the
                     // chunk is loaded, while no accumulator values are held in registers
-                    if (j == C::NBATCH - 1 && c == 0 && ti > 0) {
+                    // (FP8: before the first batch -- the staging piece is the block this warp is about to write)
+                    if (j == (FP8 ? 0 : C::NBATCH - 1) && c == 0 && ti > 0) {
                         drain_y((uint32_t)(ti - 1), prev_row);
                         if (!ok) break;
                     }
@@ -506,6 +534,31 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                         // the accumulator is in registers: GEMM1 of the next chunk may start
                         ptx::tc_fence_before_sync();
                         warp_arrive(&misc->h_tmem_empty);
+                    }
+                    if constexpr (FP8) {
+                        // 64 columns -> 64 e4m3 bytes = chunks 4j .. 4j+3 of this row of hidden block `half`
+                        uint32_t p8[16];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            p8[i] = gelu_pack_e4m3x4(__uint_as_float(h0[4 * i]) * a_scale, __uint_as_float(h0[4 * i + 1]) * a_scale,
+                                                     __uint_as_float(h0[4 * i + 2]) * a_scale, __uint_as_float(h0[4 * i + 3]) * a_scale, h_inv);
+                            p8[8 + i] = gelu_pack_e4m3x4(__uint_as_float(h1[4 * i]) * a_scale, __uint_as_float(h1[4 * i + 1]) * a_scale,
+                                                         __uint_as_float(h1[4 * i + 2]) * a_scale, __uint_as_float(h1[4 * i + 3]) * a_scale, h_inv);
+                        }
+                        if (j == 0 && !warp_wait(&misc->hs_empty[half], (g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t hrow8 = hs + half * kBlockBytes + row * 128;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t dst = hrow8 + (((4 * j + i) ^ (row & 7)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p8[4 * i]),
+                                         "r"(p8[4 * i + 1]), "r"(p8[4 * i + 2]), "r"(p8[4 * i + 3])
+                                         : "memory");
+                        }
+                        if (j == C::NBATCH - 1) {
+                            ptx::fence_proxy_async_smem();
+                            warp_arrive(&misc->hs_full[half]);
+                        }
+                        continue;
                     }
                     uint32_t pk[32];
 #pragma unroll
@@ -576,13 +629,37 @@ int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, 
     if (grid < 1) grid = 1;
     LaunchScope ls(ctx, KS_FFN_MAIN, st);
     kern<<<grid, kThreads, Cfg<D>::SMEM_BYTES, st>>>(m1, m2a, m2b, (const __nv_bfloat16*)a.X,
-                                                      (__nv_bfloat16*)a.Y, plan, d.n_lists, kc_pad, a.status);
+                                                      (__nv_bfloat16*)a.Y, plan, d.n_lists, kc_pad, a.status, 1.f, 1.f, 1.f);
+    return SENTRY_OK;
+}
+
+// FP8 (e4m3 bytes): the weight maps describe the same bytes as 16-bit elements, two e4m3 each.
+int launch_fp8(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c, int kc_pad,
+               int max_tiles, cudaStream_t st) {
+    constexpr int D = 256;
+    const sentry_ffn_desc& d = a.d;
+    CUtensorMap m1, m2a, m2b;
+    const uint64_t r1 = (uint64_t)d.n_lists * kc_pad, r2 = (uint64_t)d.n_lists * D;
+    if (!make_weight_map(&m1, w1c, r1, D / 2, 256)) return SENTRY_ERR_CUDA;
+    if (!make_weight_map(&m2a, w2c, r2, kc_pad / 2, 256)) return SENTRY_ERR_CUDA;
+    if (!make_weight_map(&m2b, w2c, r2, kc_pad / 2, 128)) return SENTRY_ERR_CUDA;
+    auto kern = ffn_tc_kernel<D, false, true>;
+    SENTRY_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D, true>::SMEM_BYTES));
+    int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;
+    if (grid < 1) grid = 1;
+    LaunchScope ls(ctx, KS_FFN_MAIN, st);
+    kern<<<grid, kThreads, Cfg<D, true>::SMEM_BYTES, st>>>(m1, m2a, m2b, (const __nv_bfloat16*)a.X, (__nv_bfloat16*)a.Y,
+                                                           plan, d.n_lists, kc_pad, a.status, a.fp8_a_scale,
+                                                           a.fp8_h_inv, a.fp8_y_scale);
     return SENTRY_OK;
 }
 
 }  // namespace
 
+bool ffn_tc_fp8_supported(const sentry_ffn_desc& d) { return d.dtype == SENTRY_FP8_E4M3 && d.D == 256; }
+
 bool ffn_tc_supported(const sentry_ffn_desc& d) {
+    if (d.dtype == SENTRY_FP8_E4M3) return d.D == 256;
     return (d.dtype == SENTRY_BF16 || d.dtype == SENTRY_F16) && (d.D == 128 || d.D == 256 || d.D == 384);
 }
 
@@ -603,6 +680,13 @@ int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* 
     int rc;
     // the two 16-bit types share everything but the operand format of the UMMAs and the roundings
     // (X, Y and the weight tiles are moved as 16-bit words)
+    if (a.d.dtype == SENTRY_FP8_E4M3) {
+        if (!ffn_tc_fp8_supported(a.d)) return SENTRY_ERR_UNSUPPORTED;
+        rc = launch_fp8(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st);
+        if (rc != SENTRY_OK) return rc;
+        SENTRY_CUDA_TRY(cudaGetLastError());
+        return SENTRY_OK;
+    }
     const bool f16 = a.d.dtype == SENTRY_F16;
     switch (a.d.D) {
         case 128: rc = f16 ? launch_d<128, true>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)

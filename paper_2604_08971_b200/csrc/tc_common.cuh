@@ -2,6 +2,7 @@
 // arithmetic, warp-level barrier helpers, single-lane election and the TMA tensor-map encoder.
 #pragma once
 #include <cuda.h>
+#include <cuda_fp8.h>
 #include <math.h>
 
 #include "common.cuh"
@@ -77,6 +78,17 @@ __device__ __forceinline__ uint32_t gelu_pack_16x2(float z0, float z1) {
     } else {
         return gelu_erf_fast_bf16x2(z0, z1);
     }
+}
+
+// gelu of four values by the tanh form, times `post`, rounded to FP8 e4m3 (saturating at +-448) and
+// packed low byte first.
+__device__ __forceinline__ uint32_t gelu_pack_e4m3x4(float z0, float z1, float z2, float z3, float post) {
+    float g0, g1, g2, g3;
+    gelu_erf_fast_x2(z0, z1, g0, g1);
+    gelu_erf_fast_x2(z2, z3, g2, g3);
+    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(g0 * post, g1 * post), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(g2 * post, g3 * post), __NV_SATFINITE, __NV_E4M3);
+    return lo | (hi << 16);
 }
 
 __device__ __forceinline__ void cp_async_wait_pending(int n) {

@@ -541,3 +541,45 @@ def test_e4m3_decode_matches_the_library_and_the_format_constants():
     # dequantisation: fp32 product, one rounding to the compute type
     w = oracle.dequantise_e4m3(np.array([0x38, 0x3C, 0xC9], dtype=np.uint8), 0.5, "bf16")
     np.testing.assert_array_equal(w.float().numpy(), np.array([0.5, 0.75, -2.25], dtype=np.float32))   # 0xC9 = -(1 + 1/8) * 2^(9-7)
+
+
+def test_e4m3_encode_is_the_nearest_code_and_inverts_decode():
+    """Encoding against the library's conversion on a dense sweep inside the finite range, exact
+    ties (to even), saturation, and decode(encode(v)) == v for every representable value."""
+    codes = np.arange(256, dtype=np.uint8)
+    vals = oracle.e4m3_decode(codes)
+    finite = ~np.isnan(vals)
+    back = oracle.e4m3_encode(vals[finite])
+    np.testing.assert_array_equal(oracle.e4m3_decode(back), vals[finite])          # round trip (the two zeros included)
+    rng = np.random.default_rng(5)
+    sweep = np.concatenate([rng.uniform(-448, 448, 20000), rng.normal(0, 1, 20000), rng.normal(0, 0.01, 20000),
+                            np.array([0.0, 2.0 ** -10, 3 * 2.0 ** -10, 1.0625, 1.1875, 447.9, 0.0009765625 * 1.5])])
+    got = oracle.e4m3_decode(oracle.e4m3_encode(sweep))
+    lib = torch.from_numpy(sweep.astype(np.float32)).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    np.testing.assert_array_equal(got, lib)
+    # ties go to the even code: 1.0625 lies halfway between 1.0 (even) and 1.125; 1.1875 between 1.125 and 1.25 (even)
+    assert oracle.e4m3_decode(oracle.e4m3_encode([1.0625]))[0] == 1.0
+    assert oracle.e4m3_decode(oracle.e4m3_encode([1.1875]))[0] == 1.25
+    # beyond the largest finite value: saturation
+    np.testing.assert_array_equal(oracle.e4m3_decode(oracle.e4m3_encode([1e4, -1e4, 460.0])), [448.0, -448.0, 448.0])
+
+
+def test_ffn_fp8_reduces_to_library_matmuls_on_the_decoded_operands():
+    """With the requantisation of the hidden activations made lossless by construction (hidden
+    values that are exactly representable), the FP8 FFN equals library matmuls on the decoded
+    operands; in general it equals them once the hidden activations are passed through the
+    library's float8 rounding."""
+    rng = np.random.default_rng(9)
+    B, T, D, F, k = 2, 5, 16, 24, 10
+    Xq = oracle.e4m3_encode(rng.normal(0, 1, (B, T, D)))
+    W1q = oracle.e4m3_encode(rng.normal(0, 0.5, (D, F)))
+    W2q = oracle.e4m3_encode(rng.normal(0, 0.5, (F, D)))
+    kept = np.sort(rng.permutation(F)[:k]).astype(np.int32)[None, :]
+    sx, sw1, sw2, sh = 0.5, 0.25, 0.125, 0.03125
+    Y = oracle.ffn_fp8(Xq, W1q, W2q, kept, None, None, None, sx, sw1, sw2, sh)
+    X, W1, W2 = oracle.e4m3_decode(Xq), oracle.e4m3_decode(W1q), oracle.e4m3_decode(W2q)
+    z = (X @ W1[:, kept[0]]) * (sx * sw1)
+    g = 0.5 * z * (1.0 + erf(z / math.sqrt(2.0)))
+    hq = torch.from_numpy((g / sh).astype(np.float32)).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    want = (hq @ W2[kept[0], :]) * (sh * sw2)
+    np.testing.assert_allclose(Y, want, rtol=0, atol=1e-12)
