@@ -9,9 +9,13 @@ Inputs may be numpy arrays or torch CPU tensors of any float dtype; they are
 widened to float64 exactly (bf16, fp16 and fp32 values are representable), so the
 oracle sees the same numbers the GPU reads.
 
-Besides the wrapper, two numpy functions of their own: ``e4m3_decode`` (the FP8
-format written out from its definition; pinned against the library's float8
-conversion on all 256 codes, tests/test_oracle_pins.py) and ``dequantise_e4m3``.
+Besides the wrapper, numpy functions of their own for the FP8 point (Section 5):
+``e4m3_decode`` (the format written out from its definition; pinned against the
+library's float8 conversion on all 256 codes, tests/test_oracle_pins.py),
+``dequantise_e4m3``, ``e4m3_encode`` (nearest code, ties to even, saturating;
+pinned against the library's rounding on a dense sweep and on exact midpoints)
+and ``ffn_fp8`` (the pruned FFN with e4m3 operands, per-tensor scales and a
+requantised hidden tile; pinned against library matmuls on the decoded operands).
 """
 from __future__ import annotations
 
