@@ -703,49 +703,65 @@ def run_ours(args, w: synth.Workload):
     s_up, s_down = torch.cuda.Stream(), torch.cuda.Stream()
     kept_c_e2e = torch.empty_like(base.kept_c)
 
-    def e2e_step():
+    def e2e_steps(n):
+        """n steps, pipelined across chunks AND steps: chunk i of step s+1 is uploaded once the
+        kernels of chunk i of step s have read their inputs, and its kernels start once chunk i's
+        results of step s have left for the host.  Every step uploads all inputs and downloads all
+        results; only the order of independent copies and kernels overlaps."""
         cur = torch.cuda.current_stream()
         s_up.wait_stream(cur)
-        ups = []
-        with torch.cuda.stream(s_up):
-            for dst, src in zip(dsmall, small_in):
-                dst.copy_(src, non_blocking=True)
+        s_down.wait_stream(cur)
+        k_done = [None] * n_chunks
+        d_done = [None] * n_chunks
+        for _ in range(n):
+            ups = []
+            with torch.cuda.stream(s_up):
+                if k_done[-1] is not None:
+                    s_up.wait_event(k_done[-1])      # the small inputs are read by every chunk's kernels
+                for dst, src in zip(dsmall, small_in):
+                    dst.copy_(src, non_blocking=True)
+                for i in range(n_chunks):
+                    b0, b1 = bounds[i], bounds[i + 1]
+                    for dst, src in zip((base.Q, base.K, base.V, base.X), host_in):
+                        dst[b0:b1].copy_(src[b0:b1], non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(s_up)
+                    ups.append(ev)
             for i in range(n_chunks):
                 b0, b1 = bounds[i], bounds[i + 1]
-                for dst, src in zip((base.Q, base.K, base.V, base.X), host_in):
-                    dst[b0:b1].copy_(src[b0:b1], non_blocking=True)
-                ev = torch.cuda.Event()
-                ev.record(s_up)
-                ups.append(ev)
-        for i in range(n_chunks):
-            b0, b1 = bounds[i], bounds[i + 1]
-            cur.wait_event(ups[i])
-            sn.gate_attend_fwd(sh, w.k_h, base.Q[b0:b1], base.K[b0:b1], base.V[b0:b1], ids, masks[b0:b1], tbl, offs, c=w.c,
-                               score_mode=wb.score_mode, O=base.O[b0:b1], kept_heads=base.kept_h[b0:b1])
-            sn.gate_select(sc, subsets, w.k_c, kept=kept_c_e2e)
-            sn.ffn_fwd(base.X[b0:b1], W1, W2, kept_c_e2e, los[b0:b1], ids, masks[b0:b1], Y=base.Y[b0:b1])
-            ev = torch.cuda.Event()
-            ev.record(cur)
-            s_down.wait_event(ev)
-            with torch.cuda.stream(s_down):
-                host_out[0][b0:b1].copy_(base.O[b0:b1], non_blocking=True)
-                host_out[1][b0:b1].copy_(base.Y[b0:b1], non_blocking=True)
+                cur.wait_event(ups[i])
+                if d_done[i] is not None:
+                    cur.wait_event(d_done[i])        # O / Y of this chunk are about to be overwritten
+                sn.gate_attend_fwd(sh, w.k_h, base.Q[b0:b1], base.K[b0:b1], base.V[b0:b1], ids, masks[b0:b1], tbl, offs,
+                                   c=w.c, score_mode=wb.score_mode, O=base.O[b0:b1], kept_heads=base.kept_h[b0:b1])
+                sn.gate_select(sc, subsets, w.k_c, kept=kept_c_e2e)
+                sn.ffn_fwd(base.X[b0:b1], W1, W2, kept_c_e2e, los[b0:b1], ids, masks[b0:b1], Y=base.Y[b0:b1])
+                k_done[i] = torch.cuda.Event()
+                k_done[i].record(cur)
+                s_down.wait_event(k_done[i])
+                with torch.cuda.stream(s_down):
+                    host_out[0][b0:b1].copy_(base.O[b0:b1], non_blocking=True)
+                    host_out[1][b0:b1].copy_(base.Y[b0:b1], non_blocking=True)
+                    d_done[i] = torch.cuda.Event()
+                    d_done[i].record(s_down)
         cur.wait_stream(s_down)
-        torch.cuda.synchronize()
+        cur.wait_stream(s_up)
 
     n_e2e = max(3, min(args.steps, 20))
     e2e_tokens, e2e_ms = None, None
     if not args.no_e2e:
-        for _ in range(3):
-            e2e_step()
+        e2e_steps(3)
         barrier_sync()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
-        for _ in range(n_e2e):
-            e2e_step()
+        e2e_steps(n_e2e)
         ev1.record()
         barrier_sync()
         e2e_tokens, e2e_ms = aggregate(float(wm["tokens"]) * n_e2e, ev0.elapsed_time(ev1), dev)
+        torch.cuda.synchronize()
+        # what reached the host is what the device holds (outside the timed region)
+        if not (torch.equal(host_out[0], base.O.cpu()) and torch.equal(host_out[1], base.Y.cpu())):
+            raise RuntimeError("end-to-end leg: host results differ from the device buffers")
     status = wb.status()
     launches = wb.launches
     graphs_on = wb.graphs is not None
@@ -844,7 +860,7 @@ def run_ours(args, w: synth.Workload):
         "materialised_once": once, "chained_layer": chained,
         "e2e": None if e2e_ms is None else {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": n_e2e,
-                "pipeline": "%d sample chunks; upload, kernels and download on three streams" % n_chunks},
+                "pipeline": "%d sample chunks; upload, kernels and download on three streams, consecutive steps overlapping chunk by chunk" % n_chunks},
         "gpu_launches": launches * args.steps,
         "clocks": clocks, "roofline": roof, "stages": stages, "kernels": per_kernel,
         "configs": table,
