@@ -41,7 +41,7 @@ SEPARATE_GATE = False     # set from --separate-gate
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
 # keyed by (kernel slot, workload); None once the kernel has changed since its capture.
-NCU_TRAFFIC = {("attend_core", "cfg4_full_layer"): 40.74e6, ("ffn_main", "cfg4_full_layer"): 36.64e6}
+NCU_TRAFFIC = {("attend_core", "cfg4_full_layer"): 40.77e6, ("ffn_main", "cfg4_full_layer"): 36.67e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -899,6 +899,8 @@ def main():
                          "(score_mode 2), plainly transposed (score_mode 2), or query-major as generated (score_mode 0); "
                          "auto: arranged where K and V of a group fit in shared memory, transposed otherwise; "
                          "the sampled sets are the same")
+    ap.add_argument("--side", default=None, choices=["moe", "ffn_fp8"],
+                    help="run only this side measurement of the configs table and print its object (for profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     global TABLE_LAYOUT, GATE_MULTI, LONG_SELECT, SEPARATE_GATE
@@ -907,6 +909,16 @@ def main():
     TABLE_LAYOUT = args.table_layout
     GATE_MULTI = args.gate_multi
     w = synth.by_name(args.config)
+    if args.side is not None:
+        import paper_2604_08971_b200 as sentry
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: libsentry has no CPU fallback")
+        sentry.build()
+        torch.cuda.set_device(0)
+        peaks, _ = load_peaks()
+        fn = {"moe": quick_moe, "ffn_fp8": quick_fp8_ffn}[args.side]
+        print(json.dumps({args.side: fn(sentry, "cuda:0", 0, peaks)}))
+        return
     if args.impl == "reference":
         run_reference(args, w)
     else:
