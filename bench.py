@@ -597,6 +597,9 @@ def quick_fp8_ffn(sentry, dev: str, local_rank: int, peaks):
         ms = float(np.median(blocks))
         out[name] = {"ms_per_call": ms, "tokens_per_s": w.B * w.T / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
                      "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+        if name == "fp8_e4m3":
+            # peak of its own operand type: the measured bf16 figure x the nominal 8-bit : 16-bit ratio (2)
+            out[name]["frac_of_fp8_peak"] = out[name]["frac_of_bf16_peak"] / 2.0
     out["device_status"] = sn.last_status()
     sn.close()
     return out
