@@ -56,7 +56,7 @@ struct Cfg {
     static constexpr int NHS = CH / EPB;               // hidden blocks per chunk
     static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
     static constexpr int SPG = (D == 384) ? 3 : KB1;   // weight stages per chunk of GEMM1 (= of GEMM2)
-    static_assert(!FP8 || D == 256, "the FP8 form is built for d_model = 256");
+    static_assert(!FP8 || D == 256 || D == 128, "the FP8 form is built for d_model = 128 and 256");
     static constexpr int OFF_H = NXS * kBlockBytes;
     static constexpr int OFF_W = OFF_H + NHS * kBlockBytes;
     static constexpr int OFF_MISC = OFF_W + kStages * kStageBytes;
@@ -634,9 +634,9 @@ int launch_d(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, 
 }
 
 // FP8 (e4m3 bytes): the weight maps describe the same bytes as 16-bit elements, two e4m3 each.
+template <int D>
 int launch_fp8(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c, void* w2c, int kc_pad,
                int max_tiles, cudaStream_t st) {
-    constexpr int D = 256;
     const sentry_ffn_desc& d = a.d;
     CUtensorMap m1, m2a, m2b;
     const uint64_t r1 = (uint64_t)d.n_lists * kc_pad, r2 = (uint64_t)d.n_lists * D;
@@ -656,10 +656,10 @@ int launch_fp8(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c
 
 }  // namespace
 
-bool ffn_tc_fp8_supported(const sentry_ffn_desc& d) { return d.dtype == SENTRY_FP8_E4M3 && d.D == 256; }
+bool ffn_tc_fp8_supported(const sentry_ffn_desc& d) { return d.dtype == SENTRY_FP8_E4M3 && (d.D == 256 || d.D == 128); }
 
 bool ffn_tc_supported(const sentry_ffn_desc& d) {
-    if (d.dtype == SENTRY_FP8_E4M3) return d.D == 256;
+    if (d.dtype == SENTRY_FP8_E4M3) return d.D == 256 || d.D == 128;
     return (d.dtype == SENTRY_BF16 || d.dtype == SENTRY_F16) && (d.D == 128 || d.D == 256 || d.D == 384);
 }
 
@@ -682,7 +682,8 @@ int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* 
     // (X, Y and the weight tiles are moved as 16-bit words)
     if (a.d.dtype == SENTRY_FP8_E4M3) {
         if (!ffn_tc_fp8_supported(a.d)) return SENTRY_ERR_UNSUPPORTED;
-        rc = launch_fp8(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st);
+        rc = a.d.D == 256 ? launch_fp8<256>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)
+                          : launch_fp8<128>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st);
         if (rc != SENTRY_OK) return rc;
         SENTRY_CUDA_TRY(cudaGetLastError());
         return SENTRY_OK;

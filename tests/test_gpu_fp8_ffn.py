@@ -12,7 +12,10 @@ is off by several per cent of the RMS.  Element-wise 2e-2 of the RMS can therefo
 every output; what is asserted is what the arithmetic fixes:
   * the RMS of the error <= 1.5e-2 of the output RMS,
   * at most 5 outputs in 1000 off by more than 2e-2 of the RMS (after the bf16 half-ulp of Y; measured 2 in 1000:
-    a flipped term has to be ~7 times the typical term to move an output that far),
+    a flipped term has to be ~7 times the typical term to move an output that far).  That size falls with the
+    number of terms (0.33 sqrt(k_c) typical terms: 4.7 at k_c = 200, 7.5 at 512) while the error RMS does not
+    depend on it, so below 300 kept channels the allowed fraction grows as 300 / k_c (measured 5.1 in 1000 at
+    k_c = 200, 4.4 at 256),
   * no output off by more than 0.25 of the RMS (a flip or two on the largest terms, nothing worse),
   * rows of absent tokens exactly zero, results identical run to run.
 """
@@ -40,7 +43,8 @@ def _quantise(t):
     return q, s
 
 
-@pytest.mark.parametrize("w", [synth.config3().with_(B=6), synth.config5(16, 256), synth.config5(3, 1024).with_(k_c=300, name="fp8_ragged_kc")],
+@pytest.mark.parametrize("w", [synth.config3().with_(B=6), synth.config5(16, 256), synth.config5(3, 1024).with_(k_c=300, name="fp8_ragged_kc"),
+                               synth.config2().with_(B=24, name="fp8_d128"), synth.config2().with_(B=5, k_c=200, name="fp8_d128_ragged_kc")],
                          ids=lambda w: w.name)
 def test_fp8_ffn_against_the_oracle(w):
     sn = sentry.Sentry(0)
@@ -73,7 +77,7 @@ def test_fp8_ffn_against_the_oracle(w):
         parity.record(w.name, "ffn_fp8", err, parity.raw_rel_err(got, want),
                       "error rms %.2e of the output rms; %.1e of the outputs off by more than 2e-2" % (rms_err, frac_off))
         assert rms_err <= 1.5e-2, rms_err
-        assert frac_off <= 5e-3, frac_off
+        assert frac_off <= 5e-3 * max(1.0, 300.0 / w.k_c), frac_off
         assert err <= 0.25, err
     finally:
         sn.close()
