@@ -29,19 +29,27 @@ moe_route_kernel(const int32_t* __restrict__ expert_ids, long long n_slots, int 
     const long long per_block = (long long)kPlanThreads * 8;
     const long long i0 = (long long)blockIdx.x * per_block;
     int my_e[8], my_pos[8];
+    const int lane = threadIdx.x & 31;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const long long i = i0 + (long long)j * kPlanThreads + threadIdx.x;
-        int e = -1;
-        if (i < n_slots) {
-            e = expert_ids[i];
-            if (e < -1 || e >= E) {
-                atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
-                e = -1;
-            }
+        my_e[j] = i < n_slots ? __ldg(expert_ids + i) : -1;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        int e = my_e[j];
+        if (e < -1 || e >= E) {
+            atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+            e = -1;
         }
         my_e[j] = e;
-        my_pos[j] = e >= 0 ? atomicAdd(&s_cnt[e], 1) : 0;
+        // one shared-memory atomic per (warp, expert): the lanes of a warp that go to the same
+        // expert take consecutive positions from their first lane's reservation
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        const int leader = __ffs(peers) - 1;
+        int base = 0;
+        if (lane == leader && e >= 0) base = atomicAdd(&s_cnt[e], __popc(peers));
+        my_pos[j] = __shfl_sync(0xffffffffu, base, leader) + __popc(peers & ((1u << lane) - 1u));
     }
     __syncthreads();
     if (phase == 0) {
@@ -157,16 +165,32 @@ moe_combine_kernel(const uint4* __restrict__ staged, const int32_t* __restrict__
         float acc[NV];
 #pragma unroll
         for (int c = 0; c < NV; ++c) acc[c] = 0.f;
-        for (int j = 0; j < top_k; ++j) {
-            const int e = expert_ids[t * top_k + j];
-            if (e < 0 || e >= E) continue;
-            const float g = weights[t * top_k + j];
-            float f[NV];
-            const uint4 raw = __ldg(&staged[(t * top_k + j) * vpr + v]);
-            if constexpr (sizeof(T) == 2 && !IS_BF16) unpack16_half(raw, f);
-            else unpack16(raw, f);
+        // four slots at a time: ids, weights and staged rows are requested together (a staged row is
+        // read whether or not its slot is routed -- the buffer is there -- and dropped afterwards, so
+        // that the row does not wait for the id); the sum runs in slot order
+        for (int j0 = 0; j0 < top_k; j0 += 4) {
+            int e[4];
+            float g[4];
+            uint4 raw[4];
 #pragma unroll
-            for (int c = 0; c < NV; ++c) acc[c] = fmaf(g, f[c], acc[c]);
+            for (int u = 0; u < 4; ++u) {
+                const int j = j0 + u;
+                e[u] = -1;
+                if (j < top_k) {
+                    e[u] = __ldg(expert_ids + t * top_k + j);
+                    g[u] = __ldg(weights + t * top_k + j);
+                    raw[u] = __ldg(&staged[(t * top_k + j) * vpr + v]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (e[u] < 0 || e[u] >= E) continue;
+                float f[NV];
+                if constexpr (sizeof(T) == 2 && !IS_BF16) unpack16_half(raw[u], f);
+                else unpack16(raw[u], f);
+#pragma unroll
+                for (int c = 0; c < NV; ++c) acc[c] = fmaf(g[u], f[c], acc[c]);
+            }
         }
         if constexpr (sizeof(T) == 2 && !IS_BF16) Y[i] = pack16_half(acc);
         else Y[i] = pack16(acc);
