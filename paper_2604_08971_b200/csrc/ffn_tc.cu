@@ -19,6 +19,10 @@
 // next chunk (or of the next tile's first chunk) before GEMM2 of the current one, so GEMM2
 // never waits for the GELU epilogue with nothing else queued.
 //
+// With d_model = 384 the tiles of a last, partial round are shared by three CTAs each when that
+// still fits one round: every one of the three forms the hidden activations, and accumulates
+// and stores one 128-column third of Y (see the kernel).
+//
 // Warp roles (512 threads): warps 0 and 2 = weight TMA producers (warp 0 owns TMEM),
 // warp 1 = UMMA issuer (warp 15 is idle), warps 3-6 = X row
 // gather, warps 7-14 = epilogue (two warps per TMEM lane quarter).  Producer and issuer warps stay
@@ -56,6 +60,7 @@ struct Cfg {
     static constexpr int NHS = CH / EPB;               // hidden blocks per chunk
     static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
     static constexpr int SPG = (D == 384) ? 3 : KB1;   // weight stages per chunk of GEMM1 (= of GEMM2)
+    static constexpr bool COLSPLIT = (D == 384) && !FP8;   // tail tiles shared by three CTAs, a third of Y each
     static_assert(!FP8 || D == 256 || D == 128, "the FP8 form is built for d_model = 128 and 256");
     static constexpr int OFF_H = NXS * kBlockBytes;
     static constexpr int OFF_W = OFF_H + NHS * kBlockBytes;
@@ -157,6 +162,19 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NC = kc_pad / C::CH;
     const int total_tiles = plan.tile_start[n_lists];
+    // Column-split tail (d_model = 384).  The tiles of the last, partial round leave most CTAs idle
+    // (340 tiles on 148 CTAs: 44 in the third round).  When three times their number still fits
+    // one round, each of them is taken by three CTAs: all three form the tile's hidden
+    // activations, and each accumulates and stores one 128-column third of Y (GEMM2 of a third =
+    // the N = 128 stage alone).  Nothing is exchanged; a third costs 4/6 of the tensor work of a
+    // whole tile.  Virtual tile v < full_v is tile v; the others are (tile, third) pairs.  A CTA's
+    // split tile, if it has one, is its last.
+    int full_v = total_tiles, n_vt = total_tiles;
+    if constexpr (C::COLSPLIT) {
+        const int rem = total_tiles % (int)gridDim.x;
+        if (rem > 0 && 3 * rem <= (int)gridDim.x) { full_v = total_tiles - rem; n_vt = full_v + 3 * rem; }
+    }
+    auto tile_of = [&](int v) { return v < full_v ? v : full_v + (v - full_v) / 3; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -189,7 +207,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
 
     constexpr int SPG = C::SPG;
     const uint32_t mb = ptx::smem_u32(misc);
-    const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_tiles = (n_vt - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int last_v = (int)blockIdx.x + (my_tiles - 1) * (int)gridDim.x;
+    const int my_third = (my_tiles > 0 && last_v >= full_v) ? (last_v - full_v) % 3 : -1;   // -1: no split tile
     const uint32_t n_chunks = (uint32_t)(my_tiles * NC);
     // Ring order: GEMM1 of chunk 0; then, per chunk q >= 1, GEMM1 of q and GEMM2 of q-1; at the
     // end GEMM2 of the last chunk.  Producers and issuers walk it as "group q = GEMM1(q), GEMM2(q-1)"
@@ -231,7 +251,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 l_last = l_cur;
                 if (q < n_chunks) {
                     int row0, n_rows;
-                    ffn_tile_lookup(plan, n_lists, (int)blockIdx.x + (int)ti * (int)gridDim.x, kTileRows, l_cur, row0, n_rows);
+                    ffn_tile_lookup(plan, n_lists, tile_of((int)blockIdx.x + (int)ti * (int)gridDim.x), kTileRows, l_cur, row0, n_rows);
                 }
             }
             if (q < n_chunks) {
@@ -247,6 +267,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             }
             if (q > 0) {
                 const int pl = c ? l_cur : l_last, x = (c ? c - 1 : NC - 1) * C::CH16, y = pl * D;
+                if (C::COLSPLIT && my_third >= 0 && (int)(c ? ti : ti - 1) == my_tiles - 1) {
+                    // a third of Y: one N = 128 stage (both K blocks of the chunk)
+                    if ((n & 1u) == me) ok = stage(n, &tm_w2_128, x, x + 64, y + 128 * my_third);
+                    n += 1;
+                    if (++c == NC) { c = 0; ++ti; }
+                    continue;
+                }
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
                     if (ok && ((n + i) & 1u) == me) {
@@ -349,6 +376,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 const bool first = (pc == 0), last = (pc == NC - 1);
                 const uint32_t ye = first ? MISC_BAR(mb, y_empty) : 0u, yp = (pti & 1u) ^ 1u;
                 const uint32_t yf = last ? MISC_BAR(mb, y_full) : 0u;
+                if (C::COLSPLIT && my_third >= 0 && (int)pti == my_tiles - 1) {
+                    ok = stage(n, tmem + 128u * (uint32_t)my_third, hs_lo, hs_lo + kBlkLo, idesc128, first,
+                               MISC_BAR(mb, hs_full), gp, MISC_BAR(mb, hs_full) + 8u, gp, ye, yp, first,
+                               MISC_BAR(mb, hs_empty), MISC_BAR(mb, hs_empty) + 8u, yf);
+                    n += 1;
+                    if (++c == NC) { c = 0; ++ti; }
+                    continue;
+                }
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
                     if (!ok) continue;
@@ -394,9 +429,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             warp_arrive(&misc->x_full[published % C::NXS]);
             ++published;
         };
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int vt = blockIdx.x; vt < n_vt && ok; vt += gridDim.x) {
             int l, row0, n_rows;
-            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
+            ffn_tile_lookup(plan, n_lists, tile_of(vt), kTileRows, l, row0, n_rows);
             int32_t rows[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -449,22 +484,24 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         // (FP8: a warp writes one 128-channel hidden block, rows of its own quarter: that piece)
         const uint32_t stg = FP8 ? hs + (uint32_t)half * kBlockBytes + (uint32_t)quarter * 4096u
                                  : hs + (uint32_t)(half * C::NBATCH + kDrainBlk) * kBlockBytes + (uint32_t)quarter * 4096u;
-        auto drain_y = [&](uint32_t t_idx, int32_t grow) {
+        auto drain_y = [&](uint32_t t_idx, int32_t grow, int third) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
             ptx::tc_fence_after_sync();
             // 64 columns per pass: two TMEM loads and one wait, bf16 rows through the staging
             // piece, then whole 128-byte row segments to global memory.  The registers a TMEM
             // load writes are not named again before its wait.
-            constexpr int NP = D / 128;
+            // a whole tile: this half's D/2 columns in passes of 64; a third: 64 of its 128 columns
+            const int NP = third < 0 ? D / 128 : 1;
+            const int cbase = third < 0 ? half * (D / 2) : third * 128 + half * 64;
             const int ch = lane & 7;
             int32_t grs[8];
 #pragma unroll
             for (int step = 0; step < 8; ++step) grs[step] = __shfl_sync(0xffffffffu, grow, step * 4 + (lane >> 3));
-            __nv_bfloat16* ycol = Y + half * (D / 2) + ch * 8;
+            __nv_bfloat16* ycol = Y + cbase + ch * 8;
 #pragma unroll 1
             for (int pass = 0; pass < NP; ++pass) {
                 uint32_t ra[32], rb[32];
-                const int col0 = half * (D / 2) + pass * 64;
+                const int col0 = cbase + pass * 64;
                 ptx::tmem_ld_32x32(lane_base + col0, ra);
                 ptx::tmem_ld_32x32(lane_base + col0 + 32, rb);
                 ptx::tmem_ld_wait();
@@ -505,9 +542,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             ptx::tc_fence_before_sync();
             warp_arrive(&misc->y_empty);
         };
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++ti) {
+        for (int vt = blockIdx.x; vt < n_vt && ok; vt += gridDim.x, ++ti) {
             int l, row0, n_rows;
-            ffn_tile_lookup(plan, n_lists, tile, kTileRows, l, row0, n_rows);
+            ffn_tile_lookup(plan, n_lists, tile_of(vt), kTileRows, l, row0, n_rows);
             prev_row = my_row;
             my_row = row < n_rows ? (plan.rowout ? plan.rowout : plan.rowidx)[row0 + row] : -1;
             for (int c = 0; c < NC && ok; ++c, ++g) {
@@ -522,7 +559,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     // chunk is loaded, while no accumulator values are held in registers
                     // (FP8: before the first batch -- the staging piece is the block this warp is about to write)
                     if (j == (FP8 ? 0 : C::NBATCH - 1) && c == 0 && ti > 0) {
-                        drain_y((uint32_t)(ti - 1), prev_row);
+                        drain_y((uint32_t)(ti - 1), prev_row, -1);   // a split tile is the last one: never drained here
                         if (!ok) break;
                     }
                     uint32_t h0[32], h1[32];
@@ -580,7 +617,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 }
             }
         }
-        if (ok && ti > 0) drain_y(ti - 1, my_row);
+        if (ok && ti > 0) drain_y(ti - 1, my_row, my_third);
     }
 
     cta_teardown(abort_flag, status, tmem, kTmemCols);
