@@ -830,13 +830,34 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
     }
     __syncthreads();   // s_mean is complete: warps without a row tile go straight to the fill
 
-    // ---- Eq. 6 on the active rows: row tiles (head slot, 16 rows) over the warps
-    const int WT = (min(U, kMaxActive) + 15) / 16;
-    const int n_tiles = rk * WT;
+    // ---- Eq. 6 on the active rows: tiles of 16 rows over the warps.  The heads of a group share K
+    // and V, so a tile may hold rows of several heads: the rk * U active rows are packed back to
+    // back (U = 35: 7 tiles for three heads instead of 3 x 3, the last of each nearly empty).
+    const int Ue = min(U, kMaxActive);
+    const int n_rows_act = rk * Ue;
+    const int n_tiles = (n_rows_act + 15) / 16;
     const int gq = lane >> 2, tq = lane & 3;
     const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;  // scale * log2(e)
     for (int tt = warp; tt < n_tiles; tt += nwarps) {
-        const int hh = tt / WT, row0 = (tt % WT) * 16;
+        // this lane's two rows (gq and gq + 8 of the tile): token, head, output head slot
+        int row_t[2], row_kh[2];
+        const __nv_bfloat16* row_q[2];
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int r = tt * 16 + gq + half * 8;
+            int hh = 0, t = -1;
+            if (r < n_rows_act) {
+                hh = r / Ue;
+                t = s_act[hh][r - hh * Ue];
+            }
+            int h_sel = hs[0], kh_sel = khs[0];
+#pragma unroll
+            for (int j = 1; j < kMaxRK; ++j)
+                if (hh == j) { h_sel = hs[j]; kh_sel = khs[j]; }
+            row_t[half] = t;
+            row_kh[half] = kh_sel;
+            row_q[half] = Q + ((size_t)b * Hq + h_sel) * Tlen * D;
+        }
         uint32_t qf[KS][4];
         float acc[NT][4];
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
@@ -848,13 +869,11 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         for (int ks = 0; ks < KS; ++ks)
 #pragma unroll
             for (int e = 0; e < 4; ++e) qf[ks][e] = 0u;
-        const __nv_bfloat16* Qh = Q + ((size_t)b * Hq + hs[hh]) * Tlen * D;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-            const int a = row0 + gq + half * 8;
-            const int t = a < kMaxActive ? s_act[hh][a] : -1;
+            const int t = row_t[half];
             if (t >= 0) {
-                const uint32_t* qrow = reinterpret_cast<const uint32_t*>(Qh + (size_t)t * D);
+                const uint32_t* qrow = reinterpret_cast<const uint32_t*>(row_q[half] + (size_t)t * D);
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     qf[ks][half] = __ldg(qrow + ks * 8 + tq);          // cols 16ks + 2t, +1
@@ -947,17 +966,15 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
             }
         }
         // normalise and store this tile's rows
-        __nv_bfloat16* Oh = O + ((size_t)b * k_h + khs[hh]) * Tlen * D;
 #pragma unroll
         for (int h2 = 0; h2 < 2; ++h2) {
             float l = l_run[h2];
             l += __shfl_xor_sync(0xffffffffu, l, 1);
             l += __shfl_xor_sync(0xffffffffu, l, 2);
-            const int a = row0 + gq + h2 * 8;
-            const int t = a < kMaxActive ? s_act[hh][a] : -1;
+            const int t = row_t[h2];
             if (t < 0) continue;
             const float inv = 1.0f / l;
-            uint32_t* orow = reinterpret_cast<uint32_t*>(Oh + (size_t)t * D);
+            uint32_t* orow = reinterpret_cast<uint32_t*>(O + ((size_t)b * k_h + row_kh[h2]) * Tlen * D + (size_t)t * D);
 #pragma unroll
             for (int n = 0; n < NT; ++n)
                 orow[n * 4 + tq] = pack2(acc[n][2 * h2] * inv, acc[n][2 * h2 + 1] * inv);
