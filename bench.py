@@ -41,7 +41,7 @@ SEPARATE_GATE = False     # set from --separate-gate
 ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
 # keyed by (kernel slot, workload); None once the kernel has changed since its capture.
-NCU_TRAFFIC = {("attend_core", "cfg4_full_layer"): 40.77e6, ("ffn_main", "cfg4_full_layer"): 36.67e6}
+NCU_TRAFFIC = {("attend_core", "cfg4_full_layer"): 41.47e6, ("ffn_main", "cfg4_full_layer"): 36.74e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
