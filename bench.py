@@ -283,14 +283,25 @@ class Workbench:
     describes for a fixed set of modality masks and a fixed budget."""
 
     def __init__(self, sentry, w: synth.Workload, dev: str, local_rank: int, rank: int, overlap: bool,
-                 use_graph: bool, attend_kernel: int, materialise_once: bool = False, max_sets: int = 16):
+                 use_graph: bool, attend_kernel: int, materialise_once: bool = False, max_sets: int = 16,
+                 lanes: int = 1):
         self.sentry, self.w, self.dev = sentry, w, dev
-        self.sn = sentry.Sentry(local_rank)
-        self.sn2 = sentry.Sentry(local_rank) if overlap else self.sn
-        for c in (self.sn, self.sn2):
-            c.set_attend_kernel(attend_kernel)
-            c.set_option(sentry.OPT_LONG_SELECT, LONG_SELECT)
-        self.branch = torch.cuda.Stream() if overlap else None
+        # lanes > 1: consecutive steps (independent batches, different buffer sets) are issued on
+        # `lanes` streams in turn, each lane with library contexts (scratch) of its own, so that
+        # one step's tail and the next step's start may share the GPU
+        self.lanes = max(1, lanes)
+        self.ctx = []
+        for _ in range(self.lanes):
+            a = sentry.Sentry(local_rank)
+            b = sentry.Sentry(local_rank) if overlap else a
+            for c in (a, b):
+                c.set_attend_kernel(attend_kernel)
+                c.set_option(sentry.OPT_LONG_SELECT, LONG_SELECT)
+            self.ctx.append((a, b))
+        self.sn, self.sn2 = self.ctx[0]
+        self.branches = [torch.cuda.Stream() if overlap else None for _ in range(self.lanes)]
+        self.branch = self.branches[0]
+        self.lane_streams = [torch.cuda.Stream() for _ in range(self.lanes)] if self.lanes > 1 else []
         self.once = materialise_once
         self.n_s_of = lambda tv: sentry.num_active_queries(tv, w.c)
         inp = synth.generate(w.with_(seed=w.seed + 1000 * rank), self.n_s_of, device=dev)
@@ -319,25 +330,27 @@ class Workbench:
         base = DeviceSet(inp, dev)
         self.set_bytes = base.nbytes()
         self.n_sets = 1 if self.set_bytes >= 2 * L2_BYTES else int(min(max_sets, -(-2 * L2_BYTES // self.set_bytes)))
+        self.n_sets = -(-self.n_sets // self.lanes) * self.lanes   # set j always runs on lane j % lanes
         self.sets = [base] + [DeviceSet(inp, dev, base) for _ in range(self.n_sets - 1)]
         self.launches = 0
         self.packed = None
         if self.once:
             self.sn2.gate_select(self.sc, self.subsets, w.k_c, kept=base.kept_c)
             self.packed = self.sn2.ffn_prepack(self.W1, self.W2, base.kept_c)
-        self.step(self.sets[0], count=True)          # sizes the workspaces before any capture
+        for lane in range(self.lanes):               # sizes the workspaces before any capture
+            self.step(self.sets[lane], count=True, lane=lane)
         torch.cuda.synchronize()
-        assert self.sn.last_status() == 0 and self.sn2.last_status() == 0, "device status word set during warm-up"
+        assert self.status() == 0, "device status word set during warm-up"
         self.graphs = None
         if use_graph:
             self.graphs = []
             side = torch.cuda.Stream()
             side.wait_stream(torch.cuda.current_stream())
             with torch.cuda.stream(side):
-                for s_ in self.sets:
+                for j, s_ in enumerate(self.sets):
                     g = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(g, stream=side):
-                        self.step(s_)
+                        self.step(s_, lane=j % self.lanes)
                     self.graphs.append(g)
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
@@ -355,19 +368,21 @@ class Workbench:
         ctx.ffn_fwd(s.X, self.W1, self.W2, s.kept_c, self.los, self.ids, self.masks, Y=s.Y)
         return n + ctx.last_launch_count()
 
-    def step(self, s: DeviceSet, count=False, fork=True):
-        w, sn = self.w, self.sn
+    def step(self, s: DeviceSet, count=False, fork=True, lane=0):
+        w = self.w
+        sn, sn2 = self.ctx[lane]
+        branch = self.branches[lane]
         n = 0
-        two = fork and self.branch is not None
+        two = fork and branch is not None
         multi = GATE_MULTI and not self.once
         if multi:   # heads and channels selected by one launch, ahead of the fork
             sn.gate_select_multi([(self.sh, self.masks, w.k_h, 0, s.kept_h), (self.sc, self.subsets, w.k_c, 0, s.kept_c)])
             n += sn.last_launch_count()
         if two:
             cur = torch.cuda.current_stream()
-            self.branch.wait_stream(cur)
-            with torch.cuda.stream(self.branch):
-                n += self.ffn_branch(s, self.sn2, gated=multi)
+            branch.wait_stream(cur)
+            with torch.cuda.stream(branch):
+                n += self.ffn_branch(s, sn2, gated=multi)
         if not multi and not SEPARATE_GATE:
             # head selection and attention in one call (one launch where K and V of a group fit in shared memory)
             sn.gate_attend_fwd(self.sh, w.k_h, s.Q, s.K, s.V, self.ids, self.masks, self.tbl, self.offs, c=w.c,
@@ -381,18 +396,32 @@ class Workbench:
                           score_mode=self.score_mode)
             n += sn.last_launch_count()
         if two:
-            torch.cuda.current_stream().wait_stream(self.branch)
+            torch.cuda.current_stream().wait_stream(branch)
         else:
             n += self.ffn_branch(s, sn, gated=multi)
         if count:
             self.launches = n
 
     def run_steps(self, n, start=0):
+        if self.lanes == 1:
+            for i in range(n):
+                if self.graphs is not None:
+                    self.graphs[(start + i) % self.n_sets].replay()
+                else:
+                    self.step(self.sets[(start + i) % self.n_sets])
+            return
+        cur = torch.cuda.current_stream()
+        for ls in self.lane_streams:
+            ls.wait_stream(cur)
         for i in range(n):
-            if self.graphs is not None:
-                self.graphs[(start + i) % self.n_sets].replay()
-            else:
-                self.step(self.sets[(start + i) % self.n_sets])
+            j = (start + i) % self.n_sets
+            with torch.cuda.stream(self.lane_streams[j % self.lanes]):
+                if self.graphs is not None:
+                    self.graphs[j].replay()
+                else:
+                    self.step(self.sets[j], lane=j % self.lanes)
+        for ls in self.lane_streams:
+            cur.wait_stream(ls)
 
     def time_blocks(self, steps: int, replays: int, warmup: int):
         """`replays` blocks of `steps` steps each, every block bracketed by a barrier and a device
@@ -486,12 +515,16 @@ class Workbench:
         return work_model(self.w, self.inp.masks, kept_h_host, self.n_s_of)
 
     def status(self):
-        return self.sn.last_status() | self.sn2.last_status()
+        st = 0
+        for a, b in self.ctx:
+            st |= a.last_status() | b.last_status()
+        return st
 
     def close(self):
-        if self.sn2 is not self.sn:
-            self.sn2.close()
-        self.sn.close()
+        for a, b in self.ctx:
+            if b is not a:
+                b.close()
+            a.close()
         self.graphs = None
         self.sets = None
         torch.cuda.empty_cache()
@@ -610,7 +643,7 @@ def quick_config(sentry, name: str, dev: str, local_rank: int, peaks, args):
     least ~10 ms, plus the per-kernel pass."""
     w = synth.by_name(name)
     wb = Workbench(sentry, w, dev, local_rank, 0, not args.no_overlap, not args.no_graph,
-                   ATTEND_KERNELS[args.attend_kernel], max_sets=8)
+                   ATTEND_KERNELS[args.attend_kernel], max_sets=8, lanes=args.lanes)
     wm = wb.work()
     probe = wb.time_blocks(5, 1, 3)[0] / 5
     steps = int(max(5, min(400, 10.0 / max(probe, 1e-3))))
@@ -642,7 +675,7 @@ def run_ours(args, w: synth.Workload):
     sampler.start()
 
     wb = Workbench(sentry, w, dev, local_rank, rank, not args.no_overlap, not args.no_graph,
-                   ATTEND_KERNELS[args.attend_kernel])
+                   ATTEND_KERNELS[args.attend_kernel], lanes=args.lanes)
     sn, inp, base = wb.sn, wb.inp, wb.sets[0]
     n_sets, set_bytes = wb.n_sets, wb.set_bytes
 
@@ -679,7 +712,7 @@ def run_ours(args, w: synth.Workload):
     once = None
     if world == 1 and not args.no_once:
         wb1 = Workbench(sentry, w, dev, local_rank, rank, not args.no_overlap, not args.no_graph,
-                        ATTEND_KERNELS[args.attend_kernel], materialise_once=True)
+                        ATTEND_KERNELS[args.attend_kernel], materialise_once=True, lanes=args.lanes)
         b1 = wb1.time_blocks(args.steps, max(3, args.replays // 2 + 1), args.warmup)
         ms1 = float(np.median(b1)) / args.steps
         once = {"value": wm["tokens"] / (ms1 * 1e-3), "unit": "tokens/s", "ms_per_step": ms1,
@@ -687,6 +720,21 @@ def run_ours(args, w: synth.Workload):
                 "what": "channel gate selection and weight gather (sentry_ffn_prepack) run once before the timed "
                         "region; a step = head gate selection + attention + sentry_ffn_fwd_packed"}
         wb1.close()
+
+    # ---- two steps in flight: consecutive steps (independent batches on different buffer sets) issued on two
+    # streams in turn, each with library contexts of its own, so that the ragged end of one step's launches and
+    # the start of the next share the GPU.  Reported beside the headline, which runs one step at a time.
+    overlapped = None
+    if world == 1 and not args.no_once and args.lanes == 1:
+        wb2 = Workbench(sentry, w, dev, local_rank, rank, not args.no_overlap, not args.no_graph,
+                        ATTEND_KERNELS[args.attend_kernel], lanes=2)
+        b2 = wb2.time_blocks(args.steps, max(3, args.replays // 2 + 1), args.warmup)
+        ms2 = float(np.median(b2)) / args.steps
+        overlapped = {"value": wm["tokens"] / (ms2 * 1e-3), "unit": "tokens/s", "ms_per_step": ms2, "steps_in_flight": 2,
+                      "device_status": wb2.status(),
+                      "what": "the same steps, issued alternately on two streams (two independent batches in flight); "
+                              "ms_per_step = block time / steps"}
+        wb2.close()
 
     # ---- end to end: pinned host buffers in, results out, every step
     ids, masks, subsets, los, sh, sc, tbl, offs, W1, W2 = (wb.ids, wb.masks, wb.subsets, wb.los, wb.sh, wb.sc,
@@ -846,6 +894,7 @@ def run_ours(args, w: synth.Workload):
                    "l2_policy": "rotating %d resident buffer sets, %.0f MB in total (> 126 MB L2)"
                                 % (n_sets, n_sets * set_bytes / 1e6),
                    "cuda_graph": graphs_on,
+                   "steps_in_flight": args.lanes,
                    "streams": "attention branch and FFN branch forked inside the step" if two_streams
                               else "one stream",
                    "attend_kernel": args.attend_kernel,
@@ -860,7 +909,7 @@ def run_ours(args, w: synth.Workload):
                              "and timed with CUDA events" % (args.replays, args.steps)},
         "block_ms": blocks, "replays": args.replays,
         "useful_tflops": (wm["att_flops"] + wm["ffn_flops"]) * world * args.steps / (ms * 1e-3) / 1e12,
-        "materialised_once": once, "chained_layer": chained,
+        "materialised_once": once, "two_steps_in_flight": overlapped, "chained_layer": chained,
         "e2e": None if e2e_ms is None else {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": n_e2e,
                 "pipeline": "%d sample chunks; upload, kernels and download on three streams, consecutive steps overlapping chunk by chunk" % n_chunks},
@@ -902,6 +951,8 @@ def main():
                          "(score_mode 2), plainly transposed (score_mode 2), or query-major as generated (score_mode 0); "
                          "auto: arranged where K and V of a group fit in shared memory, transposed otherwise; "
                          "the sampled sets are the same")
+    ap.add_argument("--lanes", type=int, default=1,
+                    help="streams that consecutive steps are issued on in turn (independent batches; 1 = one step at a time)")
     ap.add_argument("--side", default=None, choices=["moe", "ffn_fp8"],
                     help="run only this side measurement of the configs table and print its object (for profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
