@@ -152,6 +152,26 @@ def test_config4_full_layer_all_subsets(sn):
     _run_workload(sn, w, "all", "all")
 
 
+# d_model = 384: the tiles of a partial last round are shared by three CTAs each (a 128-column third
+# of Y per CTA) when three times their number fits one round of 148 CTAs.  Three batch sizes put the
+# kernel in each regime: every tile shared (B = 12: 32 tiles), two whole rounds of none and a shared
+# third (B = 64: 170 tiles = 148 + 22), a partial round too large to share (B = 78: 208 = 148 + 60).
+@pytest.mark.parametrize("B", [12, 64, 78])
+def test_ffn_d384_column_split_regimes(sn, B):
+    w = synth.config4().with_(B=B, name="cfg4_B%d" % B)
+    inp = synth.generate(w, n_s_of)
+    _, kept_c = parity.gate_lists(sn, inp)
+    strat = parity.stratified_samples(inp, 2)
+    err = parity.ffn_parity(sn, inp, kept_c, strat, full_batch=True)
+    assert err <= TOL["bf16"], (w.name, err)
+    # and twice the same bits
+    X, W1, W2 = inp.X.cuda(), inp.W1.cuda(), inp.W2.cuda()
+    los, ids, masks = dev(inp.list_of_sample), dev(inp.ids), masks_dev(inp.masks)
+    Y1 = sn.ffn_fwd(X, W1, W2, kept_c, los, ids, masks)
+    Y2 = sn.ffn_fwd(X, W1, W2, kept_c, los, ids, masks)
+    assert torch.equal(Y1, Y2)
+
+
 # All 16 cells of the throughput sweep.  Up to 2^18 tokens every sample is checked; beyond that
 # the call runs on the whole batch (inputs drawn on the device) and the oracle checks two samples
 # of each of the 7 modality subsets.
