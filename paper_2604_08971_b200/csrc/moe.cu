@@ -100,6 +100,87 @@ moe_offsets_kernel(const int32_t* __restrict__ counts, int E, int tile_rows, Ffn
     }
 }
 
+// The whole plan in ONE launch by one block, for small calls (latency: one launch instead of a
+// memset and three): count per expert in shared memory, prefix sums, then a second walk that hands
+// out the positions (one shared-memory atomic per warp and expert in both walks).
+constexpr int kPlanOneThreads = 1024;
+constexpr long long kPlanOneMaxSlots = 8192;   // one round of the block; beyond it one SM is the slower way (65 536 slots: 53 us)
+__global__ void __launch_bounds__(kPlanOneThreads)
+moe_plan_one_kernel(const int32_t* __restrict__ expert_ids, int n_slots, int E, int top_k, int tile_rows,
+                    FfnPlan plan, unsigned int* status) {
+    extern __shared__ int s_int[];
+    int* s_cnt = s_int;          // [E] slots per expert
+    int* s_cur = s_int + E;      // [E] next free row of the expert
+    const int lane = threadIdx.x & 31;
+    for (int e = threadIdx.x; e < E; e += blockDim.x) s_cnt[e] = 0;
+    __syncthreads();
+    bool bad = false;
+    const int per_round = (int)blockDim.x * 8;   // eight ids per thread are requested together
+    for (int i0 = 0; i0 < n_slots; i0 += per_round) {
+        int ev[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = i0 + j * (int)blockDim.x + (int)threadIdx.x;
+            ev[j] = i < n_slots ? __ldg(expert_ids + i) : -1;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            int e = ev[j];
+            if (e < -1 || e >= E) { bad = true; e = -1; }
+            const unsigned peers = __match_any_sync(0xffffffffu, e);
+            if (e >= 0 && lane == __ffs(peers) - 1) atomicAdd(&s_cnt[e], __popc(peers));
+        }
+    }
+    if (bad) atomicOr(status, SENTRY_STATUS_BIT_BAD_INDEX);
+    __syncthreads();
+    if (threadIdx.x < 32) {   // exclusive prefix sums over the experts, 32 at a time
+        int row0 = 0, tile0 = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane;
+            const int c = e < E ? s_cnt[e] : 0;
+            const int t = (c + tile_rows - 1) / tile_rows;
+            int ic = c, it = t;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int vc = __shfl_up_sync(0xffffffffu, ic, o), vt = __shfl_up_sync(0xffffffffu, it, o);
+                if (lane >= o) { ic += vc; it += vt; }
+            }
+            if (e < E) {
+                plan.list_row0[e] = row0 + ic - c;
+                plan.tile_start[e] = tile0 + it - t;
+                s_cur[e] = row0 + ic - c;
+            }
+            row0 += __shfl_sync(0xffffffffu, ic, 31);
+            tile0 += __shfl_sync(0xffffffffu, it, 31);
+        }
+        if (lane == 0) { plan.list_row0[E] = row0; plan.tile_start[E] = tile0; }
+    }
+    __syncthreads();
+    for (int i0 = 0; i0 < n_slots; i0 += per_round) {
+        int ev[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = i0 + j * (int)blockDim.x + (int)threadIdx.x;
+            ev[j] = i < n_slots ? __ldg(expert_ids + i) : -1;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = i0 + j * (int)blockDim.x + (int)threadIdx.x;
+            int e = ev[j];
+            if (e < -1 || e >= E) e = -1;
+            const unsigned peers = __match_any_sync(0xffffffffu, e);
+            const int leader = __ffs(peers) - 1;
+            int base = 0;
+            if (e >= 0 && lane == leader) base = atomicAdd(&s_cur[e], __popc(peers));
+            const int pos = __shfl_sync(0xffffffffu, base, leader) + __popc(peers & ((1u << lane) - 1u));
+            if (e >= 0) {
+                plan.rowidx[pos] = i / top_k;   // row of X: the token
+                plan.rowout[pos] = i;           // row of the staging buffer: (token, slot)
+            }
+        }
+    }
+}
+
 template <typename T> struct Vec16;
 template <> struct Vec16<float> { static constexpr int N = 4; };
 template <> struct Vec16<__nv_bfloat16> { static constexpr int N = 8; };
@@ -259,13 +340,17 @@ int launch_moe_ffn(sentry_ctx* ctx, const MoeArgs& m, void* ws, size_t ws_bytes,
     const unsigned route_blocks = (unsigned)((slots + kPlanThreads * 8 - 1) / (kPlanThreads * 8));
     const size_t route_smem = (size_t)2 * d.E * sizeof(int);
 
-    SENTRY_CUDA_TRY(cudaMemsetAsync(w.counts, 0, (size_t)d.E * sizeof(int32_t), st));
     if (packed == nullptr) {
         int rc = launch_moe_prepack(ctx, m, w.packed, st);
         if (rc != SENTRY_OK) return rc;
         packed = w.packed;
     }
-    {
+    if (slots <= kPlanOneMaxSlots && route_smem <= 48 * 1024) {
+        LaunchScope ls(ctx, KS_MOE_PLAN, st);
+        moe_plan_one_kernel<<<1, kPlanOneThreads, route_smem, st>>>(m.expert_ids, (int)slots, d.E, d.top_k, tile_rows,
+                                                                    w.plan, m.status);
+    } else {
+        SENTRY_CUDA_TRY(cudaMemsetAsync(w.counts, 0, (size_t)d.E * sizeof(int32_t), st));
         LaunchScope ls(ctx, KS_MOE_PLAN, st, 3);
         moe_route_kernel<<<route_blocks, kPlanThreads, route_smem, st>>>(m.expert_ids, slots, d.E, d.top_k, 0,
                                                                          w.counts, w.cursor, w.plan, m.status);

@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
 CASES = [
     ("moe_small_f32", 301, 64, 192, 5, 2, 96, "f32", 1.0, 0.0),
     ("moe_tc_d256", 2500, 256, 1024, 8, 2, 512, "bf16", 1.0, 0.0),        # several tiles per expert + tails
+    ("moe_tc_d256_multi_block_plan", 6000, 256, 1024, 8, 2, 512, "bf16", 1.0, 0.05),   # > 8192 slots: count / offsets / scatter launches
     ("moe_tc_d384_top4", 1111, 384, 768, 16, 4, 300, "bf16", 1.5, 0.1),   # k_c padded to a chunk; dropped slots
     ("moe_tc_d128_idle", 700, 128, 512, 32, 1, 256, "bf16", 3.0, 0.0),    # top-1, most experts nearly idle
     ("moe_alu_bf16_d72", 257, 72, 200, 3, 2, 77, "bf16", 0.0, 0.2),       # shape outside the tensor-core path
