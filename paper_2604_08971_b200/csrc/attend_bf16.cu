@@ -643,18 +643,32 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
         const int lane_ = threadIdx.x & 31, wid_ = threadIdx.x >> 5, nw_ = blockDim.x >> 5;
         if (threadIdx.x < 33) s_cls[threadIdx.x] = 0;
         __syncthreads();
-        for (int bb = threadIdx.x; bb < Bn; bb += blockDim.x) atomicAdd(&s_cls[__popc(masks[bb])], 1);
-        __syncthreads();
-        if (threadIdx.x == 0) {   // class (present modalities, descending) that holds rank b, and the offset in it
-            int left = b, cls = 32;
-            while (cls > 0 && left >= s_cls[cls]) { left -= s_cls[cls]; --cls; }
-            s_pick[0] = cls;
-            s_pick[1] = left;
+        // samples per class (number of present modalities): one shared-memory atomic per warp and class
+        for (int b0 = 0; b0 < Bn; b0 += blockDim.x) {
+            const int bb = b0 + threadIdx.x;
+            const int c = bb < Bn ? __popc(masks[bb]) : -1;
+            const unsigned peers = __match_any_sync(0xffffffffu, c);
+            if (c >= 0 && lane_ == __ffs(peers) - 1) atomicAdd(&s_cls[c], __popc(peers));
         }
         __syncthreads();
-        const int cls = s_pick[0];
-        int need = s_pick[1];      // the need-th sample of that class, in index order
-        __syncthreads();
+        // every warp for itself: the class that holds rank b, classes descending (lane l <-> class 32 - l;
+        // what no lane claims is class 0), and the offset in it
+        int cls, need;
+        {
+            const int mine = s_cls[32 - lane_];
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane_ >= o) incl += v;
+            }
+            const int above = incl - mine;
+            const unsigned hit = __ballot_sync(0xffffffffu, above <= b && b < incl);
+            const int src = hit ? __ffs(hit) - 1 : 31;
+            const int above_src = __shfl_sync(0xffffffffu, above, src), incl_src = __shfl_sync(0xffffffffu, incl, src);
+            cls = hit ? 32 - src : 0;
+            need = hit ? b - above_src : b - incl_src;   // the need-th sample of that class, in index order
+        }
         for (int b0 = 0; b0 < Bn; b0 += blockDim.x) {
             const int bb = b0 + threadIdx.x;
             const bool hit = bb < Bn && __popc(masks[bb]) == cls;
@@ -668,7 +682,6 @@ attend_fused_bf16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat1
             if (need < tot) break;
             need -= tot;
         }
-        __syncthreads();
         b = s_pick[0];
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
