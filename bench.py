@@ -590,49 +590,66 @@ def quick_moe(sentry, dev: str, local_rank: int, peaks):
 
 
 def quick_fp8_ffn(sentry, dev: str, local_rank: int, peaks):
-    """The FFN of workload 3 (65 536 rows, d_model 256, 512 of 1024 channels kept) with FP8 e4m3 operands
+    """The FFN of workload 3 (65 536 rows, d_model 256, 512 of 1024 channels kept, one list) and of workload 4
+    (43 520 present rows, d_model 384, 614 of 1536 channels kept, three lists) with FP8 e4m3 operands
     (sentry_ffn_fwd_fp8, weights prepacked once) beside the same call in bf16 (sentry_ffn_fwd_packed):
     median of 5 blocks of 20 calls on rotating inputs larger than L2.  FLOPs as for bf16: 4 D k_c per row."""
-    w = synth.config3()
-    rng = np.random.default_rng(5)
     sn = sentry.Sentry(local_rank)
-    kept = torch.as_tensor(np.sort(rng.permutation(w.F)[:w.k_c]).astype(np.int32)[None, :], device=dev)
-    n_sets = 8
-    Xb = [torch.randn((w.B, w.T, w.D), device=dev).to(torch.bfloat16) for _ in range(n_sets)]
-    Xq = [(x.float() * 100.0).to(torch.float8_e4m3fn).view(torch.uint8) for x in Xb]
-    W1 = (torch.randn((w.D, w.F), device=dev) * 0.02).to(torch.bfloat16)
-    W2 = (torch.randn((w.F, w.D), device=dev) * 0.02).to(torch.bfloat16)
-    W1q = (W1.float() * 5000.0).to(torch.float8_e4m3fn).view(torch.uint8)
-    W2q = (W2.float() * 5000.0).to(torch.float8_e4m3fn).view(torch.uint8)
-    Y = [torch.empty((w.B, w.T, w.D), dtype=torch.bfloat16, device=dev) for _ in range(n_sets)]
-    p16 = sn.ffn_prepack(W1, W2, kept)
-    p8 = sn.ffn_prepack_e4m3(W1q, W2q, kept)
-    flops = 4.0 * w.D * w.k_c * w.B * w.T
-    out = {"workload": "ffn of cfg3 (65536 rows, D=256, k_c=512), weights materialised once"}
-    for name in ("bf16", "fp8_e4m3"):
-        def run(i):
-            if name == "bf16":
-                sn.ffn_fwd_packed(Xb[i % n_sets], p16, w.F, w.k_c, 1, Y=Y[i % n_sets])
-            else:
-                sn.ffn_fwd_fp8(Xq[i % n_sets], p8, w.F, w.k_c, 1, 0.01, 2e-4, 2e-4, 0.01, Y=Y[i % n_sets])
-        for i in range(5):
-            run(i)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        blocks = []
-        for r in range(5):
-            e0.record()
-            for i in range(20):
-                run(r * 20 + i)
-            e1.record()
+    out = {}
+    for key, w in (("cfg3", synth.config3()), ("cfg4", synth.config4())):
+        rng = np.random.default_rng(5)
+        inp = synth.generate(w, lambda tv: sentry.num_active_queries(tv, w.c), tensors=False)
+        n_lists = len(inp.subsets)
+        kept = torch.as_tensor(np.stack([np.sort(rng.permutation(w.F)[:w.k_c]) for _ in range(n_lists)]).astype(np.int32),
+                               device=dev)
+        los = torch.as_tensor(inp.list_of_sample, device=dev)
+        ids = torch.as_tensor(inp.ids, device=dev)
+        masks = torch.as_tensor(inp.masks.astype(np.int64).astype(np.int32), device=dev)
+        rows = int(sum(synth.present_count(w, int(m)) for m in inp.masks))
+        n_sets = 8
+        Xb = [torch.randn((w.B, w.T, w.D), device=dev).to(torch.bfloat16) for _ in range(n_sets)]
+        Xq = [(x.float() * 100.0).to(torch.float8_e4m3fn).view(torch.uint8) for x in Xb]
+        W1 = (torch.randn((w.D, w.F), device=dev) * 0.02).to(torch.bfloat16)
+        W2 = (torch.randn((w.F, w.D), device=dev) * 0.02).to(torch.bfloat16)
+        W1q = (W1.float() * 5000.0).to(torch.float8_e4m3fn).view(torch.uint8)
+        W2q = (W2.float() * 5000.0).to(torch.float8_e4m3fn).view(torch.uint8)
+        Y = [torch.empty((w.B, w.T, w.D), dtype=torch.bfloat16, device=dev) for _ in range(n_sets)]
+        p16 = sn.ffn_prepack(W1, W2, kept)
+        p8 = sn.ffn_prepack_e4m3(W1q, W2q, kept)
+        flops = 4.0 * w.D * w.k_c * rows
+        res = {"workload": "ffn of %s (%d present rows, D=%d, k_c=%d, %d lists), weights materialised once"
+                           % (w.name, rows, w.D, w.k_c, n_lists)}
+        for name in ("bf16", "fp8_e4m3"):
+            def run(i):
+                if name == "bf16":
+                    sn.ffn_fwd_packed(Xb[i % n_sets], p16, w.F, w.k_c, n_lists, los, ids, masks, Y=Y[i % n_sets])
+                else:
+                    sn.ffn_fwd_fp8(Xq[i % n_sets], p8, w.F, w.k_c, n_lists, 0.01, 2e-4, 2e-4, 0.01, los, ids, masks,
+                                   Y=Y[i % n_sets])
+            for i in range(5):
+                run(i)
             torch.cuda.synchronize()
-            blocks.append(e0.elapsed_time(e1) / 20)
-        ms = float(np.median(blocks))
-        out[name] = {"ms_per_call": ms, "tokens_per_s": w.B * w.T / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
-                     "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
-        if name == "fp8_e4m3":
-            # peak of its own operand type: the measured bf16 figure x the nominal 8-bit : 16-bit ratio (2)
-            out[name]["frac_of_fp8_peak"] = out[name]["frac_of_bf16_peak"] / 2.0
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            blocks = []
+            for r in range(5):
+                e0.record()
+                for i in range(20):
+                    run(r * 20 + i)
+                e1.record()
+                torch.cuda.synchronize()
+                blocks.append(e0.elapsed_time(e1) / 20)
+            ms = float(np.median(blocks))
+            res[name] = {"ms_per_call": ms, "tokens_per_s": rows / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
+                         "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+            if name == "fp8_e4m3":
+                # peak of its own operand type: the measured bf16 figure x the nominal 8-bit : 16-bit ratio (2)
+                res[name]["frac_of_fp8_peak"] = res[name]["frac_of_bf16_peak"] / 2.0
+        if key == "cfg3":
+            out.update(res)          # the first shape keeps its place at the top level of the object
+        else:
+            out[key] = res
+        del Xb, Xq, Y
+        torch.cuda.empty_cache()
     out["device_status"] = sn.last_status()
     sn.close()
     return out

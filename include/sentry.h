@@ -313,7 +313,7 @@ SENTRY_API int sentry_ffn_prepack(sentry_ctx* ctx, const sentry_ffn_desc* desc, 
 SENTRY_API int sentry_ffn_prepack_fp8(sentry_ctx* ctx, const sentry_ffn_desc* desc, const uint8_t* W1_e4m3,
                            const uint8_t* W2_e4m3, float scale_w1, float scale_w2,
                            const int32_t* kept_channels, void* packed, size_t packed_bytes, void* stream);
-/* FP8 ARITHMETIC (Sec. 5, the FP8 point taken to the tensor cores; desc->dtype = SENTRY_FP8_E4M3, D = 128 or 256):
+/* FP8 ARITHMETIC (Sec. 5, the FP8 point taken to the tensor cores; desc->dtype = SENTRY_FP8_E4M3, D = 128, 256 or 384):
  * X [B,T,D] and the weights are e4m3 codes with per-tensor scales scale_x, scale_w1, scale_w2; the hidden
  * activations are requantised to e4m3 with scale_h (a calibration constant of the caller); Y is bf16:
  *   z = (x_q . W1_q[:, N]) * (scale_x*scale_w1);  h_q = e4m3(gelu(z) / scale_h)   (nearest, saturating at 448)

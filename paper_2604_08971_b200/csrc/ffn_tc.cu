@@ -61,9 +61,12 @@ struct Cfg {
     static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
     static constexpr int SPG = (D == 384) ? 3 : KB1;   // weight stages per chunk of GEMM1 (= of GEMM2)
     static constexpr bool COLSPLIT = (D == 384) && !FP8;   // tail tiles shared by three CTAs, a third of Y each
-    static_assert(!FP8 || D == 256 || D == 128, "the FP8 form is built for d_model = 128 and 256");
+    // FP8 with d_model = 384: one 128-channel hidden block, written by all eight epilogue warps, and two more
+    // blocks that only stage Y on its way out (the hidden block is live while Y drains)
+    static constexpr bool FP8_384 = FP8 && D == 384;
+    static constexpr int NHS_ALLOC = FP8_384 ? 3 : NHS;
     static constexpr int OFF_H = NXS * kBlockBytes;
-    static constexpr int OFF_W = OFF_H + NHS * kBlockBytes;
+    static constexpr int OFF_W = OFF_H + NHS_ALLOC * kBlockBytes;
     static constexpr int OFF_MISC = OFF_W + kStages * kStageBytes;
     static constexpr int SMEM_BYTES = OFF_MISC + 2048 + 1024;  // + misc + alignment slack
     static_assert(SMEM_BYTES <= 232448, "shared memory over the per-CTA limit");
@@ -188,7 +191,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         ptx::mbar_init(ptx::smem_u32(&misc->h_full), 1);
         ptx::mbar_init(ptx::smem_u32(&misc->h_tmem_empty), kEpiWarps);
         for (int b = 0; b < 4; ++b) {
-            ptx::mbar_init(ptx::smem_u32(&misc->hs_full[b]), 4);   // one warp per TMEM lane quarter
+            ptx::mbar_init(ptx::smem_u32(&misc->hs_full[b]), C::FP8_384 ? 8 : 4);   // one warp per TMEM lane quarter (FP8, 384: both halves)
             ptx::mbar_init(ptx::smem_u32(&misc->hs_empty[b]), 1);
         }
         ptx::mbar_init(ptx::smem_u32(&misc->y_full), 1);
@@ -225,7 +228,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         }
         __syncwarp();
         // one stage = one 32 KB box, or two 16 KB boxes (x1 < 0: single box)
-        auto stage = [&](uint32_t n, const CUtensorMap* tm, int x0, int x1, int y) -> bool {
+        auto stage = [&](uint32_t n, const CUtensorMap* tm, int x0, int x1, int y, uint32_t bytes = kStageBytes) -> bool {
             const uint32_t sl = n % kStages, use = n / kStages;
             const uint32_t we = MISC_BAR(mb, w_empty) + 8u * sl;
             if (!__all_sync(0xffffffffu, ptx::mbar_try_wait(we, (use & 1u) ^ 1u)) &&
@@ -234,7 +237,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             if (elect_one()) {
                 const uint32_t bar = MISC_BAR(mb, w_full) + 8u * sl;
                 const uint32_t dst = wsm + sl * kStageBytes;
-                ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+                ptx::mbar_arrive_expect_tx(bar, bytes);
                 ptx::tma_load_2d(dst, tm, x0, y, bar);
                 if (x1 >= 0) ptx::tma_load_2d(dst + kBlockBytes, tm, x1, y, bar);
             }
@@ -259,7 +262,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < SPG; ++i) {
                     if (ok && ((n + i) & 1u) == me) {
-                        if constexpr (D == 384) ok = stage(n + i, &tm_w1, 128 * i, 128 * i + 64, y);
+                        if constexpr (C::FP8_384) ok = stage(n + i, &tm_w1, 64 * i, -1, y, kBlockBytes);   // one 128-byte K block of 128 channels
+                        else if constexpr (D == 384) ok = stage(n + i, &tm_w1, 128 * i, 128 * i + 64, y);
                         else ok = stage(n + i, &tm_w1, 64 * i, -1, y);
                     }
                 }
@@ -267,6 +271,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             }
             if (q > 0) {
                 const int pl = c ? l_cur : l_last, x = (c ? c - 1 : NC - 1) * C::CH16, y = pl * D;
+                if constexpr (C::FP8_384) {
+                    // the chunk is one K block: columns 0..255 of Y from an N = 256 stage, 256..383 from a 16 KB N = 128 stage
+                    if (ok && (n & 1u) == me) ok = stage(n, &tm_w2_256, x, -1, y);
+                    if (ok && ((n + 1) & 1u) == me) ok = stage(n + 1, &tm_w2_128, x, -1, y + 256, kBlockBytes);
+                    n += 2;
+                    if (++c == NC) { c = 0; ++ti; }
+                    continue;
+                }
                 if (C::COLSPLIT && my_third >= 0 && (int)(c ? ti : ti - 1) == my_tiles - 1) {
                     // a third of Y: one N = 128 stage (both K blocks of the chunk)
                     if ((n & 1u) == me) ok = stage(n, &tm_w2_128, x, x + 64, y + 128 * my_third);
@@ -353,7 +365,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                     if (!ok) continue;
                     const uint32_t he = (i == 0) ? MISC_BAR(mb, h_tmem_empty) : 0u;
                     const uint32_t hf = (i == SPG - 1) ? MISC_BAR(mb, h_full) : 0u;
-                    if constexpr (D == 384) {
+                    if constexpr (D == 384 && !FP8) {
                         const uint32_t s0 = 2 * i, s1 = 2 * i + 1;   // X slots (NXS = KB1 = 6)
                         ok = stage(n + i, tm_h, xs_lo + s0 * kBlkLo, xs_lo + s1 * kBlkLo, idesc128, i == 0,
                                    first ? MISC_BAR(mb, x_full) + 8u * s0 : 0u, ti & 1u,
@@ -362,7 +374,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                                    last ? MISC_BAR(mb, x_empty) + 8u * s1 : 0u, hf);
                     } else {
                         const uint32_t gx = ti * C::KB1 + i, slot = gx % C::NXS;
-                        ok = stage(n + i, tm_h, xs_lo + slot * kBlkLo, 0u, idesc256, i == 0,
+                        ok = stage(n + i, tm_h, xs_lo + slot * kBlkLo, 0u, C::CH == 256 ? idesc256 : idesc128, i == 0,
                                    first ? MISC_BAR(mb, x_full) + 8u * slot : 0u, (gx / C::NXS) & 1u, 0u, 0u, he, hp,
                                    i == 0, last ? MISC_BAR(mb, x_empty) + 8u * slot : 0u, 0u, hf);
                     }
@@ -376,6 +388,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 const bool first = (pc == 0), last = (pc == NC - 1);
                 const uint32_t ye = first ? MISC_BAR(mb, y_empty) : 0u, yp = (pti & 1u) ^ 1u;
                 const uint32_t yf = last ? MISC_BAR(mb, y_full) : 0u;
+                if constexpr (C::FP8_384) {
+                    ok = stage(n, tmem, hs_lo, 0u, idesc256, first, MISC_BAR(mb, hs_full), gp, 0u, 0u, ye, yp, first, 0u, 0u, 0u);
+                    if (ok)
+                        ok = stage(n + 1, tmem + 256u, hs_lo, 0u, idesc128, first, 0u, 0u, 0u, 0u, 0u, 0u, first,
+                                   MISC_BAR(mb, hs_empty), 0u, yf);
+                    n += 2;
+                    if (++c == NC) { c = 0; ++ti; }
+                    continue;
+                }
                 if (C::COLSPLIT && my_third >= 0 && (int)pti == my_tiles - 1) {
                     ok = stage(n, tmem + 128u * (uint32_t)my_third, hs_lo, hs_lo + kBlkLo, idesc128, first,
                                MISC_BAR(mb, hs_full), gp, MISC_BAR(mb, hs_full) + 8u, gp, ye, yp, first,
@@ -482,7 +503,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
         // next hidden block there) so that the global stores cover whole 128-byte row segments.
         constexpr int kDrainBlk = C::NBATCH - 1;
         // (FP8: a warp writes one 128-channel hidden block, rows of its own quarter: that piece)
-        const uint32_t stg = FP8 ? hs + (uint32_t)half * kBlockBytes + (uint32_t)quarter * 4096u
+        const uint32_t stg = C::FP8_384 ? hs + (uint32_t)(1 + half) * kBlockBytes + (uint32_t)quarter * 4096u
+                           : FP8 ? hs + (uint32_t)half * kBlockBytes + (uint32_t)quarter * 4096u
                                  : hs + (uint32_t)(half * C::NBATCH + kDrainBlk) * kBlockBytes + (uint32_t)quarter * 4096u;
         auto drain_y = [&](uint32_t t_idx, int32_t grow, int third) {
             if (!warp_wait(&misc->y_full, t_idx & 1u, abort_flag)) { ok = false; return; }
@@ -582,18 +604,21 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                             p8[8 + i] = gelu_pack_e4m3x4(__uint_as_float(h1[4 * i]) * a_scale, __uint_as_float(h1[4 * i + 1]) * a_scale,
                                                          __uint_as_float(h1[4 * i + 2]) * a_scale, __uint_as_float(h1[4 * i + 3]) * a_scale, h_inv);
                         }
-                        if (j == 0 && !warp_wait(&misc->hs_empty[half], (g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                        const uint32_t hrow8 = hs + half * kBlockBytes + row * 128;
+                        // (d_model 384: one hidden block for the chunk, this warp's 64 channels are bytes 64 half .. of a row)
+                        constexpr bool ONE = C::FP8_384;
+                        const int hb = ONE ? 0 : half, cb = ONE ? 4 * half : 4 * j;
+                        if (j == 0 && !warp_wait(&misc->hs_empty[hb], (g & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t hrow8 = hs + hb * kBlockBytes + row * 128;
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const uint32_t dst = hrow8 + (((4 * j + i) ^ (row & 7)) << 4);
+                            const uint32_t dst = hrow8 + (((cb + i) ^ (row & 7)) << 4);
                             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p8[4 * i]),
                                          "r"(p8[4 * i + 1]), "r"(p8[4 * i + 2]), "r"(p8[4 * i + 3])
                                          : "memory");
                         }
                         if (j == C::NBATCH - 1) {
                             ptx::fence_proxy_async_smem();
-                            warp_arrive(&misc->hs_full[half]);
+                            warp_arrive(&misc->hs_full[hb]);
                         }
                         continue;
                     }
@@ -677,7 +702,7 @@ int launch_fp8(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c
     const sentry_ffn_desc& d = a.d;
     CUtensorMap m1, m2a, m2b;
     const uint64_t r1 = (uint64_t)d.n_lists * kc_pad, r2 = (uint64_t)d.n_lists * D;
-    if (!make_weight_map(&m1, w1c, r1, D / 2, 256)) return SENTRY_ERR_CUDA;
+    if (!make_weight_map(&m1, w1c, r1, D / 2, Cfg<D, true>::CH == 256 ? 256 : 128)) return SENTRY_ERR_CUDA;
     if (!make_weight_map(&m2a, w2c, r2, kc_pad / 2, 256)) return SENTRY_ERR_CUDA;
     if (!make_weight_map(&m2b, w2c, r2, kc_pad / 2, 128)) return SENTRY_ERR_CUDA;
     auto kern = ffn_tc_kernel<D, false, true>;
@@ -693,10 +718,12 @@ int launch_fp8(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* w1c
 
 }  // namespace
 
-bool ffn_tc_fp8_supported(const sentry_ffn_desc& d) { return d.dtype == SENTRY_FP8_E4M3 && (d.D == 256 || d.D == 128); }
+bool ffn_tc_fp8_supported(const sentry_ffn_desc& d) {
+    return d.dtype == SENTRY_FP8_E4M3 && (d.D == 128 || d.D == 256 || d.D == 384);
+}
 
 bool ffn_tc_supported(const sentry_ffn_desc& d) {
-    if (d.dtype == SENTRY_FP8_E4M3) return d.D == 256 || d.D == 128;
+    if (d.dtype == SENTRY_FP8_E4M3) return d.D == 128 || d.D == 256 || d.D == 384;
     return (d.dtype == SENTRY_BF16 || d.dtype == SENTRY_F16) && (d.D == 128 || d.D == 256 || d.D == 384);
 }
 
@@ -720,7 +747,8 @@ int launch_ffn_tc(sentry_ctx* ctx, const FfnArgs& a, const FfnPlan& plan, void* 
     if (a.d.dtype == SENTRY_FP8_E4M3) {
         if (!ffn_tc_fp8_supported(a.d)) return SENTRY_ERR_UNSUPPORTED;
         rc = a.d.D == 256 ? launch_fp8<256>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)
-                          : launch_fp8<128>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st);
+             : a.d.D == 384 ? launch_fp8<384>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st)
+                            : launch_fp8<128>(ctx, a, plan, w1c, w2c, kc_pad, max_tiles, st);
         if (rc != SENTRY_OK) return rc;
         SENTRY_CUDA_TRY(cudaGetLastError());
         return SENTRY_OK;

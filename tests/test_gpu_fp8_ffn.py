@@ -44,7 +44,8 @@ def _quantise(t):
 
 
 @pytest.mark.parametrize("w", [synth.config3().with_(B=6), synth.config5(16, 256), synth.config5(3, 1024).with_(k_c=300, name="fp8_ragged_kc"),
-                               synth.config2().with_(B=24, name="fp8_d128"), synth.config2().with_(B=5, k_c=200, name="fp8_d128_ragged_kc")],
+                               synth.config2().with_(B=24, name="fp8_d128"), synth.config2().with_(B=5, k_c=200, name="fp8_d128_ragged_kc"),
+                               synth.config4().with_(B=12, name="fp8_d384"), synth.config4().with_(B=70, name="fp8_d384_two_tiles_per_cta")],
                          ids=lambda w: w.name)
 def test_fp8_ffn_against_the_oracle(w):
     sn = sentry.Sentry(0)
