@@ -60,7 +60,7 @@ struct Cfg {
     static constexpr int NHS = CH / EPB;               // hidden blocks per chunk
     static constexpr int NBATCH = CH / 128;            // 64-column batches per epilogue warp
     static constexpr int SPG = (D == 384) ? 3 : KB1;   // weight stages per chunk of GEMM1 (= of GEMM2)
-    static constexpr bool COLSPLIT = (D == 384) && !FP8;   // tail tiles shared by three CTAs, a third of Y each
+    static constexpr bool COLSPLIT = (D == 384);   // tail tiles shared by three CTAs, a third of Y each
     // FP8 with d_model = 384: one 128-channel hidden block, written by all eight epilogue warps, and two more
     // blocks that only stage Y on its way out (the hidden block is live while Y drains)
     static constexpr bool FP8_384 = FP8 && D == 384;
@@ -165,7 +165,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NC = kc_pad / C::CH;
     const int total_tiles = plan.tile_start[n_lists];
-    // Column-split tail (d_model = 384).  The tiles of the last, partial round leave most CTAs idle
+    // Column-split tail (d_model = 384, 16-bit and FP8 operands).  The tiles of the last, partial round leave most CTAs idle
     // (340 tiles on 148 CTAs: 44 in the third round).  When three times their number still fits
     // one round, each of them is taken by three CTAs: all three form the tile's hidden
     // activations, and each accumulates and stores one 128-column third of Y (GEMM2 of a third =
@@ -272,10 +272,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
             if (q > 0) {
                 const int pl = c ? l_cur : l_last, x = (c ? c - 1 : NC - 1) * C::CH16, y = pl * D;
                 if constexpr (C::FP8_384) {
-                    // the chunk is one K block: columns 0..255 of Y from an N = 256 stage, 256..383 from a 16 KB N = 128 stage
-                    if (ok && (n & 1u) == me) ok = stage(n, &tm_w2_256, x, -1, y);
-                    if (ok && ((n + 1) & 1u) == me) ok = stage(n + 1, &tm_w2_128, x, -1, y + 256, kBlockBytes);
-                    n += 2;
+                    if (my_third >= 0 && (int)(c ? ti : ti - 1) == my_tiles - 1) {
+                        // a third of Y: one 16 KB N = 128 stage
+                        if (ok && (n & 1u) == me) ok = stage(n, &tm_w2_128, x, -1, y + 128 * my_third, kBlockBytes);
+                        n += 1;
+                    } else {
+                        // the chunk is one K block: columns 0..255 of Y from an N = 256 stage, 256..383 from a 16 KB N = 128 stage
+                        if (ok && (n & 1u) == me) ok = stage(n, &tm_w2_256, x, -1, y);
+                        if (ok && ((n + 1) & 1u) == me) ok = stage(n + 1, &tm_w2_128, x, -1, y + 256, kBlockBytes);
+                        n += 2;
+                    }
                     if (++c == NC) { c = 0; ++ti; }
                     continue;
                 }
@@ -389,11 +395,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__
                 const uint32_t ye = first ? MISC_BAR(mb, y_empty) : 0u, yp = (pti & 1u) ^ 1u;
                 const uint32_t yf = last ? MISC_BAR(mb, y_full) : 0u;
                 if constexpr (C::FP8_384) {
-                    ok = stage(n, tmem, hs_lo, 0u, idesc256, first, MISC_BAR(mb, hs_full), gp, 0u, 0u, ye, yp, first, 0u, 0u, 0u);
-                    if (ok)
-                        ok = stage(n + 1, tmem + 256u, hs_lo, 0u, idesc128, first, 0u, 0u, 0u, 0u, 0u, 0u, first,
-                                   MISC_BAR(mb, hs_empty), 0u, yf);
-                    n += 2;
+                    if (my_third >= 0 && (int)pti == my_tiles - 1) {
+                        ok = stage(n, tmem + 128u * (uint32_t)my_third, hs_lo, 0u, idesc128, first, MISC_BAR(mb, hs_full), gp,
+                                   0u, 0u, ye, yp, first, MISC_BAR(mb, hs_empty), 0u, yf);
+                        n += 1;
+                    } else {
+                        ok = stage(n, tmem, hs_lo, 0u, idesc256, first, MISC_BAR(mb, hs_full), gp, 0u, 0u, ye, yp, first, 0u, 0u, 0u);
+                        if (ok)
+                            ok = stage(n + 1, tmem + 256u, hs_lo, 0u, idesc128, first, 0u, 0u, 0u, 0u, 0u, 0u, first,
+                                       MISC_BAR(mb, hs_empty), 0u, yf);
+                        n += 2;
+                    }
                     if (++c == NC) { c = 0; ++ti; }
                     continue;
                 }
